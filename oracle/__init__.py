@@ -1,0 +1,194 @@
+"""Python face of the CPU oracle (oracle/vt_oracle.c).  TEST INFRASTRUCTURE ONLY.
+
+Only tests, the smoke check and the benchmark's CPU-baseline leg may import this package; the
+product package never does.  It compiles the C file with gcc on first use and calls it through
+ctypes on numpy arrays.  Nothing here touches CUDA.
+
+Parity pins: see the header of vt_oracle.c -- pinned to definitions, invariants, library special
+cases and brute force by the CPU tests; parity with paper-printed values is unpinned because
+the paper prints no numeric example for this path.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from ctypes import POINTER, c_double, c_float, c_int, c_int32, c_int64, c_uint16, c_uint64, c_void_p
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "vt_oracle.c")
+_LIB = os.path.join(_HERE, "libvt_oracle.so")
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (OpenMP only parallelises independent vocabulary rows)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + ".%d.tmp" % os.getpid()
+        subprocess.check_call(["gcc", "-O2", "-std=c11", "-fopenmp", "-fPIC", "-shared",
+                               "-o", tmp, _SRC, "-lm"])
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        _lib = ctypes.CDLL(build())
+        _lib.orc_softmax_row.restype = c_double
+        _lib.orc_gumbel_row.restype = c_int32
+        _lib.orc_max_threads.restype = c_int
+    return _lib
+
+
+def _p(a, ty):
+    return a.ctypes.data_as(POINTER(ty)) if a is not None else None
+
+
+def _c(a, dtype):
+    return np.ascontiguousarray(a, dtype=dtype)
+
+
+def _bits(a) -> np.ndarray:
+    """Accept raw bf16 bit patterns as uint16/int16 numpy arrays."""
+    a = np.ascontiguousarray(a)
+    if a.dtype == np.int16:
+        a = a.view(np.uint16)
+    assert a.dtype == np.uint16, "bf16 data must be passed as 16-bit patterns"
+    return a
+
+
+def max_threads() -> int:
+    return int(_load().orc_max_threads())
+
+
+def set_threads(t: int) -> None:
+    _load().orc_set_threads(c_int(int(t)))
+
+
+def decode_bf16(x) -> np.ndarray:
+    x = _bits(x)
+    out = np.empty(x.shape, dtype=np.float64)
+    _load().orc_decode_bf16(_p(x, c_uint16), c_int64(x.size), _p(out, c_double))
+    return out
+
+
+def histogram(ids, V: int, counts=None):
+    """Algorithm 1.  Returns (counts uint64 [V], n_bad).  Passing `counts` accumulates into it."""
+    ids = _c(ids, np.int32)
+    acc = counts is not None
+    if not acc:
+        counts = np.empty(V, dtype=np.uint64)
+    assert counts.dtype == np.uint64 and counts.size == V and counts.flags.c_contiguous
+    bad = c_uint64(0)
+    _load().orc_histogram(_p(ids, c_int32), c_int64(ids.size), c_int32(V), _p(counts, c_uint64),
+                          c_int(1 if acc else 0), ctypes.byref(bad))
+    return counts, int(bad.value)
+
+
+def select_topk(counts, K: int):
+    """Eq. 1, line 1.  Returns (map int32 [K] in rank order, inv_map int32 [V])."""
+    counts = _c(counts, np.uint64)
+    V = counts.size
+    m = np.empty(K, dtype=np.int32)
+    inv = np.empty(V, dtype=np.int32)
+    rc = _load().orc_select_topk(_p(counts, c_uint64), c_int32(V), c_int32(K), _p(m, c_int32),
+                                 _p(inv, c_int32))
+    if rc:
+        raise ValueError("select_topk: invalid V/K")
+    return m, inv
+
+
+def build_vocab(ids, V: int, K: int):
+    counts, bad = histogram(ids, V)
+    m, inv = select_topk(counts, K)
+    return m, inv, counts, bad
+
+
+def trim_head(W_full, map_):
+    """Eq. 1, line 2.  W_full: bf16 bit patterns [V,d]; returns bit patterns [K,d]."""
+    W_full = _bits(W_full)
+    map_ = _c(map_, np.int32)
+    K, d = map_.size, W_full.shape[1]
+    out = np.empty((K, d), dtype=np.uint16)
+    _load().orc_trim_head(_p(W_full, c_uint16), _p(map_, c_int32), c_int32(K), c_int32(d),
+                          _p(out, c_uint16))
+    return out
+
+
+def logits(h, W) -> np.ndarray:
+    """fp64 projection of bf16 rows h [B,d] onto bf16 head W [K,d]; returns [B,K]."""
+    h, W = _bits(h), _bits(W)
+    B, d = h.shape
+    K = W.shape[0]
+    assert W.shape[1] == d
+    out = np.empty((B, K), dtype=np.float64)
+    _load().orc_logits(_p(h, c_uint16), _p(W, c_uint16), c_int32(B), c_int32(K), c_int32(d),
+                       _p(out, c_double))
+    return out
+
+
+def softmax_row(logit, T: float):
+    """Returns (z = logit/T, lse) for one row."""
+    logit = _c(logit, np.float64)
+    z = np.empty_like(logit)
+    lse = _load().orc_softmax_row(_p(logit, c_double), c_int32(logit.size), c_double(float(T)),
+                                  _p(z, c_double))
+    return z, float(lse)
+
+
+def topk_row(z, topk: int) -> np.ndarray:
+    z = _c(z, np.float64)
+    idx = np.empty(topk, dtype=np.int32)
+    _load().orc_topk_row(_p(z, c_double), c_int32(z.size), c_int32(topk), _p(idx, c_int32))
+    return idx
+
+
+def gumbel_row(z, u):
+    """Returns (argmax index, score = z + g) for one row."""
+    z = _c(z, np.float64)
+    u = _c(u, np.float32)
+    score = np.empty_like(z)
+    j = _load().orc_gumbel_row(_p(z, c_double), _p(u, c_float), c_int32(z.size),
+                               _p(score, c_double))
+    return int(j), score
+
+
+class DraftHeadResult:
+    __slots__ = ("ids", "logprobs", "trim", "logits", "z", "lse", "score")
+
+
+def draft_head(h, W_trim, map_, temp, topk: int, uniforms=None, want_full: bool = True):
+    """Algorithm 2 lines 5-6, head part.  h [B,d], W_trim [K,d] as bf16 bit patterns; map_ int32
+    [K] or None (identity); temp fp32 [B]; uniforms fp32 [B,K] or None.  Returns ids/logprobs of
+    shape [B,1+topk] plus (when want_full) logits, z, lse and Gumbel scores for margin checks."""
+    h, W_trim = _bits(h), _bits(W_trim)
+    B, d = h.shape
+    K = W_trim.shape[0]
+    temp = _c(temp, np.float32)
+    assert temp.size == B
+    if map_ is not None:
+        map_ = _c(map_, np.int32)
+        assert map_.size == K
+    if uniforms is not None:
+        uniforms = _c(uniforms, np.float32)
+        assert uniforms.shape == (B, K)
+    r = DraftHeadResult()
+    r.ids = np.empty((B, 1 + topk), dtype=np.int32)
+    r.logprobs = np.empty((B, 1 + topk), dtype=np.float64)
+    r.trim = np.empty((B, 1 + topk), dtype=np.int32)
+    r.logits = np.empty((B, K), dtype=np.float64) if want_full else None
+    r.z = np.empty((B, K), dtype=np.float64) if want_full else None
+    r.lse = np.empty(B, dtype=np.float64)
+    r.score = np.empty((B, K), dtype=np.float64) if (want_full and uniforms is not None) else None
+    rc = _load().orc_draft_head(_p(h, c_uint16), _p(W_trim, c_uint16), _p(map_, c_int32),
+                                c_int32(B), c_int32(K), c_int32(d), _p(temp, c_float),
+                                c_int32(topk), _p(uniforms, c_float), _p(r.ids, c_int32),
+                                _p(r.logprobs, c_double), _p(r.trim, c_int32),
+                                _p(r.logits, c_double), _p(r.z, c_double), _p(r.lse, c_double),
+                                _p(r.score, c_double))
+    if rc:
+        raise ValueError("draft_head: invalid shape arguments")
+    return r

@@ -1,0 +1,323 @@
+"""Pins for the CPU oracle: every oracle function is checked against something other than
+itself -- a closed form, an invariant, a library routine on a special case, or brute force on
+tiny inputs -- chosen so that a dropped term, a wrong sign or index, or a transposed operand
+fails at least one of them.  No GPU is involved."""
+import itertools
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import vt_inputs
+
+
+def _bits(t: torch.Tensor) -> np.ndarray:
+    return vt_inputs.bf16_bits(t.contiguous()).numpy().view(np.uint16)
+
+
+# ----------------------------------------------------------------------------- bf16 decode
+def test_bf16_decode_all_patterns_match_torch():
+    pats = torch.arange(0, 65536, dtype=torch.int32).to(torch.int16)
+    ref = pats.view(torch.bfloat16).to(torch.float64).numpy()
+    got = oracle.decode_bf16(pats.numpy())
+    finite = np.isfinite(ref)
+    assert np.array_equal(got[finite], ref[finite])
+    assert np.array_equal(np.isnan(got), np.isnan(ref))
+    assert np.array_equal(np.isinf(got), np.isinf(ref))
+    # two hand values: 0x3F80 = 1.0, 0xC048 = -3.125
+    assert oracle.decode_bf16(np.array([0x3F80, 0xC048], dtype=np.uint16)).tolist() == [1.0, -3.125]
+
+
+# ----------------------------------------------------------------------------- histogram (Algorithm 1)
+def test_histogram_hand_example():
+    ids = np.array([3, 1, 3, 3, 0, 7, 1, -1, 8, 5], dtype=np.int32)  # V = 8: -1 and 8 are invalid
+    counts, bad = oracle.histogram(ids, 8)
+    assert counts.tolist() == [1, 2, 0, 3, 0, 1, 0, 1]
+    assert bad == 2
+
+
+def test_histogram_matches_bincount_and_sums_to_n():
+    ids = vt_inputs.zipf_ids(200_000, 4096, 1.1, seed=11, noise_frac=0.05).numpy()
+    counts, bad = oracle.histogram(ids, 4096)
+    assert bad == 0
+    assert int(counts.sum()) == ids.size
+    assert np.array_equal(counts, np.bincount(ids, minlength=4096).astype(np.uint64))
+    assert np.array_equal(counts.astype(np.int64),
+                          torch.bincount(torch.from_numpy(ids).long(), minlength=4096).numpy())
+
+
+def test_histogram_accumulates_over_chunks():
+    ids = vt_inputs.zipf_ids(50_000, 1000, 1.07, seed=5).numpy()
+    whole, _ = oracle.histogram(ids, 1000)
+    part, _ = oracle.histogram(ids[:20_000], 1000)
+    part, _ = oracle.histogram(ids[20_000:], 1000, counts=part)
+    assert np.array_equal(whole, part)
+
+
+# ----------------------------------------------------------------------------- top-K (Eq. 1, line 1)
+def _rank_by_definition(counts):
+    """rank(v) = #{u : c_u > c_v or (c_u == c_v and u < v)} -- no sort involved."""
+    V = len(counts)
+    return [sum(1 for u in range(V) if counts[u] > counts[v] or (counts[u] == counts[v] and u < v))
+            for v in range(V)]
+
+
+def test_topk_exhaustive_tiny_against_rank_definition():
+    for V in range(1, 7):
+        for cv in itertools.product((0, 1, 2), repeat=V):
+            rank = _rank_by_definition(cv)
+            for K in range(1, V + 1):
+                m, inv = oracle.select_topk(np.array(cv, dtype=np.uint64), K)
+                for v in range(V):
+                    if rank[v] < K:
+                        assert m[rank[v]] == v and inv[v] == rank[v]
+                    else:
+                        assert inv[v] == -1
+
+
+def test_topk_brute_force_best_subset():
+    """The kept set must maximise the total count over all K-subsets (exhaustive enumeration)."""
+    rng = np.random.default_rng(3)
+    for _ in range(20):
+        V, K = 9, int(rng.integers(1, 9))
+        c = rng.integers(0, 5, size=V).astype(np.uint64)
+        m, _ = oracle.select_topk(c, K)
+        best = max(int(sum(c[list(s)])) for s in itertools.combinations(range(V), K))
+        assert int(c[m].sum()) == best
+
+
+def test_topk_invariants_with_massive_ties():
+    ids = vt_inputs.zipf_ids(100_000, 4096, 1.1, seed=1001).numpy()
+    counts, _ = oracle.histogram(ids, 4096)
+    K = 1024
+    m, inv = oracle.select_topk(counts, K)
+    assert len(set(m.tolist())) == K
+    kept = counts[m].astype(np.int64)
+    assert np.all(np.diff(kept) <= 0)                        # counts non-increasing along the map
+    same = np.diff(kept) == 0
+    assert np.all(np.diff(m.astype(np.int64))[same] > 0)     # equal counts => ascending ids
+    pruned = np.setdiff1d(np.arange(4096), m)
+    assert kept.min() >= counts[pruned].max()
+    cut = kept.min()                                          # ties at the cut: lower ids are kept
+    tied_kept = m[kept == cut]
+    tied_pruned = pruned[counts[pruned] == cut]
+    if tied_pruned.size:
+        assert tied_kept.max() < tied_pruned.min()
+    assert np.array_equal(inv[m], np.arange(K))
+    assert int((inv >= 0).sum()) == K
+
+
+def test_topk_tie_free_matches_stable_argsort():
+    rng = np.random.default_rng(7)
+    c = rng.permutation(5000).astype(np.uint64)               # all counts distinct
+    m, _ = oracle.select_topk(c, 777)
+    assert np.array_equal(m, np.argsort(-c.astype(np.int64), kind="stable")[:777].astype(np.int32))
+
+
+def test_topk_fewer_seen_ids_than_K_fills_tail_in_id_order():
+    c = np.zeros(16, dtype=np.uint64)
+    c[[9, 2, 13]] = [5, 7, 5]
+    m, inv = oracle.select_topk(c, 8)
+    assert m.tolist() == [2, 9, 13, 0, 1, 3, 4, 5]
+    assert inv[6] == -1 and inv[0] == 3
+
+
+def test_topk_K_equals_V_is_a_permutation():
+    c = np.array([1, 1, 1, 1], dtype=np.uint64)
+    m, inv = oracle.select_topk(c, 4)
+    assert m.tolist() == [0, 1, 2, 3] and inv.tolist() == [0, 1, 2, 3]
+
+
+# ----------------------------------------------------------------------------- gather (Eq. 1, line 2)
+def test_trim_head_is_a_bit_copy_of_the_mapped_rows():
+    W = _bits(vt_inputs.gaussian_bf16((50, 24), 0.02, seed=2))
+    m = np.array([7, 0, 49, 7, 13], dtype=np.int32)
+    Wt = oracle.trim_head(W, m)
+    assert Wt.shape == (5, 24)
+    for j, v in enumerate(m):
+        assert np.array_equal(Wt[j], W[v])
+    ident = np.arange(50, dtype=np.int32)
+    assert np.array_equal(oracle.trim_head(W, ident), W)
+
+
+# ----------------------------------------------------------------------------- logits (Algorithm 2, line 5)
+def test_logits_match_numpy_fp64_matmul_nonsquare():
+    h = _bits(vt_inputs.gaussian_bf16((3, 40), 1.0, seed=4))
+    W = _bits(vt_inputs.gaussian_bf16((17, 40), 0.02, seed=5))
+    got = oracle.logits(h, W)
+    ref = oracle.decode_bf16(h) @ oracle.decode_bf16(W).T      # [B,d] x [d,K]: a transposed operand cannot pass
+    ref_t = (vt_inputs.gaussian_bf16((3, 40), 1.0, seed=4).double()
+             @ vt_inputs.gaussian_bf16((17, 40), 0.02, seed=5).double().T).numpy()
+    assert got.shape == (3, 17)
+    assert np.allclose(got, ref, rtol=0, atol=1e-12)
+    assert np.allclose(got, ref_t, rtol=0, atol=1e-12)
+
+
+def test_logits_exact_on_small_integers():
+    rng = np.random.default_rng(9)
+    hi = rng.integers(-4, 5, size=(2, 16))
+    Wi = rng.integers(-4, 5, size=(11, 16))
+    h = _bits(torch.from_numpy(hi).to(torch.bfloat16))
+    W = _bits(torch.from_numpy(Wi).to(torch.bfloat16))
+    assert np.array_equal(oracle.logits(h, W), (hi @ Wi.T).astype(np.float64))
+
+
+def test_trimmed_logits_equal_full_logits_at_mapped_rows_exactly():
+    V, d, K = 300, 64, 77
+    W = _bits(vt_inputs.gaussian_bf16((V, d), 0.02, seed=6))
+    h = _bits(vt_inputs.gaussian_bf16((4, d), 1.0, seed=7))
+    ids = vt_inputs.zipf_ids(5000, V, 1.1, seed=8).numpy()
+    m, inv, _, _ = oracle.build_vocab(ids, V, K)
+    full = oracle.logits(h, W)
+    trim = oracle.logits(h, oracle.trim_head(W, m))
+    assert np.array_equal(trim, full[:, m])                    # same fp64 operation order: bit equal
+
+
+def test_identity_map_reproduces_the_full_head():
+    V, d = 200, 32
+    W = _bits(vt_inputs.gaussian_bf16((V, d), 0.02, seed=16))
+    h = _bits(vt_inputs.gaussian_bf16((2, d), 1.0, seed=17))
+    T = np.array([1.0, 0.7], dtype=np.float32)
+    u = vt_inputs.uniforms((2, V), seed=18).numpy()
+    ident = np.arange(V, dtype=np.int32)
+    a = oracle.draft_head(h, W, None, T, 5, u)
+    b = oracle.draft_head(h, oracle.trim_head(W, ident), ident, T, 5, u)
+    assert np.array_equal(a.ids, b.ids) and np.array_equal(a.logprobs, b.logprobs)
+    assert np.array_equal(a.ids, a.trim)
+
+
+# ----------------------------------------------------------------------------- softmax
+def test_softmax_sums_to_one_and_is_shift_invariant():
+    rng = np.random.default_rng(12)
+    logit = rng.normal(0, 3, size=5000)
+    for T in (1.0, 0.7, 1.5):
+        z, lse = oracle.softmax_row(logit, T)
+        assert np.array_equal(z, logit / T)
+        p = np.exp(z - lse)
+        assert abs(p.sum() - 1.0) < 1e-12
+        z2, lse2 = oracle.softmax_row(logit + 5.0 * T, T)
+        assert np.allclose(z2 - lse2, z - lse, rtol=0, atol=1e-12)
+
+
+def test_softmax_matches_torch_log_softmax_fp64():
+    rng = np.random.default_rng(13)
+    logit = rng.normal(0, 2, size=3000)
+    for T in (1.0, 0.5, 2.0):
+        z, lse = oracle.softmax_row(logit, T)
+        ref = torch.log_softmax(torch.from_numpy(logit) / T, dim=0).numpy()
+        assert np.allclose(z - lse, ref, rtol=0, atol=1e-12)
+
+
+def test_softmax_closed_form_two_classes():
+    z, lse = oracle.softmax_row(np.array([0.0, math.log(3.0)]), 1.0)
+    assert abs(math.exp(z[1] - lse) - 0.75) < 1e-15 and abs(lse - math.log(4.0)) < 1e-15
+    # temperature 2 halves the logits: p = sqrt(3) / (1 + sqrt(3))
+    z, lse = oracle.softmax_row(np.array([0.0, math.log(3.0)]), 2.0)
+    assert abs(math.exp(z[1] - lse) - math.sqrt(3) / (1 + math.sqrt(3))) < 1e-15
+
+
+# ----------------------------------------------------------------------------- top-k candidates
+def test_topk_row_brute_force_and_ties_to_lower_index():
+    rng = np.random.default_rng(14)
+    for _ in range(50):
+        K = int(rng.integers(1, 9))
+        z = rng.integers(0, 4, size=K).astype(np.float64)     # many ties
+        k = int(rng.integers(1, K + 1))
+        ref = sorted(range(K), key=lambda j: (-z[j], j))[:k]
+        assert oracle.topk_row(z, k).tolist() == ref
+    z = rng.normal(size=1000)
+    idx = oracle.topk_row(z, 10)
+    assert idx[0] == int(np.argmax(z))
+    assert np.array_equal(idx, torch.topk(torch.from_numpy(z), 10).indices.numpy())
+    assert set(idx.tolist()) == set(np.nonzero(z >= z[idx[-1]])[0].tolist())
+
+
+# ----------------------------------------------------------------------------- Gumbel-max
+def test_gumbel_equal_uniforms_is_greedy_and_dominant_logit_always_wins():
+    rng = np.random.default_rng(15)
+    z = rng.normal(size=500)
+    for uval in (0.01, 0.5, 0.99):
+        j, _ = oracle.gumbel_row(z, np.full(500, uval, dtype=np.float32))
+        assert j == int(np.argmax(z))
+    z2 = z.copy()
+    z2[123] = 1e4
+    j, _ = oracle.gumbel_row(z2, vt_inputs.uniforms((500,), seed=3).numpy())
+    assert j == 123
+
+
+def test_gumbel_score_closed_form_and_clamp():
+    # u = 1/e gives g = -log(1) = 0;  u = exp(-exp(-2)) gives g = 2
+    u = np.array([math.exp(-1.0), math.exp(-math.exp(-2.0))], dtype=np.float32)
+    _, score = oracle.gumbel_row(np.array([0.25, -1.0]), u)
+    assert abs(score[0] - 0.25) < 1e-6 and abs(score[1] - 1.0) < 1e-6
+    # u = 0 and u = 1 are clamped to 2^-24 and 1 - 2^-24: finite scores with the right signs
+    _, score = oracle.gumbel_row(np.zeros(2), np.array([0.0, 1.0], dtype=np.float32))
+    assert np.all(np.isfinite(score))
+    assert abs(score[0] + math.log(24 * math.log(2.0))) < 1e-12
+    assert abs(score[1] + math.log(-math.log1p(-2.0 ** -24))) < 1e-9
+    # ties resolve to the first maximal index
+    j, _ = oracle.gumbel_row(np.zeros(4), np.full(4, 0.3, dtype=np.float32))
+    assert j == 0
+
+
+def test_gumbel_draws_follow_softmax_chi_square():
+    z = np.array([0.0, 0.5, 1.0, -1.0, 2.0, 0.3, -0.7, 1.4])
+    p = np.exp(z - np.log(np.exp(z).sum()))
+    n = 100_000
+    u = vt_inputs.uniforms((n, 8), seed=77).numpy()
+    hits = np.zeros(8)
+    for i in range(n):
+        j, _ = oracle.gumbel_row(z, u[i])
+        hits[j] += 1
+    chi2 = float((((hits - n * p) ** 2) / (n * p)).sum())
+    assert chi2 < 24.3                                           # 7 dof, p = 0.001
+
+
+def test_gumbel_restriction_property():
+    """Sampling over the kept set with the kept uniforms equals the full-vocabulary Gumbel
+    argmax restricted to the kept set."""
+    V, K = 400, 90
+    rng = np.random.default_rng(21)
+    zfull = rng.normal(size=V)
+    u = vt_inputs.uniforms((V,), seed=22).numpy()
+    kept = np.sort(rng.choice(V, K, replace=False))
+    _, score_full = oracle.gumbel_row(zfull, u)
+    j, _ = oracle.gumbel_row(zfull[kept], u[kept])
+    assert kept[j] == kept[int(np.argmax(score_full[kept]))]
+
+
+# ----------------------------------------------------------------------------- full head + remap
+def test_draft_head_outputs_are_consistent_with_its_parts():
+    V, d, K, B, topk = 512, 64, 128, 3, 4
+    W = _bits(vt_inputs.gaussian_bf16((V, d), 0.02, seed=31))
+    h = _bits(vt_inputs.gaussian_bf16((B, d), 1.0, seed=32))
+    ids = vt_inputs.zipf_ids(20_000, V, 1.1, seed=33).numpy()
+    m, inv, _, _ = oracle.build_vocab(ids, V, K)
+    Wt = oracle.trim_head(W, m)
+    T = np.array([1.0, 0.7, 1.3], dtype=np.float32)
+    u = vt_inputs.uniforms((B, K), seed=34).numpy()
+    r = oracle.draft_head(h, Wt, m, T, topk, u)
+    lg = oracle.logits(h, Wt)
+    assert np.array_equal(r.logits, lg)
+    for b in range(B):
+        z, lse = oracle.softmax_row(lg[b], float(T[b]))
+        assert np.array_equal(r.trim[b, 1:], oracle.topk_row(z, topk))
+        assert r.trim[b, 1] == int(np.argmax(z))
+        g, _ = oracle.gumbel_row(z, u[b])
+        assert r.trim[b, 0] == g
+        assert np.allclose(r.logprobs[b], z[r.trim[b]] - lse, rtol=0, atol=0)
+        ref = torch.log_softmax(torch.from_numpy(lg[b]) / float(T[b]), 0).numpy()
+        assert np.allclose(r.logprobs[b], ref[r.trim[b]], rtol=0, atol=1e-12)
+    assert np.array_equal(r.ids, m[r.trim])                     # remap T_{d->t}
+    assert np.array_equal(inv[r.ids], r.trim)                   # inverse map recovers the trimmed index
+    greedy = oracle.draft_head(h, Wt, m, T, topk, None)
+    assert np.array_equal(greedy.ids[:, 0], greedy.ids[:, 1])   # no uniforms: column 0 is the greedy id
+
+
+def test_draft_head_rejects_bad_shapes():
+    W = np.zeros((4, 8), dtype=np.uint16)
+    h = np.zeros((1, 8), dtype=np.uint16)
+    with pytest.raises(ValueError):
+        oracle.draft_head(h, W, None, np.ones(1, dtype=np.float32), 5, None)
