@@ -1,0 +1,437 @@
+#!/usr/bin/env python
+"""Benchmark of the VocabTrim hot path on B200.
+
+Headline (the JSON line's `value`): microseconds per draft step of the trimmed drafter LM head on
+the Llama-3.2-3B-class workload (V=128256, d=3072, K=32768, B=1, greedy + top-8 log-probs),
+one `vt_draft_head` call per step, inputs resident in HBM, W_trim rotated over several copies so
+that every step reads its weights from HBM and not from L2.
+
+Also on the line: `e2e` (same step through `vt_draft_head_host`: pinned host inputs copied in and
+results copied out every step), `roofline` (achieved HBM GB/s of the head kernel against the
+measured copy bandwidth), `cpu_baseline` (the fp64 CPU oracle timed on a bounded sample), `clocks`
+(SM clock and throttle reasons sampled during the timed region), `gpu_launches`, and, at N=1, the
+sweep of K for the tree-drafting head, the full-vocabulary head and the corpus-scale vocabulary
+build (Gtok/s).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--no-extras]
+
+With N > 1 (launched under torch.distributed.run) every rank runs an independent replica of the
+same step on its own GPU; the path has no exchange step, so there is no collective in the data
+path (only the barrier and the max-over-ranks of the timing).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import vt_inputs  # noqa: E402
+
+V = vt_inputs.LLAMA3_VOCAB
+HEAD = dict(d=3072, K=32768, B=1, topk=8, temp=1.0)            # BASELINE config 2 (chain drafting)
+TREE = dict(d=4096, B=10, topk=10, temp=0.7)                   # BASELINE config 3 (tree drafting)
+TREE_KS = (8192, 16384, 32768, 65536, V)
+L2_BYTES = 126 * 1024 * 1024
+FALLBACK_HBM_GBS = 6650.0
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the head kernel on the headline
+# workload, from the ncu capture summarised under profiles/ (None until a capture exists).
+NCU_TRAFFIC_BYTES = {"k_head_skinny": None, "k_hist_hot": None}
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            return json.load(open(p)), "measured"
+        except Exception:
+            pass
+    return {"hbm_gbs": FALLBACK_HBM_GBS, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}, "fallback"
+
+
+# --------------------------------------------------------------------------------------------------
+class ClockSampler:
+    """Samples SM clock and throttle reasons of one GPU through NVML while a region runs."""
+
+    SLOW_BITS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown",
+                 0x4: "sw_power_cap", 0x80: "hw_power_brake"}
+
+    def __init__(self, device_index: int, period_s: float = 0.02):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self.period, self._stop, self._thr, self._h = period_s, threading.Event(), None, None
+        try:
+            import pynvml
+            self.nv = pynvml
+            pynvml.nvmlInit()
+            try:
+                props = torch.cuda.get_device_properties(device_index)
+                bus = "%08X:%02X:%02X.0" % (props.pci_domain_id, props.pci_bus_id, props.pci_device_id)
+                self._h = pynvml.nvmlDeviceGetHandleByPciBusId(bus.encode())
+            except Exception:
+                self._h = pynvml.nvmlDeviceGetHandleByIndex(device_index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self._h = None
+
+    def _loop(self):
+        nv = self.nv
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM)))
+                mask = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self._h))
+                for bit, name in self.SLOW_BITS.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            self._stop.wait(self.period)
+
+    def __enter__(self):
+        if self._h is not None:
+            self._thr = threading.Thread(target=self._loop, daemon=True)
+            self._thr.start()
+        return self
+
+    def __exit__(self, *exc):
+        self._stop.set()
+        if self._thr is not None:
+            self._thr.join()
+
+    def summary(self):
+        s = sorted(self.samples)
+        return {"sm_mhz": (s[len(s) // 2] if s else None), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(s)}
+
+
+def _events():
+    return torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+
+def _copies_for_cold_l2(nbytes: int) -> int:
+    """Number of distinct copies of a weight matrix to rotate through so that at least 8x the L2
+    capacity is streamed between two uses of the same copy."""
+    return max(2, -(-8 * L2_BYTES // nbytes) + 1)
+
+
+# --------------------------------------------------------------------------------------------------
+def build_head_workload(vt, dev, d, K, B, topk, temp, sample, seed, use_map=True, pool=16):
+    """W_full -> map (from 1e7 synthetic ids through vt_build_vocab) -> W_trim copies, h pool, uniforms."""
+    W_full = vt_inputs.gaussian_bf16((V, d), 0.02, seed=seed, device=dev)
+    if K == V or not use_map:
+        map_, W_trim = None, W_full[:K].contiguous() if K != V else W_full
+    else:
+        ids = vt_inputs.zipf_ids(10_000_000, V, 1.07, seed=seed + 100, noise_frac=0.05, device=dev)
+        map_, _ = vt.vt_build_vocab(ids, V, K)
+        W_trim = vt.vt_trim_head(W_full, map_)
+        del ids
+    nbytes = K * d * 2
+    copies = [W_trim] + [W_trim.clone() for _ in range(_copies_for_cold_l2(nbytes) - 1)]
+    if W_trim is not W_full:
+        del W_full
+    hs = [vt_inputs.gaussian_bf16((B, d), 1.0, seed=seed + 1000 + i, device=dev) for i in range(pool)]
+    us = [vt_inputs.uniforms((B, K), seed=seed + 2000 + i, device=dev) for i in range(4)] if sample else None
+    T = vt_inputs.temperatures(B, temp, temp, 0, device=dev)
+    out = (torch.empty((B, 1 + topk), dtype=torch.int32, device=dev),
+           torch.empty((B, 1 + topk), dtype=torch.float32, device=dev))
+    ws = vt.Workspace(vt.workspace_bytes(vt.VT_OP_DRAFT_HEAD_HOST, 0, 0, K, d, B, topk), dev)
+    return dict(copies=copies, map=map_, hs=hs, us=us, T=T, out=out, ws=ws, K=K, d=d, B=B, topk=topk,
+                algo_bytes=K * d * 2 + B * d * 2 + (B * K * 4 if sample else 0) + 2 * B * (1 + topk) * 4)
+
+
+def run_head_steps(vt, wl, steps, start=0):
+    copies, hs, us = wl["copies"], wl["hs"], wl["us"]
+    for i in range(start, start + steps):
+        vt.vt_draft_head(hs[i % len(hs)], copies[i % len(copies)], wl["map"], wl["T"], wl["topk"],
+                         us[i % len(us)] if us else None, ws=wl["ws"], out=wl["out"])
+
+
+def time_head(vt, wl, steps, warmup):
+    run_head_steps(vt, wl, warmup)
+    torch.cuda.synchronize()
+    e0, e1 = _events()
+    e0.record()
+    run_head_steps(vt, wl, steps, start=warmup)
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / steps          # ms per step
+
+
+def time_head_e2e(vt, wl, steps, warmup):
+    """Same step through vt_draft_head_host: pinned host inputs, results read back every step."""
+    B, K, d, topk = wl["B"], wl["K"], wl["d"], wl["topk"]
+    hs = [h.cpu().pin_memory() for h in wl["hs"]]
+    us = [u.cpu().pin_memory() for u in wl["us"]] if wl["us"] else None
+    T = wl["T"].cpu().pin_memory()
+    out = (torch.empty((B, 1 + topk), dtype=torch.int32).pin_memory(),
+           torch.empty((B, 1 + topk), dtype=torch.float32).pin_memory())
+    copies = wl["copies"]
+    sink = 0
+
+    def step(i):
+        nonlocal sink
+        vt.vt_draft_head_host(hs[i % len(hs)], copies[i % len(copies)], wl["map"], T, topk,
+                              us[i % len(us)] if us else None, wl["ws"], out)
+        torch.cuda.current_stream().synchronize()       # the caller consumes the ids before the next step
+        sink ^= int(out[0][0, 0])
+
+    for i in range(warmup):
+        step(i)
+    torch.cuda.synchronize()
+    e0, e1 = _events()
+    e0.record()
+    for i in range(warmup, warmup + steps):
+        step(i)
+    e1.record()
+    torch.cuda.synchronize()
+    h2d = B * d * 2 + B * 4 + (B * K * 4 if us else 0)
+    d2h = 2 * B * (1 + topk) * 4
+    return e0.elapsed_time(e1) / steps, h2d, d2h
+
+
+# --------------------------------------------------------------------------------------------------
+def oracle_head_rate(wl, seconds=12.0, rows=None):
+    """Times the CPU oracle on a bounded sample (the first `rows` vocabulary rows) of one head step;
+    returns (us per FULL step scaled by K/rows, rows used, threads, repetitions)."""
+    import numpy as np
+
+    import oracle
+
+    K, B, topk = wl["K"], wl["B"], wl["topk"]
+    Wb = vt_inputs.bf16_bits(wl["copies"][0]).cpu().numpy().view(np.uint16)
+    hb = vt_inputs.bf16_bits(wl["hs"][0]).cpu().numpy().view(np.uint16)
+    T = wl["T"].cpu().numpy()
+    u = wl["us"][0].cpu().numpy() if wl["us"] else None
+    rows = K if rows is None else max(topk, min(K, rows))
+    Ws = Wb[:rows]
+    us = None if u is None else np.ascontiguousarray(u[:, :rows])
+    t0 = time.perf_counter()
+    reps = 0
+    while True:
+        oracle.draft_head(hb, Ws, None, T, topk, us, want_full=False)
+        reps += 1
+        el = time.perf_counter() - t0
+        if el >= seconds or (reps >= 3 and el >= seconds / 2):
+            break
+    return el / reps * 1e6 * (K / rows), rows, oracle.max_threads(), reps
+
+
+def run_reference(args, rank):
+    """`--impl reference`: the CPU oracle as it stands, timed on the host cores on the headline
+    workload; every step is a bounded sample (a prefix of the vocabulary rows) scaled to a full step."""
+    if rank != 0:
+        return
+    import numpy as np
+
+    import oracle
+
+    d, K, B, topk = HEAD["d"], HEAD["K"], HEAD["B"], HEAD["topk"]
+    W = vt_inputs.gaussian_bf16((K, d), 0.02, seed=1002)
+    hs = [vt_inputs.gaussian_bf16((B, d), 1.0, seed=3000 + i) for i in range(8)]
+    Wb = vt_inputs.bf16_bits(W).numpy().view(np.uint16)
+    hb = [vt_inputs.bf16_bits(h).numpy().view(np.uint16) for h in hs]
+    T = np.full(B, HEAD["temp"], dtype=np.float32)
+    # calibrate rows/s, then size the per-step sample so the whole run stays near two minutes
+    t0 = time.perf_counter()
+    oracle.draft_head(hb[0], Wb[:4096], None, T, topk, None, want_full=False)
+    per_row = (time.perf_counter() - t0) / 4096
+    total_steps = args.steps + args.warmup
+    rows = int(max(64, min(K, 120.0 / max(1, total_steps) / per_row)))
+    Ws = np.ascontiguousarray(Wb[:rows])
+    for i in range(args.warmup):
+        oracle.draft_head(hb[i % 8], Ws, None, T, topk, None, want_full=False)
+    t0 = time.perf_counter()
+    for i in range(args.steps):
+        oracle.draft_head(hb[i % 8], Ws, None, T, topk, None, want_full=False)
+    el = time.perf_counter() - t0
+    us = el / args.steps * 1e6 * (K / rows)
+    sample = "first %d of %d vocabulary rows per step, time scaled by K/rows" % (rows, K)
+    line = {"impl": "reference", "metric": "drafter_lm_head_us_per_step", "value": us, "unit": "us",
+            "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": us / 1e3,
+            "higher_is_better": False, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+            "data": "synthetic", "config": head_config(),
+            "cpu_baseline": {"value": us, "unit": "us", "cores": oracle.max_threads(), "kind": "oracle",
+                             "sample": sample},
+            "e2e": {"value": us, "unit": "us", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def head_config():
+    return {"workload": "config2: Llama-3.2-3B-class drafter head, V=128256 d=3072 K=32768 B=1 topk=8 "
+                        "T=1 greedy+top-8 (chain drafting, one vt_draft_head per step)",
+            "V": V, "d": HEAD["d"], "K": HEAD["K"], "B": HEAD["B"], "topk": HEAD["topk"],
+            "cold_l2": "W_trim rotated over distinct copies (>= 8x L2 streamed between reuses)",
+            "parallelism": "replicas"}
+
+
+# --------------------------------------------------------------------------------------------------
+def extras(vt, dev, peak_gbs):
+    """K sweep of the tree-drafting head, the full-vocabulary chain head, and the vocabulary build."""
+    out = {}
+    sweep = []
+    for K in TREE_KS:
+        wl = build_head_workload(vt, dev, TREE["d"], K, TREE["B"], TREE["topk"], TREE["temp"], True,
+                                 seed=1003)
+        n = max(50, min(2000, int(0.25 / (K * TREE["d"] * 2 / 5e12))))
+        ms = time_head(vt, wl, n, 20)
+        gbs = wl["algo_bytes"] / (ms * 1e-3) / 1e9
+        sweep.append({"K": K, "us_per_step": ms * 1e3, "gbs": gbs, "frac_of_measured": gbs / peak_gbs,
+                      "frac_of_8000": gbs / 8000.0})
+        del wl
+        torch.cuda.empty_cache()
+    out["tree_head_k_sweep"] = {"workload": "config3: d=4096 B=10 topk=10 T=0.7 Gumbel sampling, cold L2",
+                                "points": sweep}
+    wl = build_head_workload(vt, dev, HEAD["d"], V, HEAD["B"], HEAD["topk"], HEAD["temp"], False, seed=1002)
+    ms = time_head(vt, wl, 300, 20)
+    gbs = wl["algo_bytes"] / (ms * 1e-3) / 1e9
+    out["full_head"] = {"workload": "config2 with the untrimmed head K=V=128256", "us_per_step": ms * 1e3,
+                        "gbs": gbs, "frac_of_measured": gbs / peak_gbs}
+    del wl
+    torch.cuda.empty_cache()
+    # vocabulary build at corpus scale
+    n = 1_000_000_000
+    ids = vt_inputs.zipf_ids(n, V, 1.07, seed=1005, noise_frac=0.05, device=dev)
+    ws = vt.Workspace(vt.workspace_bytes(vt.VT_OP_BUILD_VOCAB, n, V, 32768), dev)
+    counts = torch.empty(V, dtype=torch.int32, device=dev)
+
+    def timed(fn, reps=5, warm=2):
+        for _ in range(warm):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = _events()
+        e0.record()
+        for _ in range(reps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / reps
+
+    ms_h = timed(lambda: vt.vt_histogram(ids, V, counts=counts, ws=ws))
+    vb = {"workload": "config5: 1e9 int32 ids, V=128256, 95% Zipf(1.07) + 5% uniform",
+          "histogram_ms": ms_h, "histogram_gtok_s": n / (ms_h * 1e-3) / 1e9,
+          "histogram_gbs": 4.0 * n / (ms_h * 1e-3) / 1e9}
+    vb["histogram_frac_of_measured"] = vb["histogram_gbs"] / peak_gbs
+    vb["histogram_frac_of_8000"] = vb["histogram_gbs"] / 8000.0
+    for K in (8192, 32768):
+        ms_b = timed(lambda: vt.vt_build_vocab(ids, V, K, ws=ws))
+        vb["build_vocab_K%d_ms" % K] = ms_b
+        vb["build_vocab_K%d_gtok_s" % K] = n / (ms_b * 1e-3) / 1e9
+    ms_s = timed(lambda: vt.vt_select_topk(counts, 32768, ws=ws), reps=20)
+    vb["select_topk_K32768_us"] = ms_s * 1e3
+    del ids
+    torch.cuda.empty_cache()
+    W_full = vt_inputs.gaussian_bf16((V, 4096), 0.02, seed=1006, device=dev)
+    map_, _ = vt.vt_select_topk(counts, 32768, ws=ws)
+    W_trim = torch.empty((32768, 4096), dtype=torch.bfloat16, device=dev)
+    ms_g = timed(lambda: vt.vt_trim_head(W_full, map_, W_trim), reps=20)
+    vb["trim_head_K32768_d4096_us"] = ms_g * 1e3
+    vb["trim_head_gbs"] = 2 * 32768 * 4096 * 2 / (ms_g * 1e-3) / 1e9
+    vb["trim_head_frac_of_measured"] = vb["trim_head_gbs"] / peak_gbs
+    out["vocab_build"] = vb
+    return out
+
+
+# --------------------------------------------------------------------------------------------------
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20000)
+    ap.add_argument("--warmup", type=int, default=200)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-extras", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(3, args.warmup)
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the product has no CPU path")
+    import paper_2506_22694_b200 as vt
+    from paper_2506_22694_b200 import build as vt_build
+
+    vt_build.build()
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    peaks, peak_kind = measured_peaks()
+    peak_gbs = float(peaks["hbm_gbs"])
+    wl = build_head_workload(vt, dev, HEAD["d"], HEAD["K"], HEAD["B"], HEAD["topk"], HEAD["temp"], False,
+                             seed=1002)
+    run_head_steps(vt, wl, args.warmup)
+    torch.cuda.synchronize()
+    if dist:
+        dist.barrier()
+    launches0 = vt.launch_count()
+    with ClockSampler(local) as clk:
+        torch.cuda.synchronize()
+        e0, e1 = _events()
+        e0.record()
+        run_head_steps(vt, wl, args.steps, start=args.warmup)
+        e1.record()
+        torch.cuda.synchronize()
+    launches = vt.launch_count() - launches0
+    if dist:
+        dist.barrier()
+    ms_total = e0.elapsed_time(e1)
+    t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
+    if dist:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_step = float(t.item()) / args.steps
+    e2e_ms, h2d, d2h = time_head_e2e(vt, wl, max(200, min(args.steps, 5000)), 50)
+    t2 = torch.tensor([e2e_ms], dtype=torch.float64, device=dev)
+    if dist:
+        dist.all_reduce(t2, op=dist.ReduceOp.MAX)
+    e2e_ms = float(t2.item())
+    st, flags, _ = wl["ws"].read_status()
+    if st != 0:
+        raise SystemExit("device-side status after the timed region: %s (flags %d)" % (vt.status_str(st), flags))
+
+    gbs = wl["algo_bytes"] / (ms_step * 1e-3) / 1e9
+    line = {
+        "metric": "drafter_lm_head_us_per_step", "value": ms_step * 1e3, "unit": "us", "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": False,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": head_config(),
+        "e2e": {"value": e2e_ms * 1e3, "unit": "us", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+        "gpu_launches": int(launches), "clocks": clk.summary(),
+        "hbm_gbs": gbs, "hbm_gbs_aggregate": gbs * world,
+        "roofline": {"kernel": "k_head_skinny", "bound": "hbm", "achieved": gbs, "peak": peak_gbs, "unit": "GB/s",
+                     "frac": gbs / peak_gbs, "frac_of_8000": gbs / 8000.0, "peak_source": peak_kind,
+                     "algorithmic_bytes_per_launch": wl["algo_bytes"],
+                     "traffic": NCU_TRAFFIC_BYTES["k_head_skinny"]},
+    }
+    if rank == 0 and world == 1:
+        if not args.no_cpu_baseline:
+            us, rows, threads, reps = oracle_head_rate(wl, seconds=12.0)
+            line["cpu_baseline"] = {"value": us, "unit": "us", "cores": threads, "kind": "oracle",
+                                    "sample": "%d full head steps (all %d rows) of the same workload" % (reps, rows)}
+        del wl
+        torch.cuda.empty_cache()
+        if not args.no_extras:
+            line.update(extras(vt, dev, peak_gbs))
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    if dist:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

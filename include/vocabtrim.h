@@ -1,0 +1,171 @@
+/*
+ * vocabtrim.h -- C ABI of the B200 (sm_100a) VocabTrim hot path.
+ *
+ * The library implements the two paths of the method:
+ *   offline  : token-frequency counting (Algorithm 1), selection of the K most frequent target
+ *              vocabulary ids and reconstruction of the drafter LM head (Eq. 1);
+ *   online   : the drafter's trimmed LM head with its token sampling and the index mapper back
+ *              to the target vocabulary (Algorithm 2, lines 5-6).
+ *
+ * Conventions (all entry points unless stated otherwise)
+ *   - Every data pointer is a DEVICE pointer owned by the caller.  Entry points whose name ends
+ *     in _host take HOST pointers where their comment says so.
+ *   - The library allocates no device memory and keeps no global state.  Scratch comes from the
+ *     caller: `ws` is a device buffer of at least vt_workspace_bytes(op, ...) bytes, 256-byte
+ *     aligned, whose first 256 bytes (the control block) must have been cleared ONCE by
+ *     vt_workspace_init before its first use.  Every call leaves the control block ready for the
+ *     next call.  One workspace serves one stream at a time.
+ *   - Calls enqueue work on `stream` (a cudaStream_t passed as void*, NULL = default stream) and
+ *     return right after launching.  Argument errors return synchronously without launching.
+ *   - Data-dependent problems (token ids outside [0,V), map entries outside [0,V), non-positive
+ *     temperatures, NaN rows) never trap and never hang: they set sticky flag bits in the control
+ *     block, which vt_read_status reads back.
+ *   - bf16 tensors are passed as uint16_t bit patterns, row-major, 16-byte aligned base.
+ *   - K is the trimmed vocabulary size (rows of W_trim), V the full target vocabulary, d the
+ *     hidden size, B the number of hidden rows per call, topk the candidates per row.
+ *   - `map` is in RANK order: map[0] is the most frequent id, ties by count go to the lower id.
+ */
+#ifndef VOCABTRIM_H
+#define VOCABTRIM_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    VT_OK = 0,
+    VT_ERR_INVALID_ARG = 1, /* null pointer, size out of range, misaligned pointer          */
+    VT_ERR_RANGE = 2,       /* data-dependent: ids / map entries out of range (read_status) */
+    VT_ERR_WORKSPACE = 3,   /* ws is NULL, misaligned or smaller than vt_workspace_bytes    */
+    VT_ERR_CUDA = 4,        /* a CUDA runtime call failed                                   */
+    VT_ERR_TIMEOUT = 5,     /* a bounded device-side wait expired (read_status)             */
+    VT_ERR_UNSUPPORTED = 6, /* shape outside what the kernels support (see each call)       */
+    VT_ERR_NUMERIC = 7      /* data-dependent: non-positive temperature or NaN row          */
+} vt_status;
+
+/* Sticky flag bits kept in the workspace control block. */
+enum {
+    VT_FLAG_BAD_ID = 1u,   /* vt_histogram / vt_build_vocab saw ids outside [0,V); they were skipped */
+    VT_FLAG_BAD_MAP = 2u,  /* vt_trim_head saw map entries outside [0,V); those rows were zero-filled */
+    VT_FLAG_BAD_TEMP = 4u, /* vt_draft_head saw T <= 0, NaN or Inf; that row reports id -1, logprob NaN */
+    VT_FLAG_NAN_ROW = 8u,  /* vt_draft_head produced no finite candidate for a row (NaN inputs)        */
+    VT_FLAG_TIMEOUT = 16u  /* a bounded device-side wait expired                                      */
+};
+
+/* Operation selectors for vt_workspace_bytes. */
+enum {
+    VT_OP_HISTOGRAM = 0,
+    VT_OP_SELECT_TOPK = 1,
+    VT_OP_BUILD_VOCAB = 2,
+    VT_OP_TRIM_HEAD = 3,
+    VT_OP_DRAFT_HEAD = 4,
+    VT_OP_DRAFT_HEAD_HOST = 5,
+    VT_OP_BUILD_VOCAB_HOST = 6
+};
+
+#define VT_MAX_TOPK 64
+#define VT_CTRL_BYTES 256
+
+/* Scratch bytes needed by `op` for the given sizes (arguments an op does not use are ignored).
+ * Returns 0 for an unknown op or sizes the op rejects.  Pure host arithmetic. */
+size_t vt_workspace_bytes(int op, int64_t n, int32_t V, int32_t K, int32_t d, int32_t B,
+                          int32_t topk);
+
+/* Clears the control block (first VT_CTRL_BYTES bytes) of a workspace.  Call once after
+ * allocating `ws`, before any other call that takes it. */
+vt_status vt_workspace_init(void *ws, size_t ws_bytes, void *stream);
+
+/* Synchronises `stream`, copies the sticky flags (VT_FLAG_*) and the count of skipped token
+ * ids to the HOST locations `flags` / `n_bad` (either may be NULL), clears them on the device
+ * and returns VT_OK, VT_ERR_RANGE (bad ids / map entries), VT_ERR_NUMERIC or VT_ERR_TIMEOUT. */
+vt_status vt_read_status(void *ws, void *stream, uint32_t *flags, uint64_t *n_bad);
+
+const char *vt_status_str(vt_status s);
+
+/* Number of kernels launched by this library since it was loaded (host counter, for
+ * benchmarks that must report their launch count). */
+uint64_t vt_launch_count(void);
+
+/*
+ * Algorithm 1 (Count Token Frequencies): counts[t] += 1 for every id of the stream.
+ *   ids     [n] int32 (any alignment of 4), n >= 0, n < 2^32 per accumulated histogram
+ *   counts  [V] uint32; cleared first unless accumulate != 0 (chunked corpora)
+ * Ids outside [0,V) are skipped, counted (vt_read_status) and flagged VT_FLAG_BAD_ID.
+ * Integer work: the result is exact.
+ */
+vt_status vt_histogram(const int32_t *ids, int64_t n, int32_t V, uint32_t *counts,
+                       int accumulate, void *ws, size_t ws_bytes, void *stream);
+
+/*
+ * Eq. 1, first line: V_trim = V[Top-K(c,k)] from existing counts.
+ *   map     [K] int32: map[j] = id of rank j under (count descending, id ascending)
+ *   inv_map [V] int32: inv_map[map[j]] = j, -1 for pruned ids
+ * 1 <= K <= V.  Integer work: the result is exact and unique.
+ */
+vt_status vt_select_topk(const uint32_t *counts, int32_t V, int32_t K, int32_t *map,
+                         int32_t *inv_map, void *ws, size_t ws_bytes, void *stream);
+
+/* Algorithm 1 followed by Eq. 1, first line: vt_histogram then vt_select_topk (the counts live
+ * in the workspace). */
+vt_status vt_build_vocab(const int32_t *ids, int64_t n, int32_t V, int32_t K, int32_t *map,
+                         int32_t *inv_map, void *ws, size_t ws_bytes, void *stream);
+
+/* Same as vt_build_vocab with `ids` in HOST memory (pinned memory makes the copies
+ * asynchronous): the stream is copied to the device in chunks staged in the workspace, each
+ * chunk counted as it arrives.  map / inv_map stay device pointers. */
+vt_status vt_build_vocab_host(const int32_t *ids_host, int64_t n, int32_t V, int32_t K,
+                              int32_t *map, int32_t *inv_map, void *ws, size_t ws_bytes,
+                              void *stream);
+
+/*
+ * Eq. 1, second line: W_trim = W[Top-K(c,k), :], a bit copy of K rows.
+ *   W_full [V,d] bf16, W_trim [K,d] bf16, d % 8 == 0, map [K] int32.
+ * `ws` may be NULL; when given, map entries outside [0,V) are flagged VT_FLAG_BAD_MAP.  Such rows
+ * are zero-filled either way.
+ */
+vt_status vt_trim_head(const uint16_t *W_full, const int32_t *map, uint16_t *W_trim, int32_t V,
+                       int32_t K, int32_t d, void *ws, void *stream);
+
+/*
+ * Algorithm 2, lines 5-6, head part: logits = h W_trim^T (bf16 inputs, fp32 accumulation),
+ * z = logits / T_b, log-softmax statistics, the `topk` best candidates per row, a Gumbel-max
+ * draw argmax_j (z_j - log(-log u_bj)) and the index mapper T_{d->t} (trimmed index -> target id).
+ * Logits never leave the chip.
+ *   h        [B,d]  bf16            W_trim  [K,d] bf16
+ *   map      [K] int32 or NULL (identity: the untrimmed head)
+ *   temp     [B] fp32, T_b > 0      uniforms [B,K] fp32 or NULL (no sampling)
+ *   out_ids      [B, 1+topk] int32: column 0 = sampled id (greedy id if uniforms == NULL),
+ *                                   columns 1.. = candidates in descending z, ties to lower index
+ *   out_logprobs [B, 1+topk] fp32 : log softmax(logits/T_b) of the id in the same column
+ * Uniforms are clamped to [2^-24, 1-2^-24].  Limits: d % 8 == 0, 1 <= topk <= min(K, 64),
+ * 1 <= B <= 256, and d <= 8192 (B <= 8) or d <= 4096 (B <= 16) on the streaming path.
+ */
+vt_status vt_draft_head(const uint16_t *h, const uint16_t *W_trim, const int32_t *map, int32_t B,
+                        int32_t K, int32_t d, const float *temp, int32_t topk,
+                        const float *uniforms, int32_t *out_ids, float *out_logprobs, void *ws,
+                        size_t ws_bytes, void *stream);
+
+/* Parity-only variant of vt_draft_head: also writes the fp32 logits [B,K] and lse [B]
+ * (log sum exp of z) when those pointers are non-NULL.  Never used for timing. */
+vt_status vt_draft_head_debug(const uint16_t *h, const uint16_t *W_trim, const int32_t *map,
+                              int32_t B, int32_t K, int32_t d, const float *temp, int32_t topk,
+                              const float *uniforms, int32_t *out_ids, float *out_logprobs,
+                              void *ws, size_t ws_bytes, void *stream, float *out_logits,
+                              float *out_lse);
+
+/* Same as vt_draft_head with the per-step tensors in HOST memory: h, temp, uniforms are copied
+ * in and out_ids, out_logprobs copied back through staging areas in the workspace, all on
+ * `stream`; the call returns after enqueueing (synchronise the stream before reading the
+ * outputs).  W_trim and map are the resident model state and stay DEVICE pointers. */
+vt_status vt_draft_head_host(const uint16_t *h_host, const uint16_t *W_trim, const int32_t *map,
+                             int32_t B, int32_t K, int32_t d, const float *temp_host,
+                             int32_t topk, const float *uniforms_host, int32_t *out_ids_host,
+                             float *out_logprobs_host, void *ws, size_t ws_bytes, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* VOCABTRIM_H */

@@ -1,0 +1,249 @@
+"""B200-native VocabTrim hot path: thin Python binding over the C-ABI CUDA library.
+
+Everything here is argument marshalling.  Tensors are torch CUDA tensors used only as device
+memory; every step of the path (histogram, top-K selection, head gather, trimmed head with its
+sampling epilogue and the remap) runs in the hand-written sm_100a kernels of libvocabtrim.so.
+There is no CPU or PyTorch fallback: if the library is missing or a call fails, an exception is
+raised.
+
+Names follow the C header (include/vocabtrim.h): vt_histogram, vt_select_topk, vt_build_vocab,
+vt_trim_head, vt_draft_head, ...  `map` is in rank order (map[0] = most frequent id).
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from ctypes import c_char_p, c_float, c_int, c_int32, c_int64, c_size_t, c_uint32, c_uint64, c_void_p
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libvocabtrim.so")
+
+VT_OK = 0
+VT_OP_HISTOGRAM, VT_OP_SELECT_TOPK, VT_OP_BUILD_VOCAB, VT_OP_TRIM_HEAD = 0, 1, 2, 3
+VT_OP_DRAFT_HEAD, VT_OP_DRAFT_HEAD_HOST, VT_OP_BUILD_VOCAB_HOST = 4, 5, 6
+VT_FLAG_BAD_ID, VT_FLAG_BAD_MAP, VT_FLAG_BAD_TEMP, VT_FLAG_NAN_ROW, VT_FLAG_TIMEOUT = 1, 2, 4, 8, 16
+VT_MAX_TOPK = 64
+VT_CTRL_BYTES = 256
+
+EXPORTS = (
+    "vt_workspace_bytes", "vt_workspace_init", "vt_read_status", "vt_status_str", "vt_launch_count",
+    "vt_histogram", "vt_select_topk", "vt_build_vocab", "vt_build_vocab_host", "vt_trim_head",
+    "vt_draft_head", "vt_draft_head_debug", "vt_draft_head_host",
+)
+
+
+class VocabTrimError(RuntimeError):
+    def __init__(self, call: str, status: int):
+        self.status = status
+        super().__init__("%s failed: %s (status %d)" % (call, status_str(status), status))
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Loads libvocabtrim.so; raises if it has not been built (python -m paper_2506_22694_b200.build)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError("libvocabtrim.so is missing: build it with "
+                               "`python -m paper_2506_22694_b200.build` (no fallback path exists)")
+        L = ctypes.CDLL(LIB_PATH)
+        L.vt_workspace_bytes.restype = c_size_t
+        L.vt_workspace_bytes.argtypes = [c_int, c_int64, c_int32, c_int32, c_int32, c_int32, c_int32]
+        L.vt_workspace_init.argtypes = [c_void_p, c_size_t, c_void_p]
+        L.vt_read_status.argtypes = [c_void_p, c_void_p, ctypes.POINTER(c_uint32), ctypes.POINTER(c_uint64)]
+        L.vt_status_str.restype = c_char_p
+        L.vt_status_str.argtypes = [c_int]
+        L.vt_launch_count.restype = c_uint64
+        L.vt_histogram.argtypes = [c_void_p, c_int64, c_int32, c_void_p, c_int, c_void_p, c_size_t, c_void_p]
+        L.vt_select_topk.argtypes = [c_void_p, c_int32, c_int32, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
+        L.vt_build_vocab.argtypes = [c_void_p, c_int64, c_int32, c_int32, c_void_p, c_void_p, c_void_p,
+                                     c_size_t, c_void_p]
+        L.vt_build_vocab_host.argtypes = L.vt_build_vocab.argtypes
+        L.vt_trim_head.argtypes = [c_void_p, c_void_p, c_void_p, c_int32, c_int32, c_int32, c_void_p, c_void_p]
+        head = [c_void_p, c_void_p, c_void_p, c_int32, c_int32, c_int32, c_void_p, c_int32, c_void_p,
+                c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
+        L.vt_draft_head.argtypes = head
+        L.vt_draft_head_host.argtypes = head
+        L.vt_draft_head_debug.argtypes = head + [c_void_p, c_void_p]
+        _lib = L
+    return _lib
+
+
+def status_str(status: int) -> str:
+    return lib().vt_status_str(int(status)).decode()
+
+
+def launch_count() -> int:
+    return int(lib().vt_launch_count())
+
+
+def _check(call: str, status: int) -> None:
+    if status != VT_OK:
+        raise VocabTrimError(call, status)
+
+
+def _ptr(t):
+    return c_void_p(t.data_ptr()) if t is not None else c_void_p(0)
+
+
+def _stream() -> c_void_p:
+    return c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _dev(t: torch.Tensor, dtype, name: str) -> torch.Tensor:
+    if not (t.is_cuda and t.dtype == dtype and t.is_contiguous()):
+        raise TypeError("%s must be a contiguous CUDA tensor of dtype %s" % (name, dtype))
+    return t
+
+
+def workspace_bytes(op: int, n: int = 0, V: int = 0, K: int = 0, d: int = 0, B: int = 0, topk: int = 0) -> int:
+    return int(lib().vt_workspace_bytes(op, n, V, K, d, B, topk))
+
+
+class Workspace:
+    """Caller-owned scratch for the library: a 256-byte-aligned device buffer whose control block
+    has been cleared once (vt_workspace_init).  One workspace serves one stream at a time."""
+
+    def __init__(self, nbytes: int, device="cuda"):
+        if nbytes <= 0:
+            raise ValueError("unsupported shape: the library reported a zero-size workspace")
+        self.nbytes = int(nbytes)
+        self.buf = torch.empty(self.nbytes + 256, dtype=torch.uint8, device=device)
+        off = (-self.buf.data_ptr()) % 256
+        self.ptr = self.buf.data_ptr() + off
+        _check("vt_workspace_init", lib().vt_workspace_init(c_void_p(self.ptr), self.nbytes, _stream()))
+
+    def read_status(self):
+        """Synchronises the current stream; returns (status, flags, n_bad) and clears the flags."""
+        flags, bad = c_uint32(0), c_uint64(0)
+        st = lib().vt_read_status(c_void_p(self.ptr), _stream(), ctypes.byref(flags), ctypes.byref(bad))
+        return int(st), int(flags.value), int(bad.value)
+
+
+def _ws(ws: Workspace | None, need: int, like: torch.Tensor) -> Workspace:
+    if ws is None:
+        return Workspace(need, like.device)
+    if ws.nbytes < need:
+        raise VocabTrimError("workspace too small (%d < %d)" % (ws.nbytes, need), 3)
+    return ws
+
+
+def vt_histogram(ids: torch.Tensor, V: int, counts: torch.Tensor | None = None, accumulate: bool = False,
+                 ws: Workspace | None = None) -> torch.Tensor:
+    """Algorithm 1.  ids int32 [n] -> counts int32 storage holding uint32 values [V]."""
+    _dev(ids, torch.int32, "ids")
+    if counts is None:
+        counts = torch.empty(V, dtype=torch.int32, device=ids.device)
+        accumulate = False
+    _dev(counts, torch.int32, "counts")
+    ws = _ws(ws, workspace_bytes(VT_OP_HISTOGRAM, ids.numel(), V), ids)
+    _check("vt_histogram", lib().vt_histogram(_ptr(ids), ids.numel(), V, _ptr(counts), int(bool(accumulate)),
+                                              c_void_p(ws.ptr), ws.nbytes, _stream()))
+    return counts
+
+
+def vt_select_topk(counts: torch.Tensor, K: int, ws: Workspace | None = None):
+    """Eq. 1, line 1.  counts [V] -> (map int32 [K], inv_map int32 [V])."""
+    _dev(counts, torch.int32, "counts")
+    V = counts.numel()
+    map_ = torch.empty(K, dtype=torch.int32, device=counts.device)
+    inv = torch.empty(V, dtype=torch.int32, device=counts.device)
+    ws = _ws(ws, workspace_bytes(VT_OP_SELECT_TOPK, 0, V, K), counts)
+    _check("vt_select_topk", lib().vt_select_topk(_ptr(counts), V, K, _ptr(map_), _ptr(inv), c_void_p(ws.ptr),
+                                                  ws.nbytes, _stream()))
+    return map_, inv
+
+
+def vt_build_vocab(ids: torch.Tensor, V: int, K: int, ws: Workspace | None = None):
+    """Algorithm 1 + Eq. 1, line 1.  Device ids -> (map [K], inv_map [V]).  A CPU (ideally pinned)
+    ids tensor goes through vt_build_vocab_host, which streams it to the device in chunks."""
+    if not ids.is_cuda:
+        return vt_build_vocab_host(ids, V, K, ws)
+    _dev(ids, torch.int32, "ids")
+    map_ = torch.empty(K, dtype=torch.int32, device=ids.device)
+    inv = torch.empty(V, dtype=torch.int32, device=ids.device)
+    ws = _ws(ws, workspace_bytes(VT_OP_BUILD_VOCAB, ids.numel(), V, K), ids)
+    _check("vt_build_vocab", lib().vt_build_vocab(_ptr(ids), ids.numel(), V, K, _ptr(map_), _ptr(inv),
+                                                  c_void_p(ws.ptr), ws.nbytes, _stream()))
+    return map_, inv
+
+
+def vt_build_vocab_host(ids_host: torch.Tensor, V: int, K: int, ws: Workspace | None = None, device="cuda",
+                        out=None):
+    if ids_host.is_cuda or ids_host.dtype != torch.int32 or not ids_host.is_contiguous():
+        raise TypeError("ids_host must be a contiguous CPU int32 tensor")
+    if out is None:
+        out = (torch.empty(K, dtype=torch.int32, device=device), torch.empty(V, dtype=torch.int32, device=device))
+    map_, inv = out
+    ws = _ws(ws, workspace_bytes(VT_OP_BUILD_VOCAB_HOST, ids_host.numel(), V, K), map_)
+    _check("vt_build_vocab_host", lib().vt_build_vocab_host(
+        c_void_p(ids_host.data_ptr()), ids_host.numel(), V, K, _ptr(map_), _ptr(inv), c_void_p(ws.ptr),
+        ws.nbytes, _stream()))
+    return map_, inv
+
+
+def vt_trim_head(W_full: torch.Tensor, map_: torch.Tensor, W_trim: torch.Tensor | None = None,
+                 ws: Workspace | None = None) -> torch.Tensor:
+    """Eq. 1, line 2.  W_full bf16 [V,d], map int32 [K] -> W_trim bf16 [K,d]."""
+    _dev(W_full, torch.bfloat16, "W_full")
+    _dev(map_, torch.int32, "map")
+    V, d = W_full.shape
+    K = map_.numel()
+    if W_trim is None:
+        W_trim = torch.empty((K, d), dtype=torch.bfloat16, device=W_full.device)
+    _dev(W_trim, torch.bfloat16, "W_trim")
+    _check("vt_trim_head", lib().vt_trim_head(_ptr(W_full), _ptr(map_), _ptr(W_trim), V, K, d,
+                                              c_void_p(ws.ptr if ws else 0), _stream()))
+    return W_trim
+
+
+def vt_draft_head(h: torch.Tensor, W_trim: torch.Tensor, map_: torch.Tensor | None, temp: torch.Tensor,
+                  topk: int, uniforms: torch.Tensor | None = None, ws: Workspace | None = None,
+                  out=None, debug: bool = False):
+    """Algorithm 2, lines 5-6 (head part).  Returns (out_ids int32 [B,1+topk], out_logprobs fp32
+    [B,1+topk]); with debug=True also (logits fp32 [B,K], lse fp32 [B])."""
+    _dev(h, torch.bfloat16, "h")
+    _dev(W_trim, torch.bfloat16, "W_trim")
+    _dev(temp, torch.float32, "temp")
+    B, d = h.shape
+    K = W_trim.shape[0]
+    if W_trim.shape[1] != d or temp.numel() != B:
+        raise ValueError("shape mismatch between h, W_trim and temp")
+    if map_ is not None and _dev(map_, torch.int32, "map").numel() != K:
+        raise ValueError("map must have K entries")
+    if uniforms is not None and tuple(_dev(uniforms, torch.float32, "uniforms").shape) != (B, K):
+        raise ValueError("uniforms must be [B,K]")
+    if out is None:
+        out = (torch.empty((B, 1 + topk), dtype=torch.int32, device=h.device),
+               torch.empty((B, 1 + topk), dtype=torch.float32, device=h.device))
+    ids, lps = out
+    ws = _ws(ws, workspace_bytes(VT_OP_DRAFT_HEAD, 0, 0, K, d, B, topk), h)
+    args = [_ptr(h), _ptr(W_trim), _ptr(map_), B, K, d, _ptr(temp), topk, _ptr(uniforms), _ptr(ids), _ptr(lps),
+            c_void_p(ws.ptr), ws.nbytes, _stream()]
+    if debug:
+        logits = torch.empty((B, K), dtype=torch.float32, device=h.device)
+        lse = torch.empty(B, dtype=torch.float32, device=h.device)
+        _check("vt_draft_head_debug", lib().vt_draft_head_debug(*args, _ptr(logits), _ptr(lse)))
+        return ids, lps, logits, lse
+    _check("vt_draft_head", lib().vt_draft_head(*args))
+    return ids, lps
+
+
+def vt_draft_head_host(h_host: torch.Tensor, W_trim: torch.Tensor, map_: torch.Tensor | None,
+                       temp_host: torch.Tensor, topk: int, uniforms_host: torch.Tensor | None,
+                       ws: Workspace, out_host):
+    """vt_draft_head with the per-step tensors in (pinned) host memory; W_trim and map stay on the
+    device.  Enqueues copies and kernels on the current stream and returns; synchronise before
+    reading out_host = (ids int32 [B,1+topk], logprobs fp32 [B,1+topk]) CPU tensors."""
+    B, d = h_host.shape
+    K = W_trim.shape[0]
+    ids, lps = out_host
+    _check("vt_draft_head_host", lib().vt_draft_head_host(
+        c_void_p(h_host.data_ptr()), _ptr(W_trim), _ptr(map_), B, K, d, c_void_p(temp_host.data_ptr()), topk,
+        c_void_p(uniforms_host.data_ptr() if uniforms_host is not None else 0), c_void_p(ids.data_ptr()),
+        c_void_p(lps.data_ptr()), c_void_p(ws.ptr), ws.nbytes, _stream()))
+    return ids, lps

@@ -1,0 +1,319 @@
+// extern "C" boundary: argument checks, workspace carving, dispatch.  See include/vocabtrim.h
+// for the contract of every entry point.
+#include <atomic>
+
+#include "vt_common.cuh"
+
+namespace vt {
+
+static std::atomic<uint64_t> g_launches{0};
+void count_launch(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
+
+int num_sms() {
+    static int cached[64] = {0};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return kNumSMsFallback;
+    if (dev >= 0 && dev < 64 && cached[dev]) return cached[dev];
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
+        n = kNumSMsFallback;
+    if (dev >= 0 && dev < 64) cached[dev] = n;
+    return n;
+}
+
+namespace {
+
+inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+inline cudaStream_t as_stream(void* s) { return reinterpret_cast<cudaStream_t>(s); }
+inline vt_status from_cuda(cudaError_t e) { return e == cudaSuccess ? VT_OK : VT_ERR_CUDA; }
+
+constexpr int64_t kHostChunkIds = 1 << 24;     // ids per staged chunk of vt_build_vocab_host
+
+bool hist_shape_ok(int32_t V) {
+    if (V < 1) return false;
+    return hist_plan(V).small || ((size_t)(V + 31) / 32 * 8 + 65536 <= (size_t)224 * 1024);
+}
+
+bool head_shape_ok(int32_t B, int32_t K, int32_t d, int32_t topk) {
+    if (B < 1 || B > 256 || K < 1 || d < 8 || (d & 7) || topk < 1 || topk > VT_MAX_TOPK || topk > K)
+        return false;
+    return head_skinny_supported(B, d) || head_dense_supported(B, K, d);
+}
+
+size_t head_scratch(int32_t B, int32_t K, int32_t d, int32_t topk) {
+    if (head_skinny_supported(B, d)) return head_skinny_scratch_bytes(B, K, topk);
+    return head_dense_scratch_bytes(B, K, topk);
+}
+
+// staging layout of vt_draft_head_host after the head scratch
+struct HostStage {
+    size_t off_h, off_temp, off_u, off_ids, off_lp, bytes;
+};
+HostStage host_stage(int32_t B, int32_t K, int32_t d, int32_t topk, size_t base) {
+    HostStage s{};
+    size_t o = align_up(base, 256);
+    s.off_h = o;     o += align_up((size_t)B * d * 2, 256);
+    s.off_temp = o;  o += align_up((size_t)B * 4, 256);
+    s.off_u = o;     o += align_up((size_t)B * K * 4, 256);
+    s.off_ids = o;   o += align_up((size_t)B * (1 + topk) * 4, 256);
+    s.off_lp = o;    o += align_up((size_t)B * (1 + topk) * 4, 256);
+    s.bytes = o;
+    return s;
+}
+
+vt_status check_ws(void* ws, size_t ws_bytes, size_t need) {
+    if (!ws || !aligned(ws, 256) || need == 0 || ws_bytes < need) return VT_ERR_WORKSPACE;
+    return VT_OK;
+}
+
+}  // namespace
+}  // namespace vt
+
+using namespace vt;
+
+extern "C" {
+
+size_t vt_workspace_bytes(int op, int64_t n, int32_t V, int32_t K, int32_t d, int32_t B,
+                          int32_t topk) {
+    switch (op) {
+        case VT_OP_HISTOGRAM:
+            if (!hist_shape_ok(V) || n < 0) return 0;
+            return VT_CTRL_BYTES + hist_plan(V).bytes;
+        case VT_OP_SELECT_TOPK:
+            if (V < 1 || K < 1 || K > V) return 0;
+            return VT_CTRL_BYTES + select_scratch_bytes(V);
+        case VT_OP_BUILD_VOCAB:
+        case VT_OP_BUILD_VOCAB_HOST: {
+            if (!hist_shape_ok(V) || n < 0 || K < 1 || K > V) return 0;
+            size_t inner = hist_plan(V).bytes;
+            if (select_scratch_bytes(V) > inner) inner = select_scratch_bytes(V);
+            size_t total = VT_CTRL_BYTES + align_up((size_t)V * 4, 256) + inner;
+            if (op == VT_OP_BUILD_VOCAB_HOST) {
+                const int64_t chunk = n < kHostChunkIds ? (n > 0 ? n : 1) : kHostChunkIds;
+                total = align_up(total, 256) + 2 * align_up((size_t)chunk * 4, 256);
+            }
+            return total;
+        }
+        case VT_OP_TRIM_HEAD:
+            return VT_CTRL_BYTES;
+        case VT_OP_DRAFT_HEAD:
+            if (!head_shape_ok(B, K, d, topk)) return 0;
+            return VT_CTRL_BYTES + head_scratch(B, K, d, topk);
+        case VT_OP_DRAFT_HEAD_HOST:
+            if (!head_shape_ok(B, K, d, topk)) return 0;
+            return host_stage(B, K, d, topk, VT_CTRL_BYTES + head_scratch(B, K, d, topk)).bytes;
+        default:
+            return 0;
+    }
+}
+
+vt_status vt_workspace_init(void* ws, size_t ws_bytes, void* stream) {
+    if (!ws || !aligned(ws, 256) || ws_bytes < VT_CTRL_BYTES) return VT_ERR_WORKSPACE;
+    return from_cuda(cudaMemsetAsync(ws, 0, VT_CTRL_BYTES, as_stream(stream)));
+}
+
+vt_status vt_read_status(void* ws, void* stream, uint32_t* flags, uint64_t* n_bad) {
+    if (!ws) return VT_ERR_WORKSPACE;
+    Ctrl host{};
+    cudaStream_t s = as_stream(stream);
+    if (cudaMemcpyAsync(&host, ws, sizeof(Ctrl), cudaMemcpyDeviceToHost, s) != cudaSuccess)
+        return VT_ERR_CUDA;
+    if (cudaStreamSynchronize(s) != cudaSuccess) return VT_ERR_CUDA;
+    if (host.flags || host.n_bad) {
+        // clear the sticky part only (flags + n_bad); tickets are left alone
+        Ctrl* dev = static_cast<Ctrl*>(ws);
+        if (cudaMemsetAsync(&dev->flags, 0, sizeof(uint32_t), s) != cudaSuccess) return VT_ERR_CUDA;
+        if (cudaMemsetAsync(&dev->n_bad, 0, sizeof(unsigned long long), s) != cudaSuccess)
+            return VT_ERR_CUDA;
+        if (cudaStreamSynchronize(s) != cudaSuccess) return VT_ERR_CUDA;
+    }
+    if (flags) *flags = host.flags;
+    if (n_bad) *n_bad = host.n_bad;
+    if (host.flags & VT_FLAG_TIMEOUT) return VT_ERR_TIMEOUT;
+    if (host.flags & (VT_FLAG_BAD_ID | VT_FLAG_BAD_MAP)) return VT_ERR_RANGE;
+    if (host.flags & (VT_FLAG_BAD_TEMP | VT_FLAG_NAN_ROW)) return VT_ERR_NUMERIC;
+    return VT_OK;
+}
+
+const char* vt_status_str(vt_status s) {
+    switch (s) {
+        case VT_OK: return "ok";
+        case VT_ERR_INVALID_ARG: return "invalid argument";
+        case VT_ERR_RANGE: return "token id or map entry out of range";
+        case VT_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+        case VT_ERR_CUDA: return "CUDA runtime error";
+        case VT_ERR_TIMEOUT: return "bounded device-side wait expired";
+        case VT_ERR_UNSUPPORTED: return "unsupported shape";
+        case VT_ERR_NUMERIC: return "non-positive temperature or NaN row";
+        default: return "unknown status";
+    }
+}
+
+uint64_t vt_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+vt_status vt_histogram(const int32_t* ids, int64_t n, int32_t V, uint32_t* counts, int accumulate,
+                       void* ws, size_t ws_bytes, void* stream) {
+    if (n < 0 || n >= ((int64_t)1 << 32) || V < 1 || !counts || (n > 0 && !ids)) return VT_ERR_INVALID_ARG;
+    if (!aligned(ids, 4) || !aligned(counts, 4)) return VT_ERR_INVALID_ARG;
+    if (!hist_shape_ok(V)) return VT_ERR_UNSUPPORTED;
+    vt_status st = check_ws(ws, ws_bytes, vt_workspace_bytes(VT_OP_HISTOGRAM, n, V, 0, 0, 0, 0));
+    if (st != VT_OK) return st;
+    uint8_t* base = static_cast<uint8_t*>(ws);
+    return from_cuda(launch_histogram(ids, n, V, counts, accumulate, reinterpret_cast<Ctrl*>(base),
+                                      base + VT_CTRL_BYTES, as_stream(stream)));
+}
+
+vt_status vt_select_topk(const uint32_t* counts, int32_t V, int32_t K, int32_t* map,
+                         int32_t* inv_map, void* ws, size_t ws_bytes, void* stream) {
+    if (!counts || !map || !inv_map || V < 1 || K < 1 || K > V) return VT_ERR_INVALID_ARG;
+    vt_status st = check_ws(ws, ws_bytes, vt_workspace_bytes(VT_OP_SELECT_TOPK, 0, V, K, 0, 0, 0));
+    if (st != VT_OK) return st;
+    uint8_t* base = static_cast<uint8_t*>(ws);
+    return from_cuda(launch_select_topk(counts, V, K, map, inv_map, base + VT_CTRL_BYTES,
+                                        as_stream(stream)));
+}
+
+vt_status vt_build_vocab(const int32_t* ids, int64_t n, int32_t V, int32_t K, int32_t* map,
+                         int32_t* inv_map, void* ws, size_t ws_bytes, void* stream) {
+    if (n < 0 || n >= ((int64_t)1 << 32) || V < 1 || K < 1 || K > V || !map || !inv_map || (n > 0 && !ids))
+        return VT_ERR_INVALID_ARG;
+    if (!aligned(ids, 4)) return VT_ERR_INVALID_ARG;
+    if (!hist_shape_ok(V)) return VT_ERR_UNSUPPORTED;
+    vt_status st = check_ws(ws, ws_bytes, vt_workspace_bytes(VT_OP_BUILD_VOCAB, n, V, K, 0, 0, 0));
+    if (st != VT_OK) return st;
+    uint8_t* base = static_cast<uint8_t*>(ws);
+    uint32_t* counts = reinterpret_cast<uint32_t*>(base + VT_CTRL_BYTES);
+    uint8_t* inner = base + VT_CTRL_BYTES + align_up((size_t)V * 4, 256);
+    cudaStream_t s = as_stream(stream);
+    cudaError_t e = launch_histogram(ids, n, V, counts, 0, reinterpret_cast<Ctrl*>(base), inner, s);
+    if (e != cudaSuccess) return VT_ERR_CUDA;
+    return from_cuda(launch_select_topk(counts, V, K, map, inv_map, inner, s));
+}
+
+vt_status vt_build_vocab_host(const int32_t* ids_host, int64_t n, int32_t V, int32_t K,
+                              int32_t* map, int32_t* inv_map, void* ws, size_t ws_bytes,
+                              void* stream) {
+    if (n < 0 || n >= ((int64_t)1 << 32) || V < 1 || K < 1 || K > V || !map || !inv_map ||
+        (n > 0 && !ids_host))
+        return VT_ERR_INVALID_ARG;
+    if (!hist_shape_ok(V)) return VT_ERR_UNSUPPORTED;
+    vt_status st = check_ws(ws, ws_bytes, vt_workspace_bytes(VT_OP_BUILD_VOCAB_HOST, n, V, K, 0, 0, 0));
+    if (st != VT_OK) return st;
+    uint8_t* base = static_cast<uint8_t*>(ws);
+    Ctrl* ctrl = reinterpret_cast<Ctrl*>(base);
+    uint32_t* counts = reinterpret_cast<uint32_t*>(base + VT_CTRL_BYTES);
+    uint8_t* inner = base + VT_CTRL_BYTES + align_up((size_t)V * 4, 256);
+    const size_t dev_part = vt_workspace_bytes(VT_OP_BUILD_VOCAB, n, V, K, 0, 0, 0);
+    const int64_t chunk = n < kHostChunkIds ? (n > 0 ? n : 1) : kHostChunkIds;
+    int32_t* stage[2];
+    stage[0] = reinterpret_cast<int32_t*>(base + align_up(dev_part, 256));
+    stage[1] = reinterpret_cast<int32_t*>(reinterpret_cast<uint8_t*>(stage[0]) + align_up((size_t)chunk * 4, 256));
+    cudaStream_t s = as_stream(stream);
+    // Copies run on a second stream so chunk i+1 arrives while chunk i is counted; events order
+    // "copy done -> count" and "count done -> buffer may be overwritten".
+    cudaStream_t copy_stream = nullptr;
+    cudaEvent_t copied[2] = {nullptr, nullptr}, counted[2] = {nullptr, nullptr}, start = nullptr;
+    cudaError_t e = cudaStreamCreateWithFlags(&copy_stream, cudaStreamNonBlocking);
+    for (int i = 0; i < 2 && e == cudaSuccess; ++i) {
+        e = cudaEventCreateWithFlags(&copied[i], cudaEventDisableTiming);
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&counted[i], cudaEventDisableTiming);
+    }
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&start, cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaMemsetAsync(counts, 0, (size_t)V * 4, s);
+    if (e == cudaSuccess) e = cudaEventRecord(start, s);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(copy_stream, start, 0);   // staging free once prior work on s is done
+    int64_t done = 0;
+    for (int i = 0; done < n && e == cudaSuccess; ++i) {
+        const int sl = i & 1;
+        const int64_t m = (n - done < chunk) ? n - done : chunk;
+        if (i >= 2) e = cudaStreamWaitEvent(copy_stream, counted[sl], 0);
+        if (e == cudaSuccess)
+            e = cudaMemcpyAsync(stage[sl], ids_host + done, (size_t)m * 4, cudaMemcpyHostToDevice, copy_stream);
+        if (e == cudaSuccess) e = cudaEventRecord(copied[sl], copy_stream);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(s, copied[sl], 0);
+        if (e == cudaSuccess) e = launch_histogram(stage[sl], m, V, counts, 1, ctrl, inner, s);
+        if (e == cudaSuccess) e = cudaEventRecord(counted[sl], s);
+        done += m;
+    }
+    if (e == cudaSuccess) e = launch_select_topk(counts, V, K, map, inv_map, inner, s);
+    for (int i = 0; i < 2; ++i) {
+        if (copied[i]) cudaEventDestroy(copied[i]);
+        if (counted[i]) cudaEventDestroy(counted[i]);
+    }
+    if (start) cudaEventDestroy(start);
+    if (copy_stream) cudaStreamDestroy(copy_stream);    // deferred until its work completes
+    return from_cuda(e);
+}
+
+vt_status vt_trim_head(const uint16_t* W_full, const int32_t* map, uint16_t* W_trim, int32_t V,
+                       int32_t K, int32_t d, void* ws, void* stream) {
+    if (!W_full || !map || !W_trim || V < 1 || K < 1 || d < 8 || (d & 7)) return VT_ERR_INVALID_ARG;
+    if (!aligned(W_full, 16) || !aligned(W_trim, 16) || !aligned(map, 4)) return VT_ERR_INVALID_ARG;
+    if (ws && !aligned(ws, 256)) return VT_ERR_WORKSPACE;
+    return from_cuda(launch_gather_rows(W_full, map, W_trim, V, K, d, static_cast<Ctrl*>(ws),
+                                        as_stream(stream)));
+}
+
+vt_status vt_draft_head_debug(const uint16_t* h, const uint16_t* W_trim, const int32_t* map,
+                              int32_t B, int32_t K, int32_t d, const float* temp, int32_t topk,
+                              const float* uniforms, int32_t* out_ids, float* out_logprobs,
+                              void* ws, size_t ws_bytes, void* stream, float* out_logits,
+                              float* out_lse) {
+    if (!h || !W_trim || !temp || !out_ids || !out_logprobs) return VT_ERR_INVALID_ARG;
+    if (B < 1 || K < 1 || d < 8 || (d & 7) || topk < 1 || topk > VT_MAX_TOPK || topk > K)
+        return VT_ERR_INVALID_ARG;
+    if (!aligned(h, 16) || !aligned(W_trim, 16)) return VT_ERR_INVALID_ARG;
+    if (!head_shape_ok(B, K, d, topk)) return VT_ERR_UNSUPPORTED;
+    vt_status st = check_ws(ws, ws_bytes, vt_workspace_bytes(VT_OP_DRAFT_HEAD, 0, 0, K, d, B, topk));
+    if (st != VT_OK) return st;
+    uint8_t* base = static_cast<uint8_t*>(ws);
+    HeadArgs a{h, W_trim, map, B, K, d, temp, topk, uniforms, out_ids, out_logprobs, out_logits, out_lse};
+    if (head_skinny_supported(B, d))
+        return from_cuda(launch_head_skinny(a, reinterpret_cast<Ctrl*>(base), base + VT_CTRL_BYTES,
+                                            as_stream(stream)));
+    return from_cuda(launch_head_dense(a, reinterpret_cast<Ctrl*>(base), base + VT_CTRL_BYTES,
+                                       as_stream(stream)));
+}
+
+vt_status vt_draft_head(const uint16_t* h, const uint16_t* W_trim, const int32_t* map, int32_t B,
+                        int32_t K, int32_t d, const float* temp, int32_t topk,
+                        const float* uniforms, int32_t* out_ids, float* out_logprobs, void* ws,
+                        size_t ws_bytes, void* stream) {
+    return vt_draft_head_debug(h, W_trim, map, B, K, d, temp, topk, uniforms, out_ids, out_logprobs,
+                               ws, ws_bytes, stream, nullptr, nullptr);
+}
+
+vt_status vt_draft_head_host(const uint16_t* h_host, const uint16_t* W_trim, const int32_t* map,
+                             int32_t B, int32_t K, int32_t d, const float* temp_host, int32_t topk,
+                             const float* uniforms_host, int32_t* out_ids_host,
+                             float* out_logprobs_host, void* ws, size_t ws_bytes, void* stream) {
+    if (!h_host || !W_trim || !temp_host || !out_ids_host || !out_logprobs_host) return VT_ERR_INVALID_ARG;
+    if (B < 1 || K < 1 || d < 8 || (d & 7) || topk < 1 || topk > VT_MAX_TOPK || topk > K)
+        return VT_ERR_INVALID_ARG;
+    if (!head_shape_ok(B, K, d, topk)) return VT_ERR_UNSUPPORTED;
+    vt_status st = check_ws(ws, ws_bytes, vt_workspace_bytes(VT_OP_DRAFT_HEAD_HOST, 0, 0, K, d, B, topk));
+    if (st != VT_OK) return st;
+    uint8_t* base = static_cast<uint8_t*>(ws);
+    const size_t head_part = VT_CTRL_BYTES + head_scratch(B, K, d, topk);
+    const HostStage hs = host_stage(B, K, d, topk, head_part);
+    cudaStream_t s = as_stream(stream);
+    uint16_t* dh = reinterpret_cast<uint16_t*>(base + hs.off_h);
+    float* dt = reinterpret_cast<float*>(base + hs.off_temp);
+    float* du = reinterpret_cast<float*>(base + hs.off_u);
+    int32_t* di = reinterpret_cast<int32_t*>(base + hs.off_ids);
+    float* dl = reinterpret_cast<float*>(base + hs.off_lp);
+    const size_t out_bytes = (size_t)B * (1 + topk) * 4;
+    cudaError_t e = cudaMemcpyAsync(dh, h_host, (size_t)B * d * 2, cudaMemcpyHostToDevice, s);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(dt, temp_host, (size_t)B * 4, cudaMemcpyHostToDevice, s);
+    if (e == cudaSuccess && uniforms_host)
+        e = cudaMemcpyAsync(du, uniforms_host, (size_t)B * K * 4, cudaMemcpyHostToDevice, s);
+    if (e != cudaSuccess) return VT_ERR_CUDA;
+    st = vt_draft_head(dh, W_trim, map, B, K, d, dt, topk, uniforms_host ? du : nullptr, di, dl, ws,
+                       head_part, stream);
+    if (st != VT_OK) return st;
+    e = cudaMemcpyAsync(out_ids_host, di, out_bytes, cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(out_logprobs_host, dl, out_bytes, cudaMemcpyDeviceToHost, s);
+    return from_cuda(e);
+}
+
+}  // extern "C"

@@ -1,0 +1,100 @@
+// Shared declarations of the CUDA side: control block layout, launch bookkeeping, small
+// device helpers.  Nothing here is seen by the CPU oracle.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "vocabtrim.h"
+
+namespace vt {
+
+// First VT_CTRL_BYTES of every workspace.  Cleared once by vt_workspace_init; every kernel
+// leaves `ticket` words at zero when it finishes.
+struct Ctrl {
+    uint32_t flags;               // sticky VT_FLAG_* bits
+    uint32_t head_ticket;         // "last CTA merges" ticket of the head kernels (wraps to 0)
+    unsigned long long n_bad;     // ids skipped by the histogram
+    uint32_t pad[60];
+};
+static_assert(sizeof(Ctrl) == VT_CTRL_BYTES, "control block size");
+
+constexpr int kNumSMsFallback = 148;
+
+int num_sms();                    // SM count of the current device (cached per device)
+void count_launch(int n = 1);     // host-side launch counter behind vt_launch_count
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// ---- launchers implemented in the .cu files (host functions) --------------------------------
+struct HistPlan {
+    bool small;            // all bins fit in one CTA's shared memory
+    size_t off_sample;     // uint32 [V]   sampled counts
+    size_t off_table;      // uint2  [ceil(V/32)] hot-bin table {bitmap word, slot base}
+    size_t bytes;          // scratch after the control block
+};
+HistPlan hist_plan(int32_t V);
+cudaError_t launch_histogram(const int32_t* ids, int64_t n, int32_t V, uint32_t* counts,
+                             int accumulate, Ctrl* ctrl, uint8_t* scratch, cudaStream_t s);
+
+size_t select_scratch_bytes(int32_t V);
+cudaError_t launch_select_topk(const uint32_t* counts, int32_t V, int32_t K, int32_t* map,
+                               int32_t* inv_map, uint8_t* scratch, cudaStream_t s);
+
+cudaError_t launch_gather_rows(const uint16_t* W_full, const int32_t* map, uint16_t* W_trim,
+                               int32_t V, int32_t K, int32_t d, Ctrl* ctrl, cudaStream_t s);
+
+struct HeadArgs {
+    const uint16_t* h;
+    const uint16_t* W;
+    const int32_t* map;
+    int32_t B, K, d;
+    const float* temp;
+    int32_t topk;
+    const float* uniforms;
+    int32_t* out_ids;
+    float* out_logprobs;
+    float* dbg_logits;
+    float* dbg_lse;
+};
+bool head_skinny_supported(int32_t B, int32_t d);
+size_t head_skinny_scratch_bytes(int32_t B, int32_t K, int32_t topk);
+cudaError_t launch_head_skinny(const HeadArgs& a, Ctrl* ctrl, uint8_t* scratch, cudaStream_t s);
+
+bool head_dense_supported(int32_t B, int32_t K, int32_t d);
+size_t head_dense_scratch_bytes(int32_t B, int32_t K, int32_t topk);
+cudaError_t launch_head_dense(const HeadArgs& a, Ctrl* ctrl, uint8_t* scratch, cudaStream_t s);
+
+// ---- device helpers ----------------------------------------------------------------------------
+#ifdef __CUDACC__
+// Streaming 128-bit load: read-only path, do not keep the line in L1 (data is used once).
+__device__ __forceinline__ uint4 ld_stream_u4(const void* p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.L2::128B.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p));
+    return v;
+}
+__device__ __forceinline__ void st_stream_u4(void* p, uint4 v) {
+    asm volatile("st.global.cs.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.x), "r"(v.y),
+                 "r"(v.z), "r"(v.w)
+                 : "memory");
+}
+// Load that bypasses L1 (partials written by other CTAs of the same grid).
+__device__ __forceinline__ float ld_cg_f32(const float* p) {
+    float v;
+    asm volatile("ld.global.cg.f32 %0, [%1];" : "=f"(v) : "l"(p));
+    return v;
+}
+__device__ __forceinline__ int ld_cg_s32(const int* p) {
+    int v;
+    asm volatile("ld.global.cg.s32 %0, [%1];" : "=r"(v) : "l"(p));
+    return v;
+}
+__device__ __forceinline__ unsigned lanemask_lt() {
+    unsigned m;
+    asm("mov.u32 %0, %%lanemask_lt;" : "=r"(m));
+    return m;
+}
+#endif
+
+}  // namespace vt

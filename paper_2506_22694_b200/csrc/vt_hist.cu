@@ -1,0 +1,312 @@
+// Token-frequency histogram (Algorithm 1: c[t_i] += 1 over the calibration stream).
+//
+// The stream is read once from HBM (4 bytes per token); everything else is arranged so that the
+// per-token work stays in shared memory:
+//   * V * 4 bytes fit in one CTA's shared memory  -> every CTA keeps a private copy of all bins
+//     (k_hist_small) and flushes the non-zero ones at the end.
+//   * otherwise (Llama-3: 128256 bins = 513 KB) a short pre-pass samples the stream, picks the
+//     hottest bins that fit (about 49.8 K of them), and the main pass keeps those in shared
+//     memory; the rare cold tokens go to L2 with one red.global each.  The hot set only steers
+//     traffic: counts are exact whichever bins were picked.
+//       hot lookup: table[id >> 5] = {32-bit membership word, slot of its first member};
+//       slot = base + popc(word & below(id)), one 8-byte shared load per token.
+#include "vt_common.cuh"
+
+namespace vt {
+
+namespace {
+
+constexpr int kThreads = 1024;
+constexpr size_t kDynSmem = 224 * 1024;        // dynamic shared memory of the counting kernels
+constexpr int kSampleSlots = 4096;             // aggregating cache of the sampling pre-pass
+constexpr int kSamplePerCta = 16384;           // ids sampled per CTA
+constexpr int kPickBins = 1024;                // sampled counts are clipped to kPickBins-1
+static_assert(kPickBins == kThreads, "one pick bin per thread");
+
+// ---- streaming loop shared by the counting kernels ---------------------------------------------
+// The CTA's share of the 16-byte-aligned body is read with four independent 128-bit loads per
+// thread per trip; the unaligned head/tail (at most 3 + 3 ids) is handled by CTA 0.
+template <class F>
+__device__ __forceinline__ void stream_ids(const int32_t* __restrict__ ids, int64_t n, F&& tally) {
+    const uintptr_t addr = reinterpret_cast<uintptr_t>(ids);
+    int64_t head = ((16 - (addr & 15)) & 15) >> 2;
+    if (head > n) head = n;
+    const int64_t nvec = (n - head) >> 2;
+    const int64_t tail0 = head + nvec * 4;
+    if (blockIdx.x == 0) {
+        if ((int64_t)threadIdx.x < head) tally((uint32_t)ids[threadIdx.x]);
+        const int64_t t = tail0 + threadIdx.x;
+        if (t < n) tally((uint32_t)ids[t]);
+    }
+    const uint4* vec = reinterpret_cast<const uint4*>(ids + head);
+    const int64_t v0 = nvec * blockIdx.x / gridDim.x;
+    const int64_t v1 = nvec * (blockIdx.x + 1) / gridDim.x;
+    for (int64_t v = v0 + threadIdx.x; v < v1; v += 4 * kThreads) {
+        uint4 a = ld_stream_u4(vec + v), b, c, d;
+        const bool pb = v + kThreads < v1, pc = v + 2 * kThreads < v1, pd = v + 3 * kThreads < v1;
+        if (pb) b = ld_stream_u4(vec + v + kThreads);
+        if (pc) c = ld_stream_u4(vec + v + 2 * kThreads);
+        if (pd) d = ld_stream_u4(vec + v + 3 * kThreads);
+        tally(a.x); tally(a.y); tally(a.z); tally(a.w);
+        if (pb) { tally(b.x); tally(b.y); tally(b.z); tally(b.w); }
+        if (pc) { tally(c.x); tally(c.y); tally(c.z); tally(c.w); }
+        if (pd) { tally(d.x); tally(d.y); tally(d.z); tally(d.w); }
+    }
+}
+
+__device__ __forceinline__ void report_bad(unsigned long long bad, Ctrl* ctrl) {
+    for (int o = 16; o; o >>= 1) bad += __shfl_xor_sync(0xffffffffu, bad, o);
+    if ((threadIdx.x & 31) == 0 && bad) {
+        atomicAdd(&ctrl->n_bad, bad);
+        atomicOr(&ctrl->flags, (uint32_t)VT_FLAG_BAD_ID);
+    }
+}
+
+// ---- all bins private to each CTA ----------------------------------------------------------------
+__global__ void __launch_bounds__(kThreads, 1)
+k_hist_small(const int32_t* __restrict__ ids, int64_t n, int32_t V, uint32_t* __restrict__ counts,
+             Ctrl* ctrl) {
+    extern __shared__ __align__(16) uint32_t s_bins[];
+    for (int i = threadIdx.x; i < V; i += kThreads) s_bins[i] = 0;
+    __syncthreads();
+    unsigned long long bad = 0;
+    stream_ids(ids, n, [&](uint32_t id) {
+        if (id < (uint32_t)V) atomicAdd(&s_bins[id], 1u);
+        else ++bad;
+    });
+    __syncthreads();
+    for (int i = threadIdx.x; i < V; i += kThreads) {
+        const int v = (i + blockIdx.x * 61) % V;        // de-phase the CTAs' flushes
+        const uint32_t c = s_bins[v];
+        if (c) atomicAdd(&counts[v], c);
+    }
+    report_bad(bad, ctrl);
+}
+
+// ---- pre-pass 1: sample the stream into sample[V] through a per-CTA aggregating cache -----------
+__global__ void __launch_bounds__(kThreads, 1)
+k_hist_sample(const int32_t* __restrict__ ids, int64_t n, int32_t V, uint32_t* __restrict__ sample) {
+    __shared__ int s_tag[kSampleSlots];
+    __shared__ uint32_t s_cnt[kSampleSlots];
+    for (int i = threadIdx.x; i < kSampleSlots; i += kThreads) { s_tag[i] = -1; s_cnt[i] = 0; }
+    __syncthreads();
+    const int64_t lo = n * blockIdx.x / gridDim.x;
+    const int64_t hi = n * (blockIdx.x + 1) / gridDim.x;
+    const int64_t end = (hi - lo > kSamplePerCta) ? lo + kSamplePerCta : hi;
+    for (int64_t i = lo + threadIdx.x; i < end; i += kThreads) {
+        const uint32_t id = (uint32_t)ids[i];
+        if (id >= (uint32_t)V) continue;
+        const uint32_t slot = (id * 2654435761u) >> 20;            // 12 bits -> kSampleSlots
+        const int old = atomicCAS(&s_tag[slot], -1, (int)id);
+        if (old == -1 || old == (int)id) atomicAdd(&s_cnt[slot], 1u);
+        else atomicAdd(&sample[id], 1u);
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < kSampleSlots; i += kThreads)
+        if (s_tag[i] >= 0) atomicAdd(&sample[s_tag[i]], s_cnt[i]);
+}
+
+// Exclusive scan over one value per thread (kThreads threads); returns the prefix, *total the sum.
+__device__ uint32_t block_excl_scan(uint32_t x, uint32_t* s_warp /*[33]*/, uint32_t* total) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    uint32_t incl = x;
+    for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t y = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += y;
+    }
+    __syncthreads();                                   // s_warp may still be read from a previous scan
+    if (lane == 31) s_warp[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+        uint32_t w = s_warp[lane], wi = w;
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t y = __shfl_up_sync(0xffffffffu, wi, o);
+            if (lane >= o) wi += y;
+        }
+        s_warp[lane] = wi - w;
+        if (lane == 31) s_warp[32] = wi;
+    }
+    __syncthreads();
+    *total = s_warp[32];
+    return s_warp[warp] + incl - x;
+}
+
+// ---- pre-pass 2: choose at most H hot bins from the sampled counts, build the lookup table ------
+// hot = sampled count >= tau, plus (in id order) as many bins with count == tau-1 as still fit.
+__global__ void __launch_bounds__(kThreads, 1)
+k_hist_pick(const uint32_t* __restrict__ sample, int32_t V, int32_t H, uint2* __restrict__ table) {
+    __shared__ uint32_t s_hist[kPickBins];
+    __shared__ uint32_t s_warp[33];
+    const int T32 = (V + 31) >> 5;
+    const int wpt = (T32 + kThreads - 1) / kThreads;
+    const int w_lo = min(T32, (int)threadIdx.x * wpt), w_hi = min(T32, w_lo + wpt);
+    s_hist[threadIdx.x] = 0;
+    __syncthreads();
+    {   // most bins were sampled a handful of times: count those in registers, one atomic per warp
+        uint32_t small[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+        for (int v = threadIdx.x; v < V; v += kThreads) {
+            const uint32_t c = min(sample[v], (uint32_t)(kPickBins - 1));
+            if (c < 8) {
+#pragma unroll
+                for (int k = 0; k < 8; ++k) small[k] += (c == (uint32_t)k);
+            } else {
+                atomicAdd(&s_hist[c], 1u);
+            }
+        }
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            uint32_t x = small[k];
+            for (int o = 16; o; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+            if ((threadIdx.x & 31) == 0 && x) atomicAdd(&s_hist[k], x);
+        }
+    }
+    __syncthreads();
+    // P[t] = #{bins with clipped count >= kPickBins-1-t}; tau = kPickBins - #{t : P[t] <= H}
+    uint32_t tot;
+    const uint32_t mine = s_hist[kPickBins - 1 - threadIdx.x];
+    const uint32_t P = block_excl_scan(mine, s_warp, &tot) + mine;
+    const int n_ok = __syncthreads_count(P <= (uint32_t)H);
+    const uint32_t tau = kPickBins - n_ok;
+    __shared__ uint32_t s_definite;
+    if (n_ok == 0 && threadIdx.x == 0) s_definite = 0;
+    if (n_ok > 0 && (int)threadIdx.x == n_ok - 1) s_definite = P;
+    __syncthreads();
+    const uint32_t quota = (uint32_t)H - s_definite;
+    // pass A: membership words for "definite" and "tie" bins
+    uint32_t tsum = 0;
+    for (int w = w_lo; w < w_hi; ++w) {
+        uint32_t def = 0, tie = 0;
+        for (int b = 0; b < 32; ++b) {
+            const int v = w * 32 + b;
+            if (v < V) {
+                const uint32_t c = min(sample[v], (uint32_t)(kPickBins - 1));
+                if (c >= tau) def |= 1u << b;
+                else if (c + 1 == tau) tie |= 1u << b;
+            }
+        }
+        table[w] = make_uint2(def, tie);
+        tsum += __popc(tie);
+    }
+    uint32_t tbase = block_excl_scan(tsum, s_warp, &tot);
+    // pass B: admit ties in id order while the quota lasts
+    uint32_t hsum = 0;
+    for (int w = w_lo; w < w_hi; ++w) {
+        const uint2 e = table[w];
+        uint32_t tie = e.y, keep = 0;
+        const uint32_t room = tbase < quota ? quota - tbase : 0u;
+        const int admit = (int)min(room, (uint32_t)__popc(tie));
+        tbase += __popc(tie);
+        for (int a = 0; a < admit; ++a) {
+            const uint32_t low = tie & (0u - tie);
+            keep |= low;
+            tie ^= low;
+        }
+        const uint32_t bits = e.x | keep;
+        table[w].x = bits;
+        hsum += __popc(bits);
+    }
+    uint32_t hbase = block_excl_scan(hsum, s_warp, &tot);
+    for (int w = w_lo; w < w_hi; ++w) {
+        table[w].y = hbase;
+        hbase += __popc(table[w].x);
+    }
+}
+
+// ---- main pass: hot bins in shared memory, cold bins through L2 ----------------------------------
+__global__ void __launch_bounds__(kThreads, 1)
+k_hist_hot(const int32_t* __restrict__ ids, int64_t n, int32_t V, uint32_t* __restrict__ counts,
+           const uint2* __restrict__ table, int32_t H, Ctrl* ctrl) {
+    extern __shared__ __align__(16) uint8_t s_raw[];
+    const int T32 = (V + 31) >> 5;
+    uint2* s_tbl = reinterpret_cast<uint2*>(s_raw);
+    uint32_t* s_cnt = reinterpret_cast<uint32_t*>(s_raw + (size_t)T32 * 8);
+    for (int i = threadIdx.x; i < T32; i += kThreads) s_tbl[i] = table[i];
+    for (int i = threadIdx.x; i < H; i += kThreads) s_cnt[i] = 0;
+    __syncthreads();
+    unsigned long long bad = 0;
+    stream_ids(ids, n, [&](uint32_t id) {
+        if (id < (uint32_t)V) {
+            const uint2 e = s_tbl[id >> 5];
+            const uint32_t bit = 1u << (id & 31);
+            if (e.x & bit) atomicAdd(&s_cnt[e.y + __popc(e.x & (bit - 1))], 1u);
+            else atomicAdd(&counts[id], 1u);
+        } else {
+            ++bad;
+        }
+    });
+    __syncthreads();
+    for (int i = threadIdx.x; i < T32; i += kThreads) {
+        const int w = (i + blockIdx.x * 27) % T32;       // de-phase the CTAs' flushes
+        const uint2 e = s_tbl[w];
+        uint32_t bits = e.x, slot = e.y;
+        while (bits) {
+            const int b = __ffs(bits) - 1;
+            bits &= bits - 1;
+            const uint32_t c = s_cnt[slot++];
+            if (c) atomicAdd(&counts[w * 32 + b], c);
+        }
+    }
+    report_bad(bad, ctrl);
+}
+
+}  // namespace
+
+HistPlan hist_plan(int32_t V) {
+    HistPlan p{};
+    p.small = (size_t)V * 4 <= kDynSmem;
+    if (p.small) { p.off_sample = p.off_table = 0; p.bytes = 0; return p; }
+    const size_t T32 = ((size_t)V + 31) / 32;
+    p.off_sample = 0;
+    p.off_table = align_up((size_t)V * 4, 256);
+    p.bytes = p.off_table + align_up(T32 * 8, 256);
+    return p;
+}
+
+cudaError_t launch_histogram(const int32_t* ids, int64_t n, int32_t V, uint32_t* counts,
+                             int accumulate, Ctrl* ctrl, uint8_t* scratch, cudaStream_t s) {
+    cudaError_t e;
+    if (!accumulate) {
+        e = cudaMemsetAsync(counts, 0, (size_t)V * 4, s);
+        if (e != cudaSuccess) return e;
+    }
+    if (n == 0) return cudaSuccess;
+    const HistPlan p = hist_plan(V);
+    const int sms = num_sms();
+    // enough CTAs to fill the chip, never more than one per 4096 ids
+    int grid = (int)((n + 4095) / 4096);
+    if (grid > sms) grid = sms;
+    if (grid < 1) grid = 1;
+    if (p.small) {
+        static bool attr_done = false;
+        if (!attr_done) {
+            e = cudaFuncSetAttribute(k_hist_small, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)kDynSmem);
+            if (e != cudaSuccess) return e;
+            attr_done = true;
+        }
+        k_hist_small<<<grid, kThreads, (size_t)V * 4, s>>>(ids, n, V, counts, ctrl);
+        count_launch();
+        return cudaGetLastError();
+    }
+    const size_t T32 = ((size_t)V + 31) / 32;
+    if (T32 * 8 + 4096 > kDynSmem) return cudaErrorInvalidValue;   // rejected earlier by the API
+    const int32_t H = (int32_t)((kDynSmem - T32 * 8) / 4);
+    uint32_t* sample = reinterpret_cast<uint32_t*>(scratch + p.off_sample);
+    uint2* table = reinterpret_cast<uint2*>(scratch + p.off_table);
+    e = cudaMemsetAsync(sample, 0, (size_t)V * 4, s);
+    if (e != cudaSuccess) return e;
+    k_hist_sample<<<grid, kThreads, 0, s>>>(ids, n, V, sample);
+    k_hist_pick<<<1, kThreads, 0, s>>>(sample, V, H, table);
+    static bool attr_done_hot = false;
+    if (!attr_done_hot) {
+        e = cudaFuncSetAttribute(k_hist_hot, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)kDynSmem);
+        if (e != cudaSuccess) return e;
+        attr_done_hot = true;
+    }
+    k_hist_hot<<<grid, kThreads, kDynSmem, s>>>(ids, n, V, counts, table, H, ctrl);
+    count_launch(3);
+    return cudaGetLastError();
+}
+
+}  // namespace vt

@@ -1,0 +1,159 @@
+// Top-K vocabulary selection (Eq. 1, first line: V_trim = V[Top-K(c,k)]) in rank order.
+//
+// The wanted order -- count descending, equal counts by ascending id -- is exactly what a STABLE
+// sort of the ids by descending count produces when it starts from ascending id order.  So the
+// whole selection is one least-significant-digit radix sort of V 32-bit counts (8-bit digits,
+// passes whose digit is constant are skipped), after which map = first K sorted ids and
+// inv_map = rank (or -1) scattered by id.
+//
+// V is about 1e5: the job is latency-bound, not bandwidth-bound.  It runs as ONE thread-block
+// cluster of 8 CTAs (one launch, no grid-wide spin): per pass each CTA counts the digits of its
+// contiguous slice, the CTAs exchange their 256 digit totals through distributed shared memory
+// between two hardware cluster barriers, and each warp then scatters its sub-slice stably using
+// warp match ranks.  Keys and ids ping-pong between two scratch arrays that stay in L2.
+#include <cooperative_groups.h>
+
+#include "vt_common.cuh"
+
+namespace cg = cooperative_groups;
+
+namespace vt {
+
+namespace {
+
+constexpr int kCluster = 8;
+constexpr int kThreads = 1024;
+constexpr int kWarps = kThreads / 32;
+constexpr int kDigits = 256;
+
+__global__ void __cluster_dims__(kCluster, 1, 1) __launch_bounds__(kThreads, 1)
+k_select_sort(const uint32_t* counts, int32_t V, int32_t K, int32_t* map, int32_t* inv_map, uint32_t* keyA, uint32_t* valA, uint32_t* keyB,
+              uint32_t* valB) {
+    cg::cluster_group cluster = cg::this_cluster();
+    const unsigned rank = cluster.block_rank();
+    __shared__ uint32_t s_wcnt[kWarps][kDigits];   // per-warp digit counts, then running offsets
+    __shared__ uint32_t s_tot[kDigits];            // this CTA's digit totals (read by the peers)
+    __shared__ uint32_t s_base[kDigits];           // global start of (digit, this CTA)
+    __shared__ uint32_t s_scan[kDigits / 32 + 1];
+    __shared__ int s_skip;
+
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int nwarps_total = kCluster * kWarps;
+    // contiguous sub-slice of each warp, a multiple of 32 long; order = (CTA rank, warp, index)
+    const int L = (((V + nwarps_total - 1) / nwarps_total) + 31) & ~31;
+    const int gw = rank * kWarps + warp;
+    const int lo = min(V, gw * L), hi = min(V, lo + L);
+
+    const uint32_t* src_key = counts;      // pass input: keys; ids are implicit until a scatter ran
+    const uint32_t* src_val = nullptr;
+    uint32_t* dst_key = keyA;
+    uint32_t* dst_val = valA;
+
+    for (int shift = 0; shift < 32; shift += 8) {
+        for (int i = threadIdx.x; i < kWarps * kDigits; i += kThreads) (&s_wcnt[0][0])[i] = 0;
+        if (threadIdx.x == 0) s_skip = 0;
+        __syncthreads();
+        // phase 1: digit counts of this warp's sub-slice (descending order: inverted digit)
+        for (int i = lo + lane; i < hi; i += 32) {
+            const uint32_t dg = 255u - ((src_key[i] >> shift) & 255u);
+            atomicAdd(&s_wcnt[warp][dg], 1u);
+        }
+        __syncthreads();
+        if (threadIdx.x < kDigits) {
+            uint32_t run = 0;
+            for (int w = 0; w < kWarps; ++w) {          // exclusive prefix over the warps
+                const uint32_t c = s_wcnt[w][threadIdx.x];
+                s_wcnt[w][threadIdx.x] = run;
+                run += c;
+            }
+            s_tot[threadIdx.x] = run;
+        }
+        cluster.sync();
+        // phase 2: global start of every (digit, CTA) from all CTAs' totals
+        uint32_t total = 0, before_me = 0;
+        if (threadIdx.x < kDigits) {
+            for (unsigned c = 0; c < kCluster; ++c) {
+                const uint32_t* peer = cluster.map_shared_rank(s_tot, c);
+                const uint32_t t = peer[threadIdx.x];
+                if (c < rank) before_me += t;
+                total += t;
+            }
+            if (total == (uint32_t)V) s_skip = 1;       // every key has this digit: nothing moves
+            // exclusive scan of `total` over the 256 digits (8 warps)
+            uint32_t incl = total;
+            for (int o = 1; o < 32; o <<= 1) {
+                const uint32_t y = __shfl_up_sync(0xffffffffu, incl, o);
+                if (lane >= o) incl += y;
+            }
+            if (lane == 31) s_scan[warp] = incl;
+            __syncwarp();
+            s_base[threadIdx.x] = incl - total + before_me;   // completed below
+        }
+        __syncthreads();
+        if (threadIdx.x < kDigits) {
+            uint32_t off = 0;
+            for (int w = 0; w < warp; ++w) off += s_scan[w];
+            s_base[threadIdx.x] += off;
+        }
+        __syncthreads();
+        const bool skip = s_skip != 0;
+        if (!skip) {
+            // phase 3: stable scatter; rank inside the warp's 32 keys by matching digits
+            for (int i0 = lo; i0 < hi; i0 += 32) {
+                const int i = i0 + lane;
+                const bool on = i < hi;
+                const unsigned active = __ballot_sync(0xffffffffu, on);
+                if (on) {
+                    const uint32_t key = src_key[i];
+                    const uint32_t val = src_val ? src_val[i] : (uint32_t)i;
+                    const uint32_t dg = 255u - ((key >> shift) & 255u);
+                    const unsigned peers = __match_any_sync(active, dg);
+                    const int leader = __ffs(peers) - 1;
+                    uint32_t old = 0;
+                    if (lane == leader) {
+                        old = s_wcnt[warp][dg];
+                        s_wcnt[warp][dg] = old + __popc(peers);
+                    }
+                    old = __shfl_sync(peers, old, leader);
+                    const uint32_t pos = s_base[dg] + old + __popc(peers & lanemask_lt());
+                    dst_key[pos] = key;
+                    dst_val[pos] = val;
+                }
+                __syncwarp();
+            }
+            __threadfence();
+        }
+        // all CTAs are done reading s_tot and writing dst before anything is reused
+        cluster.sync();
+        if (!skip) {
+            src_key = dst_key;
+            src_val = dst_val;
+            dst_key = (dst_key == keyA) ? keyB : keyA;
+            dst_val = (dst_val == valA) ? valB : valA;
+        }
+    }
+    // emit: sorted position j holds id v
+    for (int j = rank * kThreads + threadIdx.x; j < V; j += kCluster * kThreads) {
+        const int32_t v = src_val ? (int32_t)src_val[j] : j;
+        if (j < K) map[j] = v;
+        inv_map[v] = j < K ? j : -1;
+    }
+}
+
+}  // namespace
+
+size_t select_scratch_bytes(int32_t V) { return 4 * align_up((size_t)V * 4, 256); }
+
+cudaError_t launch_select_topk(const uint32_t* counts, int32_t V, int32_t K, int32_t* map,
+                               int32_t* inv_map, uint8_t* scratch, cudaStream_t s) {
+    const size_t seg = align_up((size_t)V * 4, 256);
+    uint32_t* keyA = reinterpret_cast<uint32_t*>(scratch);
+    uint32_t* valA = reinterpret_cast<uint32_t*>(scratch + seg);
+    uint32_t* keyB = reinterpret_cast<uint32_t*>(scratch + 2 * seg);
+    uint32_t* valB = reinterpret_cast<uint32_t*>(scratch + 3 * seg);
+    k_select_sort<<<kCluster, kThreads, 0, s>>>(counts, V, K, map, inv_map, keyA, valA, keyB, valB);
+    count_launch();
+    return cudaGetLastError();
+}
+
+}  // namespace vt

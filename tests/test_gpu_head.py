@@ -1,0 +1,172 @@
+"""GPU parity of the trimmed drafter head (Algorithm 2, lines 5-6) against the fp64 CPU oracle on
+seeded synthetic inputs: logits, log-probabilities, greedy / top-k / Gumbel ids and the remap."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2506_22694_b200 as vt
+import vt_inputs
+from parity_util import check_head, oracle_head
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+V3 = vt_inputs.LLAMA3_VOCAB
+
+
+def _vocab_map(V, K, seed):
+    """A map built by the real path from 1e7 synthetic ids of the corpus distribution."""
+    ids = vt_inputs.zipf_ids(10_000_000, V, 1.07, seed=seed, noise_frac=0.05, device=DEV)
+    m, inv = vt.vt_build_vocab(ids, V, K)
+    return m, inv
+
+
+def _run(h, W, m, temp, topk, u, debug=True, ws=None):
+    out = vt.vt_draft_head(h, W, m, temp, topk, u, ws=ws, debug=debug)
+    torch.cuda.synchronize()
+    return out
+
+
+def test_config1_tiny_end_to_end():
+    V, d, K, topk = 4096, 256, 1024, 4
+    ids = vt_inputs.zipf_ids(100_000, V, 1.1, seed=1001, device=DEV)
+    m, inv = vt.vt_build_vocab(ids, V, K)
+    W = vt_inputs.gaussian_bf16((V, d), 0.02, seed=1002, device=DEV)
+    Wt = vt.vt_trim_head(W, m)
+    h = vt_inputs.gaussian_bf16((1, d), 1.0, seed=1003, device=DEV)
+    T = vt_inputs.temperatures(1, 1.0, 1.0, 0, device=DEV)
+    u = vt_inputs.uniforms((1, K), seed=1004, device=DEV)
+    gi, gl, lg, lse = _run(h, Wt, m, T, topk, u)
+    ref = oracle_head(h, Wt, m, T, topk, u)
+    check_head(ref, gi, gl, T, m, lg, lse)
+    trim = inv.cpu().numpy()[gi.cpu().numpy()]                   # inverse map recovers the trimmed index
+    assert np.all(trim >= 0) and np.array_equal(m.cpu().numpy()[trim], gi.cpu().numpy())
+
+
+@pytest.mark.parametrize("B,K,d,topk,sample", [
+    (1, 8, 8, 1, True), (1, 9, 16, 9, True), (2, 100, 40, 7, True), (3, 1000, 264, 64, True),
+    (4, 5003, 1024, 8, False), (7, 2048, 3072, 8, True), (8, 777, 4096, 10, True),
+    (9, 4099, 4096, 10, True), (16, 3000, 2048, 16, True), (13, 12345, 1000, 5, True),
+    (16, 1031, 4096, 64, True), (5, 64, 8192, 4, True),
+])
+def test_small_shapes_and_ragged_tails(B, K, d, topk, sample):
+    W = vt_inputs.gaussian_bf16((K, d), 0.02, seed=K + d, device=DEV)
+    h = vt_inputs.gaussian_bf16((B, d), 1.0, seed=B + 17, device=DEV)
+    T = vt_inputs.temperatures(B, 0.5, 1.5, seed=K, device=DEV)
+    u = vt_inputs.uniforms((B, K), seed=d + 1, device=DEV) if sample else None
+    m = torch.randperm(K * 3, device=DEV)[:K].to(torch.int32)        # any injective map works for the remap
+    gi, gl, lg, lse = _run(h, W, m, T, topk, u)
+    ref = oracle_head(h, W, m, T, topk, u)
+    check_head(ref, gi, gl, T, m, lg, lse, sampled=sample)
+    if not sample:
+        assert torch.equal(gi[:, 0], gi[:, 1]) and torch.equal(gl[:, 0], gl[:, 1])
+
+
+def test_identity_map_equals_null_map_and_is_deterministic():
+    B, K, d, topk = 10, 20_000, 4096, 10
+    W = vt_inputs.gaussian_bf16((K, d), 0.02, seed=1, device=DEV)
+    h = vt_inputs.gaussian_bf16((B, d), 1.0, seed=2, device=DEV)
+    T = vt_inputs.temperatures(B, 0.7, 0.7, 0, device=DEV)
+    u = vt_inputs.uniforms((B, K), seed=3, device=DEV)
+    ident = torch.arange(K, dtype=torch.int32, device=DEV)
+    a = _run(h, W, None, T, topk, u, debug=False)
+    b = _run(h, W, ident, T, topk, u, debug=False)
+    c = _run(h, W, None, T, topk, u, debug=False)
+    assert torch.equal(a[0], b[0]) and torch.equal(a[1], b[1])
+    assert torch.equal(a[0], c[0]) and torch.equal(a[1], c[1])            # bitwise run-to-run
+
+
+def test_ties_go_to_the_lower_index():
+    B, K, d = 2, 512, 64
+    W = torch.zeros((K, d), dtype=torch.bfloat16, device=DEV)
+    W[:, 0] = 1.0
+    W[100:104, 0] = 2.0                                  # four tied maxima, everything else tied below
+    h = torch.zeros((B, d), dtype=torch.bfloat16, device=DEV)
+    h[:, 0] = 1.0
+    T = vt_inputs.temperatures(B, 1.0, 1.0, 0, device=DEV)
+    u = torch.full((B, K), 0.5, dtype=torch.float32, device=DEV)       # equal uniforms: sample == greedy
+    gi, gl = _run(h, W, None, T, 8, u, debug=False)
+    assert gi[0].tolist() == [100, 100, 101, 102, 103, 0, 1, 2, 3]
+    ref = oracle_head(h, W, None, T, 8, u)
+    assert np.array_equal(gi.cpu().numpy(), ref.ids)
+
+
+def test_uniform_edge_values_are_clamped():
+    B, K, d = 1, 256, 64
+    W = vt_inputs.gaussian_bf16((K, d), 0.02, seed=5, device=DEV)
+    h = vt_inputs.gaussian_bf16((B, d), 1.0, seed=6, device=DEV)
+    T = vt_inputs.temperatures(B, 1.0, 1.0, 0, device=DEV)
+    u = vt_inputs.uniforms((B, K), seed=7, device=DEV)
+    u[0, 10] = 0.0
+    u[0, 20] = 1.0                                       # clamps to 1 - 2^-24: a huge Gumbel, must win
+    u[0, 30] = -3.0
+    u[0, 40] = 7.0
+    gi, gl = _run(h, W, None, T, 4, u, debug=False)
+    ref = oracle_head(h, W, None, T, 4, u)
+    check_head(ref, gi, gl, T, None)
+    assert int(gi[0, 0]) in (20, 40)
+
+
+def test_bad_temperature_is_flagged_not_fatal():
+    B, K, d = 3, 300, 128
+    W = vt_inputs.gaussian_bf16((K, d), 0.02, seed=8, device=DEV)
+    h = vt_inputs.gaussian_bf16((B, d), 1.0, seed=9, device=DEV)
+    T = torch.tensor([1.0, 0.0, 0.8], dtype=torch.float32, device=DEV)
+    ws = vt.Workspace(vt.workspace_bytes(vt.VT_OP_DRAFT_HEAD, 0, 0, K, d, B, 4))
+    gi, gl = _run(h, W, None, T, 4, None, debug=False, ws=ws)
+    st, flags, _ = ws.read_status()
+    assert st == 7 and flags & vt.VT_FLAG_BAD_TEMP
+    assert gi[1].tolist() == [-1] * 5 and bool(torch.isnan(gl[1]).all())
+    ref = oracle_head(h[[0, 2]], W, None, T[[0, 2]], 4, None)
+    check_head(ref, gi[[0, 2]], gl[[0, 2]], T[[0, 2]], None, sampled=False)
+    gi2, _ = _run(h, W, None, torch.ones(B, device=DEV), 4, None, debug=False, ws=ws)   # workspace still usable
+    assert ws.read_status()[0] == 0 and int(gi2.min()) >= 0
+
+
+def test_config2_chain_drafting_trimmed_vs_full_head():
+    """V=128256, d=3072, K=32768, B=1, 7 sequential steps, greedy + top-8, against the full head."""
+    d, K, topk, steps = 3072, 32768, 8, 7
+    m, inv = _vocab_map(V3, K, seed=1102)
+    W = vt_inputs.gaussian_bf16((V3, d), 0.02, seed=1002, device=DEV)
+    Wt = vt.vt_trim_head(W, m)
+    T = vt_inputs.temperatures(1, 1.0, 1.0, 0, device=DEV)
+    ws = vt.Workspace(vt.workspace_bytes(vt.VT_OP_DRAFT_HEAD, 0, 0, V3, d, 1, topk))
+    Wb = vt_inputs.bf16_bits(W).cpu().numpy().view(np.uint16)
+    mh = m.cpu().numpy()
+    for step in range(steps):
+        h = vt_inputs.gaussian_bf16((1, d), 1.0, seed=2000 + step, device=DEV)
+        gi, gl, lg, lse = _run(h, Wt, m, T, topk, None, ws=ws)
+        ref = oracle_head(h, Wt, m, T, topk, None)
+        check_head(ref, gi, gl, T, m, lg, lse, sampled=False)
+        fi, fl, flg, flse = _run(h, W, None, T, topk, None, ws=ws)            # full K = V head, identity map
+        if step < 2:
+            full = oracle_head(h, W, None, T, topk, None)
+            check_head(full, fi, fl, T, None, flg, flse, sampled=False)
+            # trimmed logits are the full head's logits at the mapped rows (oracle: exactly)
+            assert np.array_equal(ref.logits[0], full.logits[0, mh])
+        assert torch.allclose(lg[0], flg[0, m.long()], rtol=0, atol=2e-5)
+    assert ws.read_status() == (0, 0, 0)
+
+
+@pytest.mark.parametrize("K", [8192, 32768, V3])
+def test_config3_tree_drafting_sweep(K):
+    """V=128256, d=4096, B=10 nodes, top-10, T=0.7, Gumbel sampling; K = V uses the identity map."""
+    d, B, topk = 4096, 10, 10
+    W = vt_inputs.gaussian_bf16((V3, d), 0.02, seed=1003, device=DEV)
+    if K == V3:
+        m, Wt = None, W
+    else:
+        m, _ = _vocab_map(V3, K, seed=1103)
+        Wt = vt.vt_trim_head(W, m)
+    T = vt_inputs.temperatures(B, 0.7, 0.7, 0, device=DEV)
+    ws = vt.Workspace(vt.workspace_bytes(vt.VT_OP_DRAFT_HEAD, 0, 0, K, d, B, topk))
+    depths = 6 if K == 8192 else 2
+    slack = 0
+    for depth in range(depths):
+        h = vt_inputs.gaussian_bf16((B, d), 1.0, seed=3000 + depth, device=DEV)
+        u = vt_inputs.uniforms((B, K), seed=4000 + depth, device=DEV)
+        gi, gl, lg, lse = _run(h, Wt, m, T, topk, u, ws=ws)
+        ref = oracle_head(h, Wt, m, T, topk, u)
+        slack += check_head(ref, gi, gl, T, m, lg, lse)
+    assert slack <= 0.02 * depths * B * (1 + topk)
+    assert ws.read_status() == (0, 0, 0)

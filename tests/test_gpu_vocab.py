@@ -1,0 +1,168 @@
+"""GPU parity of the vocabulary build (Algorithm 1, Eq. 1) against the CPU oracle: bit-exact
+histograms, maps, inverse maps and gathered heads, on seeded synthetic id streams."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2506_22694_b200 as vt
+import vt_inputs
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def _u32(t: torch.Tensor) -> np.ndarray:
+    return t.cpu().numpy().view(np.uint32).astype(np.uint64)
+
+
+def _assert_clean(ws):
+    st, flags, bad = ws.read_status()
+    assert (st, flags, bad) == (0, 0, 0)
+
+
+@pytest.mark.parametrize("n,V", [(0, 4096), (1, 4096), (7, 100), (100_000, 4096), (250_003, 50_000),
+                                 (1_000_003, 128256), (3_000_000, 57_345), (777, 128256)])
+def test_histogram_matches_oracle(n, V):
+    ids = vt_inputs.zipf_ids(n, V, 1.1, seed=100 + n % 97, noise_frac=0.05, device=DEV) if n else \
+        torch.empty(0, dtype=torch.int32, device=DEV)
+    ws = vt.Workspace(vt.workspace_bytes(vt.VT_OP_HISTOGRAM, n, V))
+    counts = vt.vt_histogram(ids, V, ws=ws)
+    ref, bad = oracle.histogram(ids.cpu().numpy(), V)
+    assert bad == 0
+    assert np.array_equal(_u32(counts), ref)
+    _assert_clean(ws)
+
+
+def test_histogram_unaligned_start_and_accumulate():
+    V = 128256
+    base = vt_inputs.zipf_ids(2_000_011, V, 1.07, seed=7, noise_frac=0.05, device=DEV)
+    ws = vt.Workspace(vt.workspace_bytes(vt.VT_OP_HISTOGRAM, base.numel(), V))
+    for off in (1, 2, 3):
+        ids = base[off:]                                   # 4-byte aligned only
+        counts = vt.vt_histogram(ids, V, ws=ws)
+        ref, _ = oracle.histogram(ids.cpu().numpy(), V)
+        assert np.array_equal(_u32(counts), ref)
+    counts = vt.vt_histogram(base[:900_000], V, ws=ws)
+    vt.vt_histogram(base[900_000:], V, counts=counts, accumulate=True, ws=ws)
+    ref, _ = oracle.histogram(base.cpu().numpy(), V)
+    assert np.array_equal(_u32(counts), ref)
+    _assert_clean(ws)
+
+
+@pytest.mark.parametrize("V", [4096, 128256])
+def test_histogram_skips_and_reports_out_of_range_ids(V):
+    ids = vt_inputs.zipf_ids(300_000, V, 1.1, seed=9, device=DEV)
+    ids[::1000] = V                 # just past the end
+    ids[1::1000] = -1
+    ids[2::5000] = 2**31 - 1
+    ws = vt.Workspace(vt.workspace_bytes(vt.VT_OP_HISTOGRAM, ids.numel(), V))
+    counts = vt.vt_histogram(ids, V, ws=ws)
+    ref, bad = oracle.histogram(ids.cpu().numpy(), V)
+    assert bad > 0 and np.array_equal(_u32(counts), ref)
+    st, flags, n_bad = ws.read_status()
+    assert st == 2 and flags & vt.VT_FLAG_BAD_ID and n_bad == bad
+    assert ws.read_status() == (0, 0, 0)                   # flags are cleared by the read
+
+
+def test_histogram_degenerate_streams():
+    V = 128256
+    ws = vt.Workspace(vt.workspace_bytes(vt.VT_OP_HISTOGRAM, 1 << 20, V))
+    one = torch.full((1 << 20,), 77_777, dtype=torch.int32, device=DEV)       # a single hot bin
+    c = _u32(vt.vt_histogram(one, V, ws=ws))
+    assert c[77_777] == 1 << 20 and c.sum() == 1 << 20
+    ramp = (torch.arange(1 << 20, device=DEV, dtype=torch.int32) % V).contiguous()  # every bin cold and equal
+    ref, _ = oracle.histogram(ramp.cpu().numpy(), V)
+    assert np.array_equal(_u32(vt.vt_histogram(ramp, V, ws=ws)), ref)
+
+
+@pytest.mark.parametrize("V,K", [(1, 1), (6, 3), (4096, 1024), (4096, 4096), (128256, 8192), (128256, 32768),
+                                 (128256, 128256), (131072, 1), (200_001, 70_000)])
+def test_select_topk_matches_oracle(V, K):
+    n = min(20 * V, 3_000_000)
+    ids = vt_inputs.zipf_ids(n, V, 1.07, seed=V + K, noise_frac=0.05, device=DEV)
+    counts = vt.vt_histogram(ids, V)
+    m, inv = vt.vt_select_topk(counts, K)
+    rm, rinv = oracle.select_topk(_u32(counts), K)
+    assert np.array_equal(m.cpu().numpy(), rm)
+    assert np.array_equal(inv.cpu().numpy(), rinv)
+
+
+def test_select_topk_extreme_count_patterns():
+    V, K = 70_000, 1234
+    pats = {
+        "all_equal": torch.full((V,), 5, dtype=torch.int32),
+        "all_zero": torch.zeros(V, dtype=torch.int32),
+        "two_levels": (torch.arange(V) % 2).to(torch.int32),
+        "wide": torch.from_numpy(np.random.default_rng(1).integers(0, 2**32, V, dtype=np.uint64)
+                                 .astype(np.uint32).view(np.int32)),
+        "descending": torch.arange(V, 0, -1, dtype=torch.int32),
+        "high_byte_only": (torch.from_numpy(np.random.default_rng(2).integers(0, 200, V).astype(np.int32)) << 24),
+    }
+    for name, c in pats.items():
+        m, inv = vt.vt_select_topk(c.to(DEV), K)
+        rm, rinv = oracle.select_topk(c.numpy().view(np.uint32).astype(np.uint64), K)
+        assert np.array_equal(m.cpu().numpy(), rm), name
+        assert np.array_equal(inv.cpu().numpy(), rinv), name
+
+
+def test_config1_build_vocab_and_gather():
+    """Tiny end-to-end case: V=4096, K=1024, 100k Zipf(1.1) ids, d=256."""
+    V, K, d = 4096, 1024, 256
+    ids = vt_inputs.zipf_ids(100_000, V, 1.1, seed=1001, device=DEV)
+    m, inv = vt.vt_build_vocab(ids, V, K)
+    rm, rinv, _, _ = oracle.build_vocab(ids.cpu().numpy(), V, K)
+    assert np.array_equal(m.cpu().numpy(), rm) and np.array_equal(inv.cpu().numpy(), rinv)
+    W = vt_inputs.gaussian_bf16((V, d), 0.02, seed=1002, device=DEV)
+    Wt = vt.vt_trim_head(W, m)
+    ref = oracle.trim_head(vt_inputs.bf16_bits(W).cpu().numpy(), rm)
+    assert np.array_equal(vt_inputs.bf16_bits(Wt).cpu().numpy().view(np.uint16), ref)
+
+
+def test_build_vocab_from_host_memory_matches_device_path():
+    V, K = 128256, 8192
+    ids = vt_inputs.zipf_ids(40_000_000, V, 1.07, seed=55, noise_frac=0.05, device=DEV)
+    m, inv = vt.vt_build_vocab(ids, V, K)
+    host = ids.cpu().pin_memory()
+    m2, inv2 = vt.vt_build_vocab(host, V, K)
+    torch.cuda.synchronize()
+    assert torch.equal(m, m2) and torch.equal(inv, inv2)
+    rm, rinv, _, _ = oracle.build_vocab(host.numpy(), V, K)
+    assert np.array_equal(m.cpu().numpy(), rm) and np.array_equal(inv.cpu().numpy(), rinv)
+
+
+def test_trim_head_identity_and_bad_map_entries():
+    V, d = 1000, 64
+    W = vt_inputs.gaussian_bf16((V, d), 0.02, seed=3, device=DEV)
+    ident = torch.arange(V, dtype=torch.int32, device=DEV)
+    assert torch.equal(vt_inputs.bf16_bits(vt.vt_trim_head(W, ident)), vt_inputs.bf16_bits(W))
+    ws = vt.Workspace(vt.workspace_bytes(vt.VT_OP_TRIM_HEAD))
+    bad = torch.tensor([5, -1, V, 7], dtype=torch.int32, device=DEV)
+    Wt = vt.vt_trim_head(W, bad, ws=ws)
+    st, flags, _ = ws.read_status()
+    assert st == 2 and flags & vt.VT_FLAG_BAD_MAP
+    assert torch.equal(vt_inputs.bf16_bits(Wt[0]), vt_inputs.bf16_bits(W[5]))
+    assert torch.equal(vt_inputs.bf16_bits(Wt[3]), vt_inputs.bf16_bits(W[7]))
+    assert int(vt_inputs.bf16_bits(Wt[1:3]).abs().sum()) == 0
+
+
+def test_config5_corpus_scale_build_and_gather():
+    """1e9 ids over V=128256 (95% Zipf(1.07) over a seeded permutation, 5% uniform noise), top-K
+    for K in {8192, 32768}, then the gather of W_trim[K,4096]: all outputs bit-exact."""
+    V, d, n = 128256, 4096, 1_000_000_000
+    ids = vt_inputs.zipf_ids(n, V, 1.07, seed=1005, noise_frac=0.05, device=DEV)
+    ws = vt.Workspace(vt.workspace_bytes(vt.VT_OP_BUILD_VOCAB, n, V, 32768))
+    counts = vt.vt_histogram(ids, V, ws=ws)
+    host_ids = ids.cpu().numpy()
+    ref_counts, bad = oracle.histogram(host_ids, V)
+    assert bad == 0 and int(ref_counts.sum()) == n
+    assert np.array_equal(_u32(counts), ref_counts)
+    W = vt_inputs.gaussian_bf16((V, d), 0.02, seed=1006, device=DEV)
+    Wbits = vt_inputs.bf16_bits(W).cpu().numpy().view(np.uint16)
+    for K in (8192, 32768):
+        m, inv = vt.vt_build_vocab(ids, V, K, ws=ws)
+        rm, rinv = oracle.select_topk(ref_counts, K)
+        assert np.array_equal(m.cpu().numpy(), rm) and np.array_equal(inv.cpu().numpy(), rinv)
+        Wt = vt.vt_trim_head(W, m)
+        assert np.array_equal(vt_inputs.bf16_bits(Wt).cpu().numpy().view(np.uint16), oracle.trim_head(Wbits, rm))
+    _assert_clean(ws)
