@@ -85,6 +85,9 @@ vt_status vt_read_status(void *ws, void *stream, uint32_t *flags, uint64_t *n_ba
 
 const char *vt_status_str(vt_status s);
 
+/* Text of the CUDA runtime error behind the calling thread's most recent VT_ERR_CUDA. */
+const char *vt_last_cuda_error(void);
+
 /* Number of kernels launched by this library since it was loaded (host counter, for
  * benchmarks that must report their launch count). */
 uint64_t vt_launch_count(void);

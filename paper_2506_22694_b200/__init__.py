@@ -29,6 +29,7 @@ VT_CTRL_BYTES = 256
 
 EXPORTS = (
     "vt_workspace_bytes", "vt_workspace_init", "vt_read_status", "vt_status_str", "vt_launch_count",
+    "vt_last_cuda_error",
     "vt_histogram", "vt_select_topk", "vt_build_vocab", "vt_build_vocab_host", "vt_trim_head",
     "vt_draft_head", "vt_draft_head_debug", "vt_draft_head_host",
 )
@@ -37,7 +38,8 @@ EXPORTS = (
 class VocabTrimError(RuntimeError):
     def __init__(self, call: str, status: int):
         self.status = status
-        super().__init__("%s failed: %s (status %d)" % (call, status_str(status), status))
+        detail = " [%s]" % lib().vt_last_cuda_error().decode() if status == 4 else ""
+        super().__init__("%s failed: %s (status %d)%s" % (call, status_str(status), status, detail))
 
 
 _lib = None
@@ -58,6 +60,7 @@ def lib() -> ctypes.CDLL:
         L.vt_status_str.restype = c_char_p
         L.vt_status_str.argtypes = [c_int]
         L.vt_launch_count.restype = c_uint64
+        L.vt_last_cuda_error.restype = c_char_p
         L.vt_histogram.argtypes = [c_void_p, c_int64, c_int32, c_void_p, c_int, c_void_p, c_size_t, c_void_p]
         L.vt_select_topk.argtypes = [c_void_p, c_int32, c_int32, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
         L.vt_build_vocab.argtypes = [c_void_p, c_int64, c_int32, c_int32, c_void_p, c_void_p, c_void_p,

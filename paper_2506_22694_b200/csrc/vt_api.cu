@@ -25,7 +25,12 @@ namespace {
 
 inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 inline cudaStream_t as_stream(void* s) { return reinterpret_cast<cudaStream_t>(s); }
-inline vt_status from_cuda(cudaError_t e) { return e == cudaSuccess ? VT_OK : VT_ERR_CUDA; }
+thread_local cudaError_t t_last_cuda = cudaSuccess;
+inline vt_status from_cuda(cudaError_t e) {
+    if (e == cudaSuccess) return VT_OK;
+    t_last_cuda = e;
+    return VT_ERR_CUDA;
+}
 
 constexpr int64_t kHostChunkIds = 1 << 24;     // ids per staged chunk of vt_build_vocab_host
 
@@ -151,6 +156,8 @@ const char* vt_status_str(vt_status s) {
 
 uint64_t vt_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
+const char* vt_last_cuda_error(void) { return cudaGetErrorString(t_last_cuda); }
+
 vt_status vt_histogram(const int32_t* ids, int64_t n, int32_t V, uint32_t* counts, int accumulate,
                        void* ws, size_t ws_bytes, void* stream) {
     if (n < 0 || n >= ((int64_t)1 << 32) || V < 1 || !counts || (n > 0 && !ids)) return VT_ERR_INVALID_ARG;
@@ -186,7 +193,7 @@ vt_status vt_build_vocab(const int32_t* ids, int64_t n, int32_t V, int32_t K, in
     uint8_t* inner = base + VT_CTRL_BYTES + align_up((size_t)V * 4, 256);
     cudaStream_t s = as_stream(stream);
     cudaError_t e = launch_histogram(ids, n, V, counts, 0, reinterpret_cast<Ctrl*>(base), inner, s);
-    if (e != cudaSuccess) return VT_ERR_CUDA;
+    if (e != cudaSuccess) return from_cuda(e);
     return from_cuda(launch_select_topk(counts, V, K, map, inv_map, inner, s));
 }
 
@@ -307,7 +314,7 @@ vt_status vt_draft_head_host(const uint16_t* h_host, const uint16_t* W_trim, con
     if (e == cudaSuccess) e = cudaMemcpyAsync(dt, temp_host, (size_t)B * 4, cudaMemcpyHostToDevice, s);
     if (e == cudaSuccess && uniforms_host)
         e = cudaMemcpyAsync(du, uniforms_host, (size_t)B * K * 4, cudaMemcpyHostToDevice, s);
-    if (e != cudaSuccess) return VT_ERR_CUDA;
+    if (e != cudaSuccess) return from_cuda(e);
     st = vt_draft_head(dh, W_trim, map, B, K, d, dt, topk, uniforms_host ? du : nullptr, di, dl, ws,
                        head_part, stream);
     if (st != VT_OK) return st;

@@ -30,6 +30,7 @@ constexpr int kPartStride = 136;        // floats per warp partial tile: 16 x 8 
 constexpr int kMaxB = 16;
 constexpr int kMaxGrid = 160;           // merge: each lane owns at most kMaxOwn CTA records
 constexpr int kMaxOwn = kMaxGrid / 32;
+constexpr size_t kMaxDynSmem = 227 * 1024 - 1024;   // opt-in limit minus static shared memory
 constexpr int kRecHdr = 8;              // record: m, s, gumbel score, gumbel j, gumbel z, pad[3]
 
 __host__ __device__ inline int rec_words(int topk) { return kRecHdr + 2 * topk; }
@@ -364,7 +365,7 @@ cudaError_t launch_variant(const HeadArgs& a, Ctrl* ctrl, float* recs, int grid,
     cudaGetDevice(&dev);
     if (dev < 0 || dev >= 64 || !attr_done[dev]) {
         cudaError_t e = cudaFuncSetAttribute(k_head_skinny<U, NBUF, TWO>,
-                                             cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+                                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxDynSmem);
         if (e != cudaSuccess) return e;
         if (dev >= 0 && dev < 64) attr_done[dev] = 1;
     }
@@ -377,7 +378,7 @@ cudaError_t launch_variant(const HeadArgs& a, Ctrl* ctrl, float* recs, int grid,
 
 bool head_skinny_supported(int32_t B, int32_t d) {
     if (B < 1 || B > kMaxB || d < 8 || (d & 7)) return false;
-    return skinny_smem_bytes(skinny_kbw(d), B > 8) <= (size_t)227 * 1024;
+    return skinny_smem_bytes(skinny_kbw(d), B > 8) <= kMaxDynSmem;
 }
 
 size_t head_skinny_scratch_bytes(int32_t B, int32_t K, int32_t topk) {
