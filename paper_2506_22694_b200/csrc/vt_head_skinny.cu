@@ -1,21 +1,29 @@
 // Trimmed LM head for a few hidden rows (B <= 16), fused with its sampling epilogue
 // (Algorithm 2, lines 5-6: drafter head over the trimmed vocabulary, then the index mapper).
 //
-// HBM-bound: the only large operand is W_trim [K,d] bf16, read exactly once.  The vocabulary rows
-// are split over one persistent CTA per SM (contiguous slabs of 8-row blocks); inside a CTA the 16
-// warps split the hidden dimension, every lane keeping a ring of independent 128-bit streaming
-// loads of W in flight (no shared-memory staging of W).  The inner product runs on the warp-level
-// tensor instruction mma.m16n8k16 (bf16 in, fp32 accumulate) with the hidden rows as the 16-row
-// operand and 8 vocabulary rows as the 8-column operand: a dot product does not care in which
-// order k is visited, so the 16 contiguous bytes a lane loads from a W row serve directly as its
-// fragment as long as the h fragment is taken from the same k positions.  This only off-loads the
-// FMAs (at B = 10 the fp32 pipe could not keep up with HBM); the kernel remains a streaming read.
+// HBM-bound: the only large operand is W_trim [K,d] bf16, read exactly once.  One persistent CTA
+// per SM owns a contiguous slab of vocabulary rows and streams it through a shared-memory ring
+// filled by the bulk-copy engine (cp.async.bulk + mbarrier transaction counts): one warp issues,
+// besides its share of the math, one multi-kilobyte copy per vocabulary row of a stage (8 rows x
+// up to 2048 columns), refilling each stage one step after it was released, so well over 100 KB
+// per SM stay in flight whatever the other warps are doing.
 //
-// Per 8-row block the 16 partial sums are reduced through shared memory and one warp per hidden
-// row updates, on chip: running max / sum-exp of z = logit / T, the row's top-k list, and the
-// Gumbel-max candidate from the caller's uniforms.  Logits never go to HBM.  Each CTA leaves one
-// small record per hidden row; the last CTA to finish (atomic ticket, no spinning) merges the
-// records in CTA order, remaps trimmed indices through `map` and writes the outputs.
+// Sixteen consumer warps split the hidden dimension.  Each keeps its slice of h in registers as
+// ready-made operand fragments and feeds the warp-level tensor instruction mma.m16n8k16 (bf16 in,
+// fp32 accumulate) with the hidden rows as the 16-row operand and the stage's 8 vocabulary rows
+// as the 8-column operand.  A dot product does not care in which order k is visited, so the 16
+// contiguous bytes a lane reads from a W row serve directly as its fragment as long as the h
+// fragment is taken from the same k positions.  The tensor instruction only off-loads the FMAs
+// (at B = 10 the fp32 pipe could not keep up with HBM); the kernel remains a streaming read.
+//
+// Per 8-row block the 16 partial tiles meet in shared memory and warp b updates hidden row b, on
+// chip: running max / sum-exp of z = logit / T, the row's top-k list, and the Gumbel-max
+// candidate from the caller's uniforms.  Logits never go to HBM.  Warps only meet through
+// mbarriers (stage full/empty, partial tile full/empty), never through a CTA-wide barrier inside
+// the loop.  Each CTA leaves one small record per hidden row; the last CTA to finish (atomic
+// ticket, no spinning) merges the records in CTA order, remaps trimmed indices through `map` and
+// writes the outputs.  Every wait is bounded: on expiry the CTA raises VT_FLAG_TIMEOUT, drains
+// its own copies and leaves.
 #include <math_constants.h>
 
 #include "vt_common.cuh"
@@ -24,16 +32,74 @@ namespace vt {
 
 namespace {
 
-constexpr int kNW = 16;                 // warps per CTA: split of the hidden dimension
+constexpr int kNW = 16;                          // consumer warps: split of the hidden dimension
 constexpr int kThreads = kNW * 32;
-constexpr int kPartStride = 136;        // floats per warp partial tile: 16 x 8 + pad (bank spread)
+constexpr int kLag = 2;                          // a stage is refilled kLag items after its release
+constexpr int kRows = 8;                         // vocabulary rows per stage (mma n)
+constexpr int kMaxStages = 8;
 constexpr int kMaxB = 16;
-constexpr int kMaxGrid = 160;           // merge: each lane owns at most kMaxOwn CTA records
+constexpr int kMaxGrid = 160;                    // merge: each lane owns at most kMaxOwn CTA records
 constexpr int kMaxOwn = kMaxGrid / 32;
-constexpr size_t kMaxDynSmem = 227 * 1024 - 1024;   // opt-in limit minus static shared memory
-constexpr int kRecHdr = 8;              // record: m, s, gumbel score, gumbel j, gumbel z, pad[3]
+constexpr size_t kSmemLimit = 227 * 1024 - 1024; // opt-in limit minus static shared memory
+constexpr int kCand = 128;                       // candidate buffer entries per hidden row
+constexpr int kSelPerLane = (VT_MAX_TOPK + kCand) / 32;
+constexpr int kMergeDepth = 4;                   // list entries per CTA staged on chip by the merge
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 
-__host__ __device__ inline int rec_words(int topk) { return kRecHdr + 2 * topk; }
+__host__ __device__ inline int rec_fields(int topk) { return 5 + 2 * topk; }
+
+struct Geo {
+    int RB;            // row blocks of 8 vocabulary rows
+    int S;             // ring stages
+    int pitch;         // bytes between rows of a stage (odd multiple of 64: conflict-free 128-bit reads)
+    int part_stride;   // floats per warp partial tile
+    int ring_bytes;
+};
+
+// ---- mbarrier / bulk copy primitives -------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint64_t* b, int count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(b)), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* b, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(b)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* b) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(b)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint64_t* b, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
+        : "=r"(ok) : "r"(smem_u32(b)), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+// Bounded wait; false when the CTA is aborting or the time limit expired (which starts an abort).
+__device__ __forceinline__ bool mbar_wait(uint64_t* b, uint32_t parity, volatile int* abort_flag) {
+    if (mbar_try(b, parity)) return true;
+    const unsigned long long t0 = global_ns();
+    for (;;) {
+#pragma unroll 1
+        for (int i = 0; i < 128; ++i)
+            if (mbar_try(b, parity)) return true;
+        if (*abort_flag) return false;
+        if (global_ns() - t0 > kWaitLimitNs) { *abort_flag = 1; return false; }
+    }
+}
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint64_t* bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ uint4 lds_u4(uint32_t addr) {
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    return v;
+}
 
 __device__ __forceinline__ void mma_bf16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2,
                                          uint32_t a3, uint32_t b0, uint32_t b1) {
@@ -56,104 +122,363 @@ __device__ __forceinline__ void lse_merge(float& m, float& s, float m2, float s2
     m = M;
 }
 
-struct Smem {
-    float* part;       // [2][kNW][kPartStride]
-    float* topv;       // [kMaxB][VT_MAX_TOPK]
-    int* topj;         // [kMaxB][VT_MAX_TOPK]
-    uint4* h;          // [KBpad][halves][32]
+
+// Order-preserving map of a float onto unsigned integers (and back); no NaN ever reaches it.
+__device__ __forceinline__ unsigned f2ord(float f) {
+    const unsigned u = __float_as_uint(f);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__device__ __forceinline__ float ord2f(unsigned k) {
+    return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
+}
+
+struct TopkState {
+    int cnt;       // entries in the list
+    float thr;     // value of entry topk-1 once the list is full, else -inf
 };
 
-template <int U, int NBUF, bool TWO>
+// Warp-cooperative selection: the best min(topk, cnt + n_c) of a sorted list (tv/tj, cnt entries) and
+// a batch of unsorted candidates (cv/cj, n_c entries) become the new sorted list (descending value,
+// ties to the lower index).  All elements sit in registers (at most kSelPerLane per lane); every
+// round is two warp reductions.  Runs once per full candidate buffer, so rarely once `thr` is warm.
+__device__ __noinline__ TopkState topk_flush(float* tv, int* tj, int cnt, const float* cv, const int* cj, int n_c,
+                                             int topk) {
+    const int lane = threadIdx.x & 31;
+    unsigned ek[kSelPerLane];
+    int ej[kSelPerLane];
+    __syncwarp();
+#pragma unroll
+    for (int i = 0; i < kSelPerLane; ++i) {
+        const int idx = lane + 32 * i;
+        ek[i] = 0u;
+        ej[i] = 0x7fffffff;
+        if (idx < cnt) { ek[i] = f2ord(tv[idx]); ej[i] = tj[idx]; }
+        else if (idx - cnt < n_c) { ek[i] = f2ord(cv[idx - cnt]); ej[i] = cj[idx - cnt]; }
+    }
+    __syncwarp();
+    const int out = min(topk, cnt + n_c);
+    unsigned kmax = 0u;
+    for (int r = 0; r < out; ++r) {
+        unsigned lk = ek[0];
+        int lj = ej[0];
+#pragma unroll
+        for (int i = 1; i < kSelPerLane; ++i)
+            if (ek[i] > lk || (ek[i] == lk && ej[i] < lj)) { lk = ek[i]; lj = ej[i]; }
+        kmax = __reduce_max_sync(0xffffffffu, lk);
+        const unsigned jmin = __reduce_min_sync(0xffffffffu, lk == kmax ? (unsigned)lj : 0xffffffffu);
+        if (lk == kmax && (unsigned)lj == jmin) {
+#pragma unroll
+            for (int i = 0; i < kSelPerLane; ++i)
+                if (ek[i] == lk && ej[i] == lj) { ek[i] = 0u; ej[i] = 0x7fffffff; }
+        }
+        if (lane == 0) { tv[r] = ord2f(kmax); tj[r] = (int)jmin; }
+    }
+    __syncwarp();
+    return TopkState{out, (out == topk) ? ord2f(kmax) : -CUDART_INF_F};
+}
+
+// Records: one word per (hidden row b, field f, CTA c) at recs[(b * rec_fields(topk) + f) * kMaxGrid + c],
+// CTA index fastest so that the merging warp reads every field with coalesced loads.
+// Fields: 0 m, 1 s, 2 Gumbel score, 3 Gumbel j, 4 Gumbel z, 5+r value of list entry r, 5+topk+r its index.
+__device__ __forceinline__ size_t rec_at(int b, int f, int topk) {
+    return ((size_t)b * rec_fields(topk) + f) * kMaxGrid;
+}
+
+// Last CTA: merge all CTA records of hidden row b in CTA order (one warp per row), remap through
+// `map`, write the outputs.  All loads of a phase are issued before the first use, so the merge
+// costs a couple of L2 round trips.  `stage` is idle shared memory for the heads of the lists.
+struct MergeOut {
+    const int32_t* map;
+    int32_t* out_ids;
+    float* out_logprobs;
+    float* dbg_lse;
+    int topk;
+    int sampled;       // uniforms were given: column 0 is the Gumbel-max draw
+};
+__device__ __noinline__ void merge_records(const int32_t* map, int32_t* out_ids, float* out_logprobs, float* dbg_lse,
+                                           int topk, int sampled, Ctrl* ctrl, const float* recs, int b, bool row_ok,
+                                           float* stage) {
+    const MergeOut a{map, out_ids, out_logprobs, dbg_lse, topk, sampled};
+    const int lane = threadIdx.x & 31;
+    const int G = gridDim.x;
+    const int* irecs = reinterpret_cast<const int*>(recs);
+    const int depth = min(topk, kMergeDepth);
+    float hm[kMaxOwn], hs[kMaxOwn], hgs[kMaxOwn], hgz[kMaxOwn];
+    int hgj[kMaxOwn];
+    float ev[kMergeDepth][kMaxOwn];
+    int ej[kMergeDepth][kMaxOwn];
+#pragma unroll
+    for (int o = 0; o < kMaxOwn; ++o) {
+        const int c = lane + 32 * o;
+        const bool on = c < G;
+        hm[o] = on ? ld_cg_f32(recs + rec_at(b, 0, topk) + c) : -CUDART_INF_F;
+        hs[o] = on ? ld_cg_f32(recs + rec_at(b, 1, topk) + c) : 0.f;
+        hgs[o] = on ? ld_cg_f32(recs + rec_at(b, 2, topk) + c) : -CUDART_INF_F;
+        hgj[o] = on ? ld_cg_s32(irecs + rec_at(b, 3, topk) + c) : -1;
+        hgz[o] = on ? ld_cg_f32(recs + rec_at(b, 4, topk) + c) : 0.f;
+#pragma unroll
+        for (int r = 0; r < kMergeDepth; ++r) {
+            const bool on2 = on && r < depth;
+            ev[r][o] = on2 ? ld_cg_f32(recs + rec_at(b, 5 + r, topk) + c) : -CUDART_INF_F;
+            ej[r][o] = on2 ? ld_cg_s32(irecs + rec_at(b, 5 + topk + r, topk) + c) : -1;
+        }
+    }
+    float M = -CUDART_INF_F, Ssum = 0.f, GS = -CUDART_INF_F, GZ = 0.f;
+    int GJ = -1;
+#pragma unroll
+    for (int o = 0; o < kMaxOwn; ++o) {
+        lse_merge(M, Ssum, hm[o], hs[o]);
+        if (hgj[o] >= 0 && (GJ < 0 || better(hgs[o], hgj[o], GS, GJ))) { GS = hgs[o]; GJ = hgj[o]; GZ = hgz[o]; }
+    }
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const float m2 = __shfl_xor_sync(0xffffffffu, M, o), s2 = __shfl_xor_sync(0xffffffffu, Ssum, o);
+        lse_merge(M, Ssum, m2, s2);
+        const float gs2 = __shfl_xor_sync(0xffffffffu, GS, o), gz2 = __shfl_xor_sync(0xffffffffu, GZ, o);
+        const int gj2 = __shfl_xor_sync(0xffffffffu, GJ, o);
+        if (gj2 >= 0 && (GJ < 0 || better(gs2, gj2, GS, GJ))) { GS = gs2; GJ = gj2; GZ = gz2; }
+    }
+    const float lse = M + logf(Ssum);
+    // heads of the lists: entry r of CTA c at stv[r * kMaxGrid + c]
+    float* stv = stage + (size_t)b * (2 * kMergeDepth * kMaxGrid);
+    int* stj = reinterpret_cast<int*>(stv) + kMergeDepth * kMaxGrid;
+#pragma unroll
+    for (int o = 0; o < kMaxOwn; ++o)
+#pragma unroll
+        for (int r = 0; r < kMergeDepth; ++r) {
+            stv[r * kMaxGrid + lane + 32 * o] = ev[r][o];
+            stj[r * kMaxGrid + lane + 32 * o] = ej[r][o];
+        }
+    __syncwarp();
+    // k rounds; every lane keeps the current head of each of its lists in registers, a round is two
+    // warp reductions, and the winner alone advances (from the staged entries, else from global memory)
+    int head[kMaxOwn], cj[kMaxOwn];
+    unsigned ck[kMaxOwn];
+#pragma unroll
+    for (int o = 0; o < kMaxOwn; ++o) {
+        head[o] = 0;
+        const bool live = (lane + 32 * o < G) && ej[0][o] >= 0;
+        ck[o] = live ? f2ord(ev[0][o]) : 0u;
+        cj[o] = live ? ej[0][o] : 0x7fffffff;
+    }
+    float res_v[2] = {0.f, 0.f};
+    int res_j[2] = {-1, -1};
+    for (int r = 0; r < topk; ++r) {
+        unsigned lk = ck[0];
+        int lj = cj[0];
+#pragma unroll
+        for (int o = 1; o < kMaxOwn; ++o)
+            if (ck[o] > lk || (ck[o] == lk && cj[o] < lj)) { lk = ck[o]; lj = cj[o]; }
+        const unsigned kmax = __reduce_max_sync(0xffffffffu, lk);
+        const unsigned jmin = __reduce_min_sync(0xffffffffu, lk == kmax ? (unsigned)lj : 0xffffffffu);
+        if (kmax == 0u) break;                                // every list is exhausted
+        if (lk == kmax && (unsigned)lj == jmin) {
+#pragma unroll
+            for (int o = 0; o < kMaxOwn; ++o)
+                if (ck[o] == lk && cj[o] == lj) {
+                    const int c = lane + 32 * o;
+                    const int hd = ++head[o];
+                    float v = -CUDART_INF_F;
+                    int j = -1;
+                    if (hd < depth) { v = stv[hd * kMaxGrid + c]; j = stj[hd * kMaxGrid + c]; }
+                    else if (hd < topk) {
+                        v = ld_cg_f32(recs + rec_at(b, 5 + hd, topk) + c);
+                        j = ld_cg_s32(irecs + rec_at(b, 5 + topk + hd, topk) + c);
+                    }
+                    ck[o] = j >= 0 ? f2ord(v) : 0u;
+                    cj[o] = j >= 0 ? j : 0x7fffffff;
+                }
+        }
+        if (lane == (r & 31)) {
+            if (r < 32) { res_v[0] = ord2f(kmax); res_j[0] = (int)jmin; }
+            else { res_v[1] = ord2f(kmax); res_j[1] = (int)jmin; }
+        }
+    }
+    const int row_w = 1 + topk;
+    int* oid = a.out_ids + (size_t)b * row_w;
+    float* olp = a.out_logprobs + (size_t)b * row_w;
+    bool miss = false;
+#pragma unroll
+    for (int sl = 0; sl < 2; ++sl) {
+        const int r = lane + 32 * sl;
+        if (r < topk) {
+            const bool ok = row_ok && res_j[sl] >= 0;
+            const int id = ok ? (a.map ? __ldg(a.map + res_j[sl]) : res_j[sl]) : -1;
+            const float lp = ok ? res_v[sl] - lse : CUDART_NAN_F;
+            oid[1 + r] = id;
+            olp[1 + r] = lp;
+            if (!ok) miss = true;
+            if (r == 0 && !a.sampled) { oid[0] = id; olp[0] = lp; }
+        }
+    }
+    bool any_missing = __any_sync(0xffffffffu, miss);
+    if (lane == 0) {
+        if (a.sampled) {
+            const bool ok = row_ok && GJ >= 0;
+            oid[0] = ok ? (a.map ? __ldg(a.map + GJ) : GJ) : -1;
+            olp[0] = ok ? GZ - lse : CUDART_NAN_F;
+            if (!ok) any_missing = true;
+        }
+        if (a.dbg_lse) a.dbg_lse[b] = lse;
+        if (!row_ok) atomicOr(&ctrl->flags, (uint32_t)VT_FLAG_BAD_TEMP);
+        else if (any_missing) atomicOr(&ctrl->flags, (uint32_t)VT_FLAG_NAN_ROW);
+    }
+}
+
+// NCH column chunks per row, KBC 32-column blocks per warp and chunk; TWO: hidden rows 8..15 present.
+template <int NCH, int KBC, bool TWO>
 __global__ void __launch_bounds__(kThreads, 1)
-k_head_skinny(const HeadArgs a, Ctrl* ctrl, float* __restrict__ recs, int RB, int KBW) {
-    extern __shared__ __align__(16) uint8_t s_raw[];
-    __shared__ int s_last;
-    constexpr int HALVES = TWO ? 2 : 1;
-    Smem sm;
-    sm.part = reinterpret_cast<float*>(s_raw);
-    sm.topv = sm.part + 2 * kNW * kPartStride;
-    sm.topj = reinterpret_cast<int*>(sm.topv + kMaxB * VT_MAX_TOPK);
-    sm.h = reinterpret_cast<uint4*>(sm.topj + kMaxB * VT_MAX_TOPK);
+k_head_stream(const HeadArgs a, Ctrl* ctrl, float* __restrict__ recs, const Geo geo) {
+    extern __shared__ __align__(128) uint8_t s_raw[];
+    __shared__ uint64_t s_full[kMaxStages], s_empty[kMaxStages], s_pfull[2], s_pempty[2];
+    __shared__ int s_last, s_abort;
+    constexpr int KC = kNW * KBC * 32;                   // columns per chunk
+    const int B = a.B, K = a.K, d = a.d, topk = a.topk;
+    const int S = geo.S, pitch = geo.pitch, PT = geo.part_stride;
+    const int stage_bytes = kRows * pitch;
+    uint8_t* ring = s_raw;
+    float* part = reinterpret_cast<float*>(s_raw + geo.ring_bytes);           // [2][kNW][PT]
+    float* topv = part + 2 * kNW * PT;                                        // [B][topk]
+    int* topj = reinterpret_cast<int*>(topv + B * topk);                      // [B][topk]
+    float* candv = reinterpret_cast<float*>(topj + B * topk);                 // [B][kCand]
+    int* candj = reinterpret_cast<int*>(candv + B * kCand);                   // [B][kCand]
 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int g = lane >> 2, t = lane & 3;
-    const int B = a.B, K = a.K, d = a.d, topk = a.topk;
-    const int NG = KBW / U;                              // groups of U k-blocks per warp and row block
-    const int KBpad = KBW * kNW;
-    const int rb0 = (int)((long long)RB * blockIdx.x / gridDim.x);
-    const int rb1 = (int)((long long)RB * (blockIdx.x + 1) / gridDim.x);
-    const int n_items = (rb1 - rb0) * NG;
+    const int rb0 = (int)((long long)geo.RB * blockIdx.x / gridDim.x);
+    const int rb1 = (int)((long long)geo.RB * (blockIdx.x + 1) / gridDim.x);
 
-    // ---- ring of W loads: start streaming before anything else --------------------------------
-    uint4 buf[NBUF][U];
-    int ld_rb = rb0, ld_grp = 0, ld_item = 0;
-    auto load_item = [&](uint4 (&bf)[U]) {
-        if (ld_item < n_items) {
-            const int row = min(ld_rb * 8 + g, K - 1);
-            const uint16_t* base = a.W + (size_t)row * d + 8 * t;
-#pragma unroll
-            for (int u = 0; u < U; ++u) {
-                const int kb = warp + kNW * (ld_grp * U + u);
-                bf[u] = (kb * 32 + 8 * t < d) ? ld_stream_u4(base + kb * 32) : make_uint4(0, 0, 0, 0);
-            }
-            ++ld_item;
-            if (++ld_grp == NG) { ld_grp = 0; ++ld_rb; }
-        }
-    };
-#pragma unroll
-    for (int s = 0; s < NBUF; ++s) load_item(buf[s]);
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < S; ++s) { mbar_init(&s_full[s], 1); mbar_init(&s_empty[s], kNW); }
+        for (int p = 0; p < 2; ++p) { mbar_init(&s_pfull[p], kNW); mbar_init(&s_pempty[p], B); }
+        s_abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    for (int i = threadIdx.x; i < B * topk; i += kThreads) { topv[i] = -CUDART_INF_F; topj[i] = -1; }
+    __syncthreads();
+    volatile int* abort_flag = &s_abort;
 
-    // ---- stage h as ready-made fragments, init the per-row state ---------------------------------
-    for (int i = threadIdx.x; i < KBpad * HALVES * 32; i += kThreads) {
-        const int ln = i & 31, half = (i >> 5) % HALVES, kb = (i >> 5) / HALVES;
-        const int brow = half * 8 + (ln >> 2), k0 = kb * 32 + 8 * (ln & 3);
-        uint4 v = make_uint4(0, 0, 0, 0);
-        if (brow < B && k0 < d) v = *reinterpret_cast<const uint4*>(a.h + (size_t)brow * d + k0);
-        sm.h[i] = v;
-    }
-    for (int i = threadIdx.x; i < kMaxB * VT_MAX_TOPK; i += kThreads) {
-        sm.topv[i] = -CUDART_INF_F;
-        sm.topj[i] = -1;
-    }
-    // per-row state lives in the registers of warp b (identical in its four 8-lane groups)
+    // per-row state of warp b (identical in its four 8-lane groups); declared here so that the
+    // record code after the loop sees it
     const int b = warp;
     float invT = 1.f;
     bool row_ok = true;
+    float st_m = -CUDART_INF_F, st_s = 0.f;                 // running max / sum exp (per lane)
+    float gb_s = -CUDART_INF_F, gb_z = 0.f;                 // Gumbel best (per lane)
+    int gb_j = -1;
+
+    // ---- producer duty: one bulk copy per vocabulary row of a stage (lanes 0..7 of the duty warp) ----
+    // Every warp tracks the fetch sequence; fetch f is issued by one warp of the duty group (the
+    // warps that own no hidden row, so the epilogue warps are spared), in rotation.
+    const int n_items = (rb1 - rb0) * NCH;
+    const int n_duty = (B < kNW) ? kNW - B : 1;
+    int f_item = 0, f_rb = rb0, f_c = 0, f_s = 0, f_duty = kNW - 1;   // next item to fetch, its duty warp
+    uint32_t f_ph = 0;
+    auto fetch_next = [&]() -> bool {                         // false = abort
+        bool ok = true;
+        if (warp == f_duty) {
+            if (f_item >= S && !mbar_wait(&s_empty[f_s], f_ph ^ 1, abort_flag)) ok = false;
+            if (ok) {
+                const int nrows = min(kRows, K - f_rb * kRows);
+                const int col0 = f_c * KC;
+                const uint32_t cbytes = (uint32_t)(min(d, col0 + KC) - col0) * 2u;
+                if (lane == 0) mbar_expect_tx(&s_full[f_s], cbytes * (uint32_t)nrows);
+                __syncwarp();
+                if (lane < nrows)
+                    bulk_g2s(smem_u32(ring + (size_t)f_s * stage_bytes + lane * pitch),
+                             a.W + (size_t)(f_rb * kRows + lane) * d + col0, cbytes, &s_full[f_s]);
+            }
+        }
+        ++f_item;
+        if (++f_c == NCH) { f_c = 0; ++f_rb; }
+        if (++f_s == S) { f_s = 0; f_ph ^= 1; }
+        if (--f_duty < kNW - n_duty) f_duty = kNW - 1;
+        return ok;
+    };
+    for (int i = 0; i < S && f_item < n_items; ++i) fetch_next();          // fill the ring (no waits)
+
+    // ---- h fragments of this warp's columns, straight from global memory into registers ----------
+    uint4 hl[NCH][KBC], hh[NCH][KBC];
+#pragma unroll
+    for (int c = 0; c < NCH; ++c)
+#pragma unroll
+        for (int i = 0; i < KBC; ++i) {
+            const int col = c * KC + (warp * KBC + i) * 32 + 8 * t;
+            hl[c][i] = make_uint4(0, 0, 0, 0);
+            hh[c][i] = make_uint4(0, 0, 0, 0);
+            if (col < d) {
+                if (g < B) hl[c][i] = __ldg(reinterpret_cast<const uint4*>(a.h + (size_t)g * d + col));
+                if (TWO && g + 8 < B)
+                    hh[c][i] = __ldg(reinterpret_cast<const uint4*>(a.h + (size_t)(g + 8) * d + col));
+            }
+        }
     if (b < B) {
         const float T = a.temp[b];
         row_ok = (T > 0.f) && (T < CUDART_INF_F);
         invT = row_ok ? 1.f / T : CUDART_NAN_F;
     }
-    float st_m = -CUDART_INF_F, st_s = 0.f;                 // running max / sum exp (per lane)
-    float gb_s = -CUDART_INF_F, gb_z = 0.f;                 // Gumbel best (per lane)
-    int gb_j = -1;
     float thr = -CUDART_INF_F;                              // k-th best so far (warp uniform)
-    int tk_cnt = 0;
+    int tk_cnt = 0, n_cand = 0;
     const int v8 = lane & 7, q = lane >> 3;
     float u_next = 0.5f;
     if (a.uniforms && b < B && rb0 < rb1) {
-        const int j = rb0 * 8 + v8;
+        const int j = rb0 * kRows + v8;
         if (j < K) u_next = __ldg(a.uniforms + (size_t)b * K + j);
     }
-    __syncthreads();
-
-    // ---- end of a row block: reduce the 16 partial tiles, update the row's running state ---------
-    auto finish_row_block = [&](int rb, float (&acc0)[4], float (&acc1)[4]) {
-        const int pb = (rb - rb0) & 1;
-        float* mine = sm.part + (pb * kNW + warp) * kPartStride;
+    const uint32_t lane_off = (uint32_t)(g * pitch + warp * KBC * 64 + t * 16);
+    const uint32_t ring_u32 = smem_u32(ring);
+    int s = 0, item = 0;
+    uint32_t ph = 0;
+    bool alive = true;
+#pragma unroll 1
+    for (int rb = rb0; rb < rb1 && alive; ++rb) {
+        float acc0[4] = {0.f, 0.f, 0.f, 0.f}, acc1[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int c = 0; c < NCH; ++c) {
+            if (!mbar_wait(&s_full[s], ph, abort_flag)) { alive = false; break; }
+            const uint32_t base = ring_u32 + (uint32_t)s * (uint32_t)stage_bytes + lane_off;
+            uint4 w[KBC];
+#pragma unroll
+            for (int i = 0; i < KBC; ++i) {
+                const int col = c * KC + (warp * KBC + i) * 32 + 8 * t;
+                w[i] = (col < d) ? lds_u4(base + i * 64) : make_uint4(0, 0, 0, 0);
+            }
+#pragma unroll
+            for (int i = 0; i < KBC; ++i) {
+                mma_bf16(acc0, hl[c][i].x, hh[c][i].x, hl[c][i].y, hh[c][i].y, w[i].x, w[i].y);
+                mma_bf16(acc1, hl[c][i].z, hh[c][i].z, hl[c][i].w, hh[c][i].w, w[i].z, w[i].w);
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&s_empty[s]);
+            if (++s == S) { s = 0; ph ^= 1; }
+            // refill the stage released kLag items ago (by now every warp has normally left it)
+            if (item >= kLag && f_item < n_items && !fetch_next()) { alive = false; break; }
+            ++item;
+        }
+        if (!alive) break;
+        // ---- hand the partial tile over -------------------------------------------------------------
+        const int n = rb - rb0, pb = n & 1;
+        const uint32_t use = (uint32_t)(n >> 1);
+        if (n >= 2 && !mbar_wait(&s_pempty[pb], (use - 1) & 1, abort_flag)) break;
+        float* mine = part + (pb * kNW + warp) * PT;
         *reinterpret_cast<float2*>(mine + g * 8 + 2 * t) = make_float2(acc0[0] + acc1[0], acc0[1] + acc1[1]);
         if (TWO)
             *reinterpret_cast<float2*>(mine + 64 + g * 8 + 2 * t) =
                 make_float2(acc0[2] + acc1[2], acc0[3] + acc1[3]);
-        __syncthreads();
-        if (b >= B) return;
-        const float* src = sm.part + pb * kNW * kPartStride + b * 8 + v8;
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&s_pfull[pb]);
+        if (b >= B) continue;
+        // ---- warp b: reduce the 16 tiles, update hidden row b -----------------------------------------
+        if (!mbar_wait(&s_pfull[pb], use & 1, abort_flag)) break;
+        const float* src = part + pb * kNW * PT + b * 8 + v8;
         float x = 0.f;
 #pragma unroll
-        for (int i = 0; i < 4; ++i) x += src[(q + 4 * i) * kPartStride];
+        for (int i = 0; i < 4; ++i) x += src[(q + 4 * i) * PT];
         x += __shfl_xor_sync(0xffffffffu, x, 8);
         x += __shfl_xor_sync(0xffffffffu, x, 16);
-        const int j = rb * 8 + v8;
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&s_pempty[pb]);
+        const int j = rb * kRows + v8;
         const bool valid = j < K;
         if (a.dbg_logits && valid && q == 0) a.dbg_logits[(size_t)b * K + j] = x;
         const float z = x * invT;
@@ -165,68 +490,44 @@ k_head_skinny(const HeadArgs a, Ctrl* ctrl, float* __restrict__ recs, int RB, in
             const float uc = fminf(fmaxf(u_next, 0x1p-24f), 1.f - 0x1p-24f);
             const float sc = z - logf(-logf(uc));
             if (valid && sc > gb_s) { gb_s = sc; gb_j = j; gb_z = z; }
-            const int jn = (rb + 1) * 8 + v8;
+            const int jn = (rb + 1) * kRows + v8;
             if (rb + 1 < rb1 && jn < K) u_next = __ldg(a.uniforms + (size_t)b * K + jn);
         }
-        unsigned cand = __ballot_sync(0xffffffffu, valid && q == 0 && z > thr);
-        while (cand) {
-            const int l = __ffs(cand) - 1;
-            cand &= cand - 1;
-            const float cz = __shfl_sync(0xffffffffu, z, l);
-            if (!(cz > thr)) continue;                       // thr may have risen meanwhile
-            const int cj = rb * 8 + l;
-            float* tv = sm.topv + b * VT_MAX_TOPK;
-            int* tj = sm.topj + b * VT_MAX_TOPK;
-            const int p0 = lane, p1 = lane + 32;
-            const float v0 = p0 < tk_cnt ? tv[p0] : -CUDART_INF_F;
-            const float v1 = p1 < tk_cnt ? tv[p1] : -CUDART_INF_F;
-            const int j0 = p0 < tk_cnt ? tj[p0] : -1, j1 = p1 < tk_cnt ? tj[p1] : -1;
-            const int pos = __popc(__ballot_sync(0xffffffffu, p0 < tk_cnt && v0 >= cz)) +
-                            __popc(__ballot_sync(0xffffffffu, p1 < tk_cnt && v1 >= cz));
-            const int ncnt = min(tk_cnt + 1, topk);
-            __syncwarp();
-            if (p0 >= pos && p0 < tk_cnt && p0 + 1 < ncnt) { tv[p0 + 1] = v0; tj[p0 + 1] = j0; }
-            if (p1 >= pos && p1 < tk_cnt && p1 + 1 < ncnt) { tv[p1 + 1] = v1; tj[p1 + 1] = j1; }
-            if (lane == 0) { tv[pos] = cz; tj[pos] = cj; }
-            __syncwarp();
-            tk_cnt = ncnt;
-            thr = (tk_cnt == topk) ? tv[topk - 1] : -CUDART_INF_F;
-        }
-    };
-
-    // ---- main loop ---------------------------------------------------------------------------------
-    float acc0[4] = {0.f, 0.f, 0.f, 0.f}, acc1[4] = {0.f, 0.f, 0.f, 0.f};
-    int c_rb = rb0, c_grp = 0;
-#pragma unroll 1
-    for (int it = 0; it < n_items; it += NBUF) {
-#pragma unroll
-        for (int s = 0; s < NBUF; ++s) {
-            if (it + s < n_items) {
-#pragma unroll
-                for (int u = 0; u < U; ++u) {
-                    const int kb = warp + kNW * (c_grp * U + u);
-                    const uint4 w = buf[s][u];
-                    const uint4 hlo = sm.h[(kb * HALVES) * 32 + lane];
-                    uint4 hhi = make_uint4(0, 0, 0, 0);
-                    if (TWO) hhi = sm.h[(kb * HALVES + 1) * 32 + lane];
-                    mma_bf16(acc0, hlo.x, hhi.x, hlo.y, hhi.y, w.x, w.y);
-                    mma_bf16(acc1, hlo.z, hhi.z, hlo.w, hhi.w, w.z, w.w);
-                }
-                load_item(buf[s]);
-                if (++c_grp == NG) {
-                    c_grp = 0;
-                    finish_row_block(c_rb, acc0, acc1);
-                    ++c_rb;
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) acc0[i] = acc1[i] = 0.f;
-                }
+        const bool is_cand = valid && q == 0 && z > thr;
+        const unsigned cand = __ballot_sync(0xffffffffu, is_cand);
+        if (cand) {
+            if (is_cand) {
+                const int pos = n_cand + __popc(cand & lanemask_lt());
+                candv[b * kCand + pos] = z;
+                candj[b * kCand + pos] = j;
             }
+            n_cand += __popc(cand);
+            if (n_cand + kRows > kCand) {
+                const TopkState ts = topk_flush(topv + b * topk, topj + b * topk, tk_cnt, candv + b * kCand,
+                                                candj + b * kCand, n_cand, topk);
+                tk_cnt = ts.cnt;
+                thr = ts.thr;
+                n_cand = 0;
+            }
+        }
+    }
+    if (warp == kNW - 1 && *abort_flag) {
+        // drain: every stage that was filled must have landed before the CTA may leave
+        const int back = min(f_item, S);
+        for (int i = 1; i <= back; ++i) {
+            const int it = f_item - i;
+            const unsigned long long t0 = global_ns();
+            while (!mbar_try(&s_full[it % S], (uint32_t)((it / S) & 1)) && global_ns() - t0 < kWaitLimitNs) {}
         }
     }
 
     // ---- this CTA's record per hidden row ----------------------------------------------------------
-    const int RW = rec_words(topk);
-    if (b < B) {
+    if (b < B && !*abort_flag) {
+        if (n_cand > 0) {
+            const TopkState ts = topk_flush(topv + b * topk, topj + b * topk, tk_cnt, candv + b * kCand,
+                                            candj + b * kCand, n_cand, topk);
+            tk_cnt = ts.cnt;
+        }
 #pragma unroll
         for (int o = 1; o < 8; o <<= 1) {
             const float m2 = __shfl_xor_sync(0xffffffffu, st_m, o);
@@ -237,172 +538,124 @@ k_head_skinny(const HeadArgs a, Ctrl* ctrl, float* __restrict__ recs, int RB, in
             const int gj2 = __shfl_xor_sync(0xffffffffu, gb_j, o);
             if (gj2 >= 0 && (gb_j < 0 || better(gs2, gj2, gb_s, gb_j))) { gb_s = gs2; gb_j = gj2; gb_z = gz2; }
         }
-        float* rec = recs + ((size_t)blockIdx.x * B + b) * RW;
+        int* irecs = reinterpret_cast<int*>(recs);
+        const int c = blockIdx.x;
         if (lane == 0) {
-            rec[0] = st_m; rec[1] = st_s; rec[2] = gb_s;
-            reinterpret_cast<int*>(rec)[3] = gb_j;
-            rec[4] = gb_z;
-            reinterpret_cast<int*>(rec)[5] = row_ok ? 1 : 0;
+            recs[rec_at(b, 0, topk) + c] = st_m;
+            recs[rec_at(b, 1, topk) + c] = st_s;
+            recs[rec_at(b, 2, topk) + c] = gb_s;
+            irecs[rec_at(b, 3, topk) + c] = gb_j;
+            recs[rec_at(b, 4, topk) + c] = gb_z;
         }
         for (int r = lane; r < topk; r += 32) {
-            rec[kRecHdr + r] = sm.topv[b * VT_MAX_TOPK + r];
-            reinterpret_cast<int*>(rec)[kRecHdr + topk + r] = sm.topj[b * VT_MAX_TOPK + r];
+            recs[rec_at(b, 5 + r, topk) + c] = topv[b * topk + r];
+            irecs[rec_at(b, 5 + topk + r, topk) + c] = topj[b * topk + r];
         }
     }
     __threadfence();
     __syncthreads();
-    if (threadIdx.x == 0)
+    if (threadIdx.x == 0) {
+        if (s_abort) atomicOr(&ctrl->flags, (uint32_t)VT_FLAG_TIMEOUT);
         s_last = (atomicInc(&ctrl->head_ticket, gridDim.x - 1) == gridDim.x - 1);
+    }
     __syncthreads();
     if (!s_last || b >= B) return;
     __threadfence();
 
-    // ---- last CTA: merge all records of row b in CTA order ------------------------------------------
-    const int G = gridDim.x;
-    float M = -CUDART_INF_F, S = 0.f, GS = -CUDART_INF_F, GZ = 0.f;
-    int GJ = -1;
-    for (int c = lane; c < G; c += 32) {
-        const float* rec = recs + ((size_t)c * B + b) * RW;
-        lse_merge(M, S, ld_cg_f32(rec + 0), ld_cg_f32(rec + 1));
-        const float gs2 = ld_cg_f32(rec + 2), gz2 = ld_cg_f32(rec + 4);
-        const int gj2 = ld_cg_s32(reinterpret_cast<const int*>(rec) + 3);
-        if (gj2 >= 0 && (GJ < 0 || better(gs2, gj2, GS, GJ))) { GS = gs2; GJ = gj2; GZ = gz2; }
-    }
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const float m2 = __shfl_xor_sync(0xffffffffu, M, o), s2 = __shfl_xor_sync(0xffffffffu, S, o);
-        lse_merge(M, S, m2, s2);
-        const float gs2 = __shfl_xor_sync(0xffffffffu, GS, o), gz2 = __shfl_xor_sync(0xffffffffu, GZ, o);
-        const int gj2 = __shfl_xor_sync(0xffffffffu, GJ, o);
-        if (gj2 >= 0 && (GJ < 0 || better(gs2, gj2, GS, GJ))) { GS = gs2; GJ = gj2; GZ = gz2; }
-    }
-    const float lse = M + logf(S);
-    // stage the first `depth` entries of every CTA's list in shared memory (h is no longer needed)
-    const int cap = (KBpad * HALVES * 32 * 16) / (B * 8);     // (value, index) pairs per row
-    const int depth = min(topk, cap / G);
-    float* stv = reinterpret_cast<float*>(sm.h) + (size_t)b * cap * 2;
-    int* stj = reinterpret_cast<int*>(stv) + cap;
-    for (int e = lane; e < G * depth; e += 32) {
-        const int c = e / depth, r = e - c * depth;
-        const float* rec = recs + ((size_t)c * B + b) * RW;
-        stv[e] = ld_cg_f32(rec + kRecHdr + r);
-        stj[e] = ld_cg_s32(reinterpret_cast<const int*>(rec) + kRecHdr + topk + r);
-    }
-    __syncwarp();
-    int head[kMaxOwn];
-#pragma unroll
-    for (int o = 0; o < kMaxOwn; ++o) head[o] = 0;
-    const int row_w = 1 + topk;
-    int* oid = a.out_ids + (size_t)b * row_w;
-    float* olp = a.out_logprobs + (size_t)b * row_w;
-    int first_id = -1;
-    float first_lp = CUDART_NAN_F;
-    bool any_missing = false;
-    for (int r = 0; r < topk; ++r) {
-        float lv = -CUDART_INF_F;
-        int lj = -1, lo = -1;
-#pragma unroll
-        for (int o = 0; o < kMaxOwn; ++o) {
-            const int c = lane + 32 * o;
-            if (c < G && head[o] < topk) {
-                float v;
-                int j;
-                if (head[o] < depth) { v = stv[c * depth + head[o]]; j = stj[c * depth + head[o]]; }
-                else {
-                    const float* rec = recs + ((size_t)c * B + b) * RW;
-                    v = ld_cg_f32(rec + kRecHdr + head[o]);
-                    j = ld_cg_s32(reinterpret_cast<const int*>(rec) + kRecHdr + topk + head[o]);
-                }
-                if (j >= 0 && (lj < 0 || better(v, j, lv, lj))) { lv = v; lj = j; lo = o; }
-            }
-        }
-        float wv = lv;
-        int wj = lj;
-#pragma unroll
-        for (int o = 16; o; o >>= 1) {
-            const float v2 = __shfl_xor_sync(0xffffffffu, wv, o);
-            const int j2 = __shfl_xor_sync(0xffffffffu, wj, o);
-            if (j2 >= 0 && (wj < 0 || better(v2, j2, wv, wj))) { wv = v2; wj = j2; }
-        }
-#pragma unroll
-        for (int o = 0; o < kMaxOwn; ++o)
-            if (o == lo && lj == wj && wj >= 0) ++head[o];
-        const bool ok = row_ok && wj >= 0;
-        const int id = ok ? (a.map ? __ldg(a.map + wj) : wj) : -1;
-        const float lp = ok ? wv - lse : CUDART_NAN_F;
-        if (r == 0) { first_id = id; first_lp = lp; }
-        if (!ok) any_missing = true;
-        if (lane == 0) { oid[1 + r] = id; olp[1 + r] = lp; }
-    }
-    if (lane == 0) {
-        if (a.uniforms) {
-            const bool ok = row_ok && GJ >= 0;
-            oid[0] = ok ? (a.map ? __ldg(a.map + GJ) : GJ) : -1;
-            olp[0] = ok ? GZ - lse : CUDART_NAN_F;
-            if (!ok) any_missing = true;
-        } else {
-            oid[0] = first_id;
-            olp[0] = first_lp;
-        }
-        if (a.dbg_lse) a.dbg_lse[b] = lse;
-        if (!row_ok) atomicOr(&ctrl->flags, (uint32_t)VT_FLAG_BAD_TEMP);
-        else if (any_missing) atomicOr(&ctrl->flags, (uint32_t)VT_FLAG_NAN_ROW);
-    }
+    merge_records(a.map, a.out_ids, a.out_logprobs, a.dbg_lse, topk, a.uniforms != nullptr, ctrl, recs, b, row_ok,
+                  reinterpret_cast<float*>(ring));
 }
 
-size_t skinny_smem_bytes(int KBW, bool two) {
-    return (size_t)2 * kNW * kPartStride * 4 + (size_t)kMaxB * VT_MAX_TOPK * 8 +
-           (size_t)KBW * kNW * (two ? 2 : 1) * 512;
+// ---- host side ---------------------------------------------------------------------------------------
+struct Shape {
+    int nch, kbc;      // template selection; 0 = unsupported
+};
+
+// 32-column blocks per warp needed for d, rounded up to a supported (chunks, blocks per chunk) pair
+Shape pick_shape(int d) {
+    const int nkb = (d + 31) / 32;
+    const int kbw = (nkb + kNW - 1) / kNW;
+    static const int table[17][2] = {{0, 0}, {1, 1}, {1, 2}, {1, 3}, {1, 4}, {2, 3}, {2, 3}, {2, 4}, {2, 4},
+                                     {3, 3}, {3, 4}, {3, 4}, {3, 4}, {4, 4}, {4, 4}, {4, 4}, {4, 4}};
+    if (kbw < 1 || kbw > 16) return Shape{0, 0};
+    return Shape{table[kbw][0], table[kbw][1]};
 }
 
-int skinny_kbw(int d) { return ((d + 31) / 32 + kNW - 1) / kNW; }
+bool shape_ok(int B, int d) {
+    if (B < 1 || B > kMaxB || d < 8 || (d & 7)) return false;
+    const Shape sh = pick_shape(d);
+    if (!sh.nch) return false;
+    if (B > 8 && sh.nch * sh.kbc > 8) return false;      // h fragments must fit the register file
+    return true;
+}
 
-template <int U, int NBUF, bool TWO>
-cudaError_t launch_variant(const HeadArgs& a, Ctrl* ctrl, float* recs, int grid, int RB, int KBW,
+Geo make_geo(int B, int K, int d, int topk, size_t* smem_bytes) {
+    const Shape sh = pick_shape(d);
+    Geo g{};
+    g.RB = (K + kRows - 1) / kRows;
+    const int kc_bytes = kNW * sh.kbc * 32 * 2;
+    g.pitch = kc_bytes + 64;                              // kc_bytes is a multiple of 128
+    g.part_stride = (B > 8 ? 128 : 64) + 8;
+    const size_t fixed = (size_t)2 * kNW * g.part_stride * 4 + (size_t)B * (topk + kCand) * 8;
+    const size_t stage = (size_t)kRows * g.pitch;
+    int S = (int)((kSmemLimit - fixed) / stage);
+    if (S > kMaxStages) S = kMaxStages;
+    g.S = S;
+    g.ring_bytes = (int)(S * stage);
+    *smem_bytes = g.ring_bytes + fixed;
+    const size_t merge_bytes = (size_t)B * 2 * kMergeDepth * kMaxGrid * 4;   // staging area of the merge
+    if (*smem_bytes < merge_bytes) *smem_bytes = merge_bytes;
+    return g;
+}
+
+template <int NCH, int KBC, bool TWO>
+cudaError_t launch_variant(const HeadArgs& a, Ctrl* ctrl, float* recs, int grid, const Geo& geo,
                            size_t smem, cudaStream_t s) {
     static int attr_done[64] = {0};
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev < 0 || dev >= 64 || !attr_done[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(k_head_skinny<U, NBUF, TWO>,
-                                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxDynSmem);
+        cudaError_t e = cudaFuncSetAttribute(k_head_stream<NCH, KBC, TWO>,
+                                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit);
         if (e != cudaSuccess) return e;
         if (dev >= 0 && dev < 64) attr_done[dev] = 1;
     }
-    k_head_skinny<U, NBUF, TWO><<<grid, kThreads, smem, s>>>(a, ctrl, recs, RB, KBW);
+    k_head_stream<NCH, KBC, TWO><<<grid, kThreads, smem, s>>>(a, ctrl, recs, geo);
     count_launch();
     return cudaGetLastError();
 }
 
 }  // namespace
 
-bool head_skinny_supported(int32_t B, int32_t d) {
-    if (B < 1 || B > kMaxB || d < 8 || (d & 7)) return false;
-    return skinny_smem_bytes(skinny_kbw(d), B > 8) <= kMaxDynSmem;
-}
+bool head_skinny_supported(int32_t B, int32_t d) { return shape_ok(B, d); }
 
 size_t head_skinny_scratch_bytes(int32_t B, int32_t K, int32_t topk) {
     (void)K;
-    return align_up((size_t)kMaxGrid * B * rec_words(topk) * 4, 256);
+    return align_up((size_t)kMaxGrid * B * rec_fields(topk) * 4, 256);
 }
 
 cudaError_t launch_head_skinny(const HeadArgs& a, Ctrl* ctrl, uint8_t* scratch, cudaStream_t s) {
-    const int RB = (a.K + 7) / 8;
+    if (!shape_ok(a.B, a.d)) return cudaErrorInvalidValue;
+    size_t smem = 0;
+    const Geo geo = make_geo(a.B, a.K, a.d, a.topk, &smem);
+    if (geo.S < kLag + 1) return cudaErrorInvalidValue;
     int grid = num_sms();
     if (grid > kMaxGrid) grid = kMaxGrid;
-    if (grid > RB) grid = RB;
-    const int KBW = skinny_kbw(a.d);
-    const bool two = a.B > 8;
-    const size_t smem = skinny_smem_bytes(KBW, two);
+    if (grid > geo.RB) grid = geo.RB;
     float* recs = reinterpret_cast<float*>(scratch);
-#define VT_LAUNCH(U, NBUF)                                                                       \
-    (two ? launch_variant<U, NBUF, true>(a, ctrl, recs, grid, RB, KBW, smem, s)                  \
-         : launch_variant<U, NBUF, false>(a, ctrl, recs, grid, RB, KBW, smem, s))
-    if (KBW % 4 == 0) return VT_LAUNCH(4, 3);
-    if (KBW % 3 == 0) return VT_LAUNCH(3, 4);
-    if (KBW % 2 == 0) return VT_LAUNCH(2, 6);
-    return VT_LAUNCH(1, 8);
-#undef VT_LAUNCH
+    const Shape sh = pick_shape(a.d);
+    const bool two = a.B > 8;
+#define VT_CASE(N, C)                                                                            \
+    if (sh.nch == N && sh.kbc == C)                                                              \
+        return two ? launch_variant<N, C, true>(a, ctrl, recs, grid, geo, smem, s)               \
+                   : launch_variant<N, C, false>(a, ctrl, recs, grid, geo, smem, s);
+#define VT_CASE1(N, C)                                                                           \
+    if (sh.nch == N && sh.kbc == C) return launch_variant<N, C, false>(a, ctrl, recs, grid, geo, smem, s);
+    VT_CASE(1, 1) VT_CASE(1, 2) VT_CASE(1, 3) VT_CASE(1, 4) VT_CASE(2, 3) VT_CASE(2, 4)
+    VT_CASE1(3, 3) VT_CASE1(3, 4) VT_CASE1(4, 4)
+#undef VT_CASE
+#undef VT_CASE1
+    return cudaErrorInvalidValue;
 }
 
 }  // namespace vt
