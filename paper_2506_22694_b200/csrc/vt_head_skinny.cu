@@ -41,7 +41,7 @@ constexpr int kMaxB = 16;
 constexpr int kMaxGrid = 160;                    // merge: each lane owns at most kMaxOwn CTA records
 constexpr int kMaxOwn = kMaxGrid / 32;
 constexpr size_t kSmemLimit = 227 * 1024 - 1024; // opt-in limit minus static shared memory
-constexpr int kCand = 128;                       // candidate buffer entries per hidden row
+constexpr int kCand = 64;                        // candidate buffer entries per hidden row
 constexpr int kSelPerLane = (VT_MAX_TOPK + kCand) / 32;
 constexpr int kMergeDepth = 4;                   // list entries per CTA staged on chip by the merge
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
@@ -132,6 +132,15 @@ __device__ __forceinline__ float ord2f(unsigned k) {
     return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
 }
 
+// (value, index) as one unsigned 64-bit key: larger key = better candidate (higher value, then lower
+// index).  Comparing keys needs no data-dependent branch; per-lane branches inside a warp cost far
+// more than the arithmetic they skip.
+__device__ __forceinline__ unsigned long long key64(float v, int j) {
+    return ((unsigned long long)f2ord(v) << 32) | (unsigned)(~j);
+}
+__device__ __forceinline__ float key_val(unsigned long long k) { return ord2f((unsigned)(k >> 32)); }
+__device__ __forceinline__ int key_idx(unsigned long long k) { return (int)~(unsigned)k; }
+
 struct TopkState {
     int cnt;       // entries in the list
     float thr;     // value of entry topk-1 once the list is full, else -inf
@@ -139,42 +148,54 @@ struct TopkState {
 
 // Warp-cooperative selection: the best min(topk, cnt + n_c) of a sorted list (tv/tj, cnt entries) and
 // a batch of unsorted candidates (cv/cj, n_c entries) become the new sorted list (descending value,
-// ties to the lower index).  All elements sit in registers (at most kSelPerLane per lane); every
-// round is two warp reductions.  Runs once per full candidate buffer, so rarely once `thr` is warm.
-__device__ __noinline__ TopkState topk_flush(float* tv, int* tj, int cnt, const float* cv, const int* cj, int n_c,
+// ties to the lower index).  Every element's final position is its rank -- the number of elements
+// that beat it -- so there are no sequential selection rounds: each lane keeps up to kSelPerLane
+// elements in registers while all elements stream by as broadcast shared-memory reads.  The cost
+// does not depend on topk and is small when few candidates are pending.
+template <int NS>
+__device__ __forceinline__ void rank_scatter(float* tv, int* tj, int cnt, const float* cv, const int* cj, int n_c,
                                              int topk) {
     const int lane = threadIdx.x & 31;
-    unsigned ek[kSelPerLane];
-    int ej[kSelPerLane];
-    __syncwarp();
+    const int N = cnt + n_c;
+    unsigned long long ek[NS];
+    int rk[NS];
 #pragma unroll
-    for (int i = 0; i < kSelPerLane; ++i) {
+    for (int i = 0; i < NS; ++i) {
         const int idx = lane + 32 * i;
-        ek[i] = 0u;
-        ej[i] = 0x7fffffff;
-        if (idx < cnt) { ek[i] = f2ord(tv[idx]); ej[i] = tj[idx]; }
-        else if (idx - cnt < n_c) { ek[i] = f2ord(cv[idx - cnt]); ej[i] = cj[idx - cnt]; }
+        ek[i] = 0ull;
+        rk[i] = 0;
+        if (idx < cnt) ek[i] = key64(tv[idx], tj[idx]);
+        else if (idx < N) ek[i] = key64(cv[idx - cnt], cj[idx - cnt]);
     }
-    __syncwarp();
-    const int out = min(topk, cnt + n_c);
-    unsigned kmax = 0u;
-    for (int r = 0; r < out; ++r) {
-        unsigned lk = ek[0];
-        int lj = ej[0];
+#pragma unroll 2
+    for (int e = 0; e < cnt; ++e) {
+        const unsigned long long k = key64(tv[e], tj[e]);
 #pragma unroll
-        for (int i = 1; i < kSelPerLane; ++i)
-            if (ek[i] > lk || (ek[i] == lk && ej[i] < lj)) { lk = ek[i]; lj = ej[i]; }
-        kmax = __reduce_max_sync(0xffffffffu, lk);
-        const unsigned jmin = __reduce_min_sync(0xffffffffu, lk == kmax ? (unsigned)lj : 0xffffffffu);
-        if (lk == kmax && (unsigned)lj == jmin) {
-#pragma unroll
-            for (int i = 0; i < kSelPerLane; ++i)
-                if (ek[i] == lk && ej[i] == lj) { ek[i] = 0u; ej[i] = 0x7fffffff; }
-        }
-        if (lane == 0) { tv[r] = ord2f(kmax); tj[r] = (int)jmin; }
+        for (int i = 0; i < NS; ++i) rk[i] += (k > ek[i]) ? 1 : 0;
     }
+#pragma unroll 4
+    for (int e = 0; e < n_c; ++e) {
+        const unsigned long long k = key64(cv[e], cj[e]);
+#pragma unroll
+        for (int i = 0; i < NS; ++i) rk[i] += (k > ek[i]) ? 1 : 0;
+    }
+    __syncwarp();                                         // every read of the old list is done
+#pragma unroll
+    for (int i = 0; i < NS; ++i)
+        if (lane + 32 * i < N && rk[i] < topk) { tv[rk[i]] = key_val(ek[i]); tj[rk[i]] = key_idx(ek[i]); }
+}
+
+__device__ __noinline__ TopkState topk_flush(float* tv, int* tj, int cnt, const float* cv, const int* cj, int n_c,
+                                             int topk) {
+    const int N = cnt + n_c;
     __syncwarp();
-    return TopkState{out, (out == topk) ? ord2f(kmax) : -CUDART_INF_F};
+    if (N <= 32) rank_scatter<1>(tv, tj, cnt, cv, cj, n_c, topk);
+    else if (N <= 64) rank_scatter<2>(tv, tj, cnt, cv, cj, n_c, topk);
+    else if (N <= 96) rank_scatter<3>(tv, tj, cnt, cv, cj, n_c, topk);
+    else rank_scatter<kSelPerLane>(tv, tj, cnt, cv, cj, n_c, topk);
+    __syncwarp();
+    const int out = min(topk, N);
+    return TopkState{out, (out == topk) ? tv[topk - 1] : -CUDART_INF_F};
 }
 
 // Records: one word per (hidden row b, field f, CTA c) at recs[(b * rec_fields(topk) + f) * kMaxGrid + c],
@@ -252,30 +273,29 @@ __device__ __noinline__ void merge_records(const int32_t* map, int32_t* out_ids,
     __syncwarp();
     // k rounds; every lane keeps the current head of each of its lists in registers, a round is two
     // warp reductions, and the winner alone advances (from the staged entries, else from global memory)
-    int head[kMaxOwn], cj[kMaxOwn];
-    unsigned ck[kMaxOwn];
+    int head[kMaxOwn];
+    unsigned long long ck[kMaxOwn];
 #pragma unroll
     for (int o = 0; o < kMaxOwn; ++o) {
         head[o] = 0;
         const bool live = (lane + 32 * o < G) && ej[0][o] >= 0;
-        ck[o] = live ? f2ord(ev[0][o]) : 0u;
-        cj[o] = live ? ej[0][o] : 0x7fffffff;
+        ck[o] = live ? key64(ev[0][o], ej[0][o]) : 0ull;
     }
     float res_v[2] = {0.f, 0.f};
     int res_j[2] = {-1, -1};
     for (int r = 0; r < topk; ++r) {
-        unsigned lk = ck[0];
-        int lj = cj[0];
+        unsigned long long lk = ck[0];
 #pragma unroll
-        for (int o = 1; o < kMaxOwn; ++o)
-            if (ck[o] > lk || (ck[o] == lk && cj[o] < lj)) { lk = ck[o]; lj = cj[o]; }
-        const unsigned kmax = __reduce_max_sync(0xffffffffu, lk);
-        const unsigned jmin = __reduce_min_sync(0xffffffffu, lk == kmax ? (unsigned)lj : 0xffffffffu);
+        for (int o = 1; o < kMaxOwn; ++o) lk = ck[o] > lk ? ck[o] : lk;
+        const unsigned hi = (unsigned)(lk >> 32);
+        const unsigned kmax = __reduce_max_sync(0xffffffffu, hi);
+        const unsigned lomax = __reduce_max_sync(0xffffffffu, hi == kmax ? (unsigned)lk : 0u);
         if (kmax == 0u) break;                                // every list is exhausted
-        if (lk == kmax && (unsigned)lj == jmin) {
+        const unsigned long long win = ((unsigned long long)kmax << 32) | lomax;
+        if (lk == win) {                                      // one lane: advance the list it came from
 #pragma unroll
             for (int o = 0; o < kMaxOwn; ++o)
-                if (ck[o] == lk && cj[o] == lj) {
+                if (ck[o] == win) {
                     const int c = lane + 32 * o;
                     const int hd = ++head[o];
                     float v = -CUDART_INF_F;
@@ -285,13 +305,12 @@ __device__ __noinline__ void merge_records(const int32_t* map, int32_t* out_ids,
                         v = ld_cg_f32(recs + rec_at(b, 5 + hd, topk) + c);
                         j = ld_cg_s32(irecs + rec_at(b, 5 + topk + hd, topk) + c);
                     }
-                    ck[o] = j >= 0 ? f2ord(v) : 0u;
-                    cj[o] = j >= 0 ? j : 0x7fffffff;
+                    ck[o] = j >= 0 ? key64(v, j) : 0ull;
                 }
         }
         if (lane == (r & 31)) {
-            if (r < 32) { res_v[0] = ord2f(kmax); res_j[0] = (int)jmin; }
-            else { res_v[1] = ord2f(kmax); res_j[1] = (int)jmin; }
+            if (r < 32) { res_v[0] = key_val(win); res_j[0] = key_idx(win); }
+            else { res_v[1] = key_val(win); res_j[1] = key_idx(win); }
         }
     }
     const int row_w = 1 + topk;
@@ -337,8 +356,8 @@ k_head_stream(const HeadArgs a, Ctrl* ctrl, float* __restrict__ recs, const Geo 
     const int S = geo.S, pitch = geo.pitch, PT = geo.part_stride;
     const int stage_bytes = kRows * pitch;
     uint8_t* ring = s_raw;
-    float* part = reinterpret_cast<float*>(s_raw + geo.ring_bytes);           // [2][kNW][PT]
-    float* topv = part + 2 * kNW * PT;                                        // [B][topk]
+    float* part = reinterpret_cast<float*>(s_raw + geo.ring_bytes);           // [2][kNW][R][PT]
+    float* topv = part + 2 * kNW * (TWO ? 2 : 4) * PT;                                        // [B][topk]
     int* topj = reinterpret_cast<int*>(topv + B * topk);                      // [B][topk]
     float* candv = reinterpret_cast<float*>(topj + B * topk);                 // [B][kCand]
     int* candj = reinterpret_cast<int*>(candv + B * kCand);                   // [B][kCand]
@@ -419,81 +438,106 @@ k_head_stream(const HeadArgs a, Ctrl* ctrl, float* __restrict__ recs, const Geo 
     }
     float thr = -CUDART_INF_F;                              // k-th best so far (warp uniform)
     int tk_cnt = 0, n_cand = 0;
-    const int v8 = lane & 7, q = lane >> 3;
-    float u_next = 0.5f;
-    if (a.uniforms && b < B && rb0 < rb1) {
-        const int j = rb0 * kRows + v8;
-        if (j < K) u_next = __ldg(a.uniforms + (size_t)b * K + j);
-    }
     const uint32_t lane_off = (uint32_t)(g * pitch + warp * KBC * 64 + t * 16);
     const uint32_t ring_u32 = smem_u32(ring);
-    int s = 0, item = 0;
+    // epilogue lane roles: a group of R row blocks has 8R logits per hidden row; LPR lanes share one
+    // logit, each summing the partial tiles of kNW / LPR warps
+    constexpr int R = TWO ? 2 : 4;                          // row blocks per exchange
+    constexpr int LPR = 4 / R;
+    const int e_ri = lane % (8 * R), e_q = lane / (8 * R);
+    const int e_r = e_ri >> 3, e_v8 = e_ri & 7;
+    float u_next = 0.5f;
+    if (a.uniforms && b < B && rb0 + e_r < rb1) {
+        const int j = (rb0 + e_r) * kRows + e_v8;
+        if (j < K) u_next = __ldg(a.uniforms + (size_t)b * K + j);
+    }
+    int s = 0, item = 0, n = 0;
     uint32_t ph = 0;
     bool alive = true;
 #pragma unroll 1
-    for (int rb = rb0; rb < rb1 && alive; ++rb) {
-        float acc0[4] = {0.f, 0.f, 0.f, 0.f}, acc1[4] = {0.f, 0.f, 0.f, 0.f};
+    for (int rb = rb0; rb < rb1 && alive; rb += R, ++n) {
+        const int rc = min(R, rb1 - rb);
+        float res[R][TWO ? 4 : 2];
 #pragma unroll
-        for (int c = 0; c < NCH; ++c) {
-            if (!mbar_wait(&s_full[s], ph, abort_flag)) { alive = false; break; }
-            const uint32_t base = ring_u32 + (uint32_t)s * (uint32_t)stage_bytes + lane_off;
-            uint4 w[KBC];
+        for (int r = 0; r < R; ++r) {
+            if (r < rc && alive) {
+                float acc0[4] = {0.f, 0.f, 0.f, 0.f}, acc1[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-            for (int i = 0; i < KBC; ++i) {
-                const int col = c * KC + (warp * KBC + i) * 32 + 8 * t;
-                w[i] = (col < d) ? lds_u4(base + i * 64) : make_uint4(0, 0, 0, 0);
+                for (int c = 0; c < NCH; ++c) {
+                    if (!alive || !mbar_wait(&s_full[s], ph, abort_flag)) { alive = false; continue; }
+                    const uint32_t base = ring_u32 + (uint32_t)s * (uint32_t)stage_bytes + lane_off;
+                    uint4 w[KBC];
+#pragma unroll
+                    for (int i = 0; i < KBC; ++i) {
+                        const int col = c * KC + (warp * KBC + i) * 32 + 8 * t;
+                        w[i] = (col < d) ? lds_u4(base + i * 64) : make_uint4(0, 0, 0, 0);
+                    }
+#pragma unroll
+                    for (int i = 0; i < KBC; ++i) {
+                        mma_bf16(acc0, hl[c][i].x, hh[c][i].x, hl[c][i].y, hh[c][i].y, w[i].x, w[i].y);
+                        mma_bf16(acc1, hl[c][i].z, hh[c][i].z, hl[c][i].w, hh[c][i].w, w[i].z, w[i].w);
+                    }
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&s_empty[s]);
+                    if (++s == S) { s = 0; ph ^= 1; }
+                    // refill the stage released kLag items ago (by now every warp has normally left it)
+                    if (item >= kLag && f_item < n_items && !fetch_next()) alive = false;
+                    ++item;
+                }
+                res[r][0] = acc0[0] + acc1[0];
+                res[r][1] = acc0[1] + acc1[1];
+                if (TWO) { res[r][2] = acc0[2] + acc1[2]; res[r][3] = acc0[3] + acc1[3]; }
             }
-#pragma unroll
-            for (int i = 0; i < KBC; ++i) {
-                mma_bf16(acc0, hl[c][i].x, hh[c][i].x, hl[c][i].y, hh[c][i].y, w[i].x, w[i].y);
-                mma_bf16(acc1, hl[c][i].z, hh[c][i].z, hl[c][i].w, hh[c][i].w, w[i].z, w[i].w);
-            }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&s_empty[s]);
-            if (++s == S) { s = 0; ph ^= 1; }
-            // refill the stage released kLag items ago (by now every warp has normally left it)
-            if (item >= kLag && f_item < n_items && !fetch_next()) { alive = false; break; }
-            ++item;
         }
         if (!alive) break;
-        // ---- hand the partial tile over -------------------------------------------------------------
-        const int n = rb - rb0, pb = n & 1;
+        // ---- hand the partial tiles over ------------------------------------------------------------
+        const int pb = n & 1;
         const uint32_t use = (uint32_t)(n >> 1);
         if (n >= 2 && !mbar_wait(&s_pempty[pb], (use - 1) & 1, abort_flag)) break;
-        float* mine = part + (pb * kNW + warp) * PT;
-        *reinterpret_cast<float2*>(mine + g * 8 + 2 * t) = make_float2(acc0[0] + acc1[0], acc0[1] + acc1[1]);
-        if (TWO)
-            *reinterpret_cast<float2*>(mine + 64 + g * 8 + 2 * t) =
-                make_float2(acc0[2] + acc1[2], acc0[3] + acc1[3]);
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+            if (r < rc) {
+                float* mine = part + ((pb * kNW + warp) * R + r) * PT;
+                if (g < B) *reinterpret_cast<float2*>(mine + g * 8 + 2 * t) = make_float2(res[r][0], res[r][1]);
+                if (TWO && g + 8 < B)
+                    *reinterpret_cast<float2*>(mine + (g + 8) * 8 + 2 * t) = make_float2(res[r][2], res[r][3]);
+            }
+        }
         __syncwarp();
         if (lane == 0) mbar_arrive(&s_pfull[pb]);
         if (b >= B) continue;
-        // ---- warp b: reduce the 16 tiles, update hidden row b -----------------------------------------
+        // ---- warp b: reduce the tiles, update hidden row b --------------------------------------------
         if (!mbar_wait(&s_pfull[pb], use & 1, abort_flag)) break;
-        const float* src = part + pb * kNW * PT + b * 8 + v8;
+        const bool in_group = e_r < rc;
         float x = 0.f;
+        if (in_group) {
+            const float* src = part + ((pb * kNW + e_q) * R + e_r) * PT + b * 8 + e_v8;
 #pragma unroll
-        for (int i = 0; i < 4; ++i) x += src[(q + 4 * i) * PT];
-        x += __shfl_xor_sync(0xffffffffu, x, 8);
-        x += __shfl_xor_sync(0xffffffffu, x, 16);
+            for (int i = 0; i < kNW / LPR; ++i) x += src[i * LPR * R * PT];
+        }
+        if (LPR >= 2) x += __shfl_xor_sync(0xffffffffu, x, 8 * R);
+        if (LPR >= 4) x += __shfl_xor_sync(0xffffffffu, x, 16 * R);
         __syncwarp();
         if (lane == 0) mbar_arrive(&s_pempty[pb]);
-        const int j = rb * kRows + v8;
-        const bool valid = j < K;
-        if (a.dbg_logits && valid && q == 0) a.dbg_logits[(size_t)b * K + j] = x;
+        const int j = (rb + e_r) * kRows + e_v8;
+        const bool valid = in_group && j < K;
+        if (a.dbg_logits && valid && e_q == 0) a.dbg_logits[(size_t)b * K + j] = x;
         const float z = x * invT;
-        if (valid) {
-            if (z > st_m) { st_s = st_s * __expf(st_m - z) + 1.f; st_m = z; }
-            else st_s += __expf(z - st_m);
+        {   // online max / sum-exp without a per-lane branch
+            const float zz = valid ? z : -CUDART_INF_F;
+            const float m_new = fmaxf(st_m, zz);
+            const float m_ref = (m_new == -CUDART_INF_F) ? 0.f : m_new;
+            st_s = st_s * __expf(st_m - m_ref) + __expf(zz - m_ref);
+            st_m = m_new;
         }
         if (a.uniforms) {
             const float uc = fminf(fmaxf(u_next, 0x1p-24f), 1.f - 0x1p-24f);
             const float sc = z - logf(-logf(uc));
             if (valid && sc > gb_s) { gb_s = sc; gb_j = j; gb_z = z; }
-            const int jn = (rb + 1) * kRows + v8;
-            if (rb + 1 < rb1 && jn < K) u_next = __ldg(a.uniforms + (size_t)b * K + jn);
+            const int jn = (rb + R + e_r) * kRows + e_v8;
+            if (rb + R + e_r < rb1 && jn < K) u_next = __ldg(a.uniforms + (size_t)b * K + jn);
         }
-        const bool is_cand = valid && q == 0 && z > thr;
+        const bool is_cand = valid && e_q == 0 && z > thr;
         const unsigned cand = __ballot_sync(0xffffffffu, is_cand);
         if (cand) {
             if (is_cand) {
@@ -502,7 +546,7 @@ k_head_stream(const HeadArgs a, Ctrl* ctrl, float* __restrict__ recs, const Geo 
                 candj[b * kCand + pos] = j;
             }
             n_cand += __popc(cand);
-            if (n_cand + kRows > kCand) {
+            if (n_cand + kRows * R > kCand) {
                 const TopkState ts = topk_flush(topv + b * topk, topj + b * topk, tk_cnt, candv + b * kCand,
                                                 candj + b * kCand, n_cand, topk);
                 tk_cnt = ts.cnt;
@@ -528,8 +572,9 @@ k_head_stream(const HeadArgs a, Ctrl* ctrl, float* __restrict__ recs, const Geo 
                                             candj + b * kCand, n_cand, topk);
             tk_cnt = ts.cnt;
         }
+        // lanes sharing a logit hold identical state: fold the 8R distinct lanes only
 #pragma unroll
-        for (int o = 1; o < 8; o <<= 1) {
+        for (int o = 1; o < 8 * (TWO ? 2 : 4); o <<= 1) {
             const float m2 = __shfl_xor_sync(0xffffffffu, st_m, o);
             const float s2 = __shfl_xor_sync(0xffffffffu, st_s, o);
             lse_merge(st_m, st_s, m2, s2);
@@ -595,8 +640,9 @@ Geo make_geo(int B, int K, int d, int topk, size_t* smem_bytes) {
     g.RB = (K + kRows - 1) / kRows;
     const int kc_bytes = kNW * sh.kbc * 32 * 2;
     g.pitch = kc_bytes + 64;                              // kc_bytes is a multiple of 128
-    g.part_stride = (B > 8 ? 128 : 64) + 8;
-    const size_t fixed = (size_t)2 * kNW * g.part_stride * 4 + (size_t)B * (topk + kCand) * 8;
+    g.part_stride = ((B * 8 - 8 + 31) / 32) * 32 + 8;     // >= 8 B floats and = 8 (mod 32): conflict-free reduce
+    const int R = B > 8 ? 2 : 4;
+    const size_t fixed = (size_t)2 * kNW * R * g.part_stride * 4 + (size_t)B * (topk + kCand) * 8;
     const size_t stage = (size_t)kRows * g.pitch;
     int S = (int)((kSmemLimit - fixed) / stage);
     if (S > kMaxStages) S = kMaxStages;
