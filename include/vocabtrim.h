@@ -111,6 +111,27 @@ vt_status vt_histogram(const int32_t *ids, int64_t n, int32_t V, uint32_t *count
 vt_status vt_select_topk(const uint32_t *counts, int32_t V, int32_t K, int32_t *map,
                          int32_t *inv_map, void *ws, size_t ws_bytes, void *stream);
 
+/*
+ * vt_select_topk without a workspace.  (The paper has no counterpart: this entry point exists for
+ * the sake of callers, not of the method.)  Same result as vt_select_topk, for callers that cannot
+ * allocate device memory or pass scratch along: code living inside another runtime's memory pool,
+ * processes whose device memory is fully committed at start-up, call sites where the CUDA
+ * allocator must not be entered.  The scratch is a fixed array inside the library image:
+ * 16 * VT_STATIC_SELECT_MAX_V bytes (2 MiB) held on every GPU that loads the library until the
+ * process exits.  No CUDA allocation or free is made by this call, now or later.
+ *   - V > VT_STATIC_SELECT_MAX_V returns VT_ERR_UNSUPPORTED; other argument rules as vt_select_topk.
+ *   - The first call on each device looks up the array's device address (one synchronous runtime
+ *     query, cached afterwards): make that first call outside any stream capture.
+ *   - All calls on a device share the one array and it keeps whatever the last call left in it.
+ *     Nothing in it needs clearing between calls (every word is written before it is read), but
+ *     two calls whose kernels overlap on the GPU -- different streams, no ordering between them --
+ *     race on it and both results are undefined.  Order them on one stream or with events.
+ *   - A CUDA failure returns VT_ERR_CUDA (vt_last_cuda_error does not cover this entry point).
+ */
+#define VT_STATIC_SELECT_MAX_V 131072
+vt_status vt_select_topk_static(const uint32_t *counts, int32_t V, int32_t K, int32_t *map,
+                                int32_t *inv_map, void *stream);
+
 /* Algorithm 1 followed by Eq. 1, first line: vt_histogram then vt_select_topk (the counts live
  * in the workspace). */
 vt_status vt_build_vocab(const int32_t *ids, int64_t n, int32_t V, int32_t K, int32_t *map,

@@ -31,7 +31,7 @@ EXPORTS = (
     "vt_workspace_bytes", "vt_workspace_init", "vt_read_status", "vt_status_str", "vt_launch_count",
     "vt_last_cuda_error",
     "vt_histogram", "vt_select_topk", "vt_build_vocab", "vt_build_vocab_host", "vt_trim_head",
-    "vt_draft_head", "vt_draft_head_debug", "vt_draft_head_host",
+    "vt_draft_head", "vt_draft_head_debug", "vt_draft_head_host", "vt_select_topk_static",
 )
 
 
@@ -63,6 +63,7 @@ def lib() -> ctypes.CDLL:
         L.vt_last_cuda_error.restype = c_char_p
         L.vt_histogram.argtypes = [c_void_p, c_int64, c_int32, c_void_p, c_int, c_void_p, c_size_t, c_void_p]
         L.vt_select_topk.argtypes = [c_void_p, c_int32, c_int32, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
+        L.vt_select_topk_static.argtypes = [c_void_p, c_int32, c_int32, c_void_p, c_void_p, c_void_p]
         L.vt_build_vocab.argtypes = [c_void_p, c_int64, c_int32, c_int32, c_void_p, c_void_p, c_void_p,
                                      c_size_t, c_void_p]
         L.vt_build_vocab_host.argtypes = L.vt_build_vocab.argtypes
@@ -158,6 +159,20 @@ def vt_select_topk(counts: torch.Tensor, K: int, ws: Workspace | None = None):
     ws = _ws(ws, workspace_bytes(VT_OP_SELECT_TOPK, 0, V, K), counts)
     _check("vt_select_topk", lib().vt_select_topk(_ptr(counts), V, K, _ptr(map_), _ptr(inv), c_void_p(ws.ptr),
                                                   ws.nbytes, _stream()))
+    return map_, inv
+
+
+def vt_select_topk_static(counts: torch.Tensor, K: int, out=None):
+    """vt_select_topk for callers that may not allocate: the scratch is a fixed array inside the
+    library (vocabularies up to VT_STATIC_SELECT_MAX_V ids).  Pass `out` = (map [K], inv_map [V])
+    to keep this wrapper allocation-free as well; calls on different streams must not overlap."""
+    _dev(counts, torch.int32, "counts")
+    V = counts.numel()
+    if out is None:
+        out = (torch.empty(K, dtype=torch.int32, device=counts.device),
+               torch.empty(V, dtype=torch.int32, device=counts.device))
+    map_, inv = out
+    _check("vt_select_topk_static", lib().vt_select_topk_static(_ptr(counts), V, K, _ptr(map_), _ptr(inv), _stream()))
     return map_, inv
 
 
