@@ -45,7 +45,7 @@ FALLBACK_HBM_GBS = 6650.0
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the head kernel on the headline
 # workload, from the ncu capture summarised under profiles/ (None until a capture exists).
-NCU_TRAFFIC_BYTES = {"k_head_skinny": None, "k_hist_hot": None}
+NCU_TRAFFIC_BYTES = {"k_head_stream": None, "k_hist_hot": None}
 
 
 def measured_peaks():
@@ -340,6 +340,33 @@ def extras(vt, dev, peak_gbs):
     return out
 
 
+def small_case(vt, dev, args, peak_gbs):
+    """Short single-kernel runs sized for profiler captures (inputs larger than L2, a few launches)."""
+    if args.case == "hist":
+        n = args.hist_n
+        ids = vt_inputs.zipf_ids(n, V, 1.07, seed=1005, noise_frac=0.05, device=dev)
+        ws = vt.Workspace(vt.workspace_bytes(vt.VT_OP_BUILD_VOCAB, n, V, 32768), dev)
+        counts = torch.empty(V, dtype=torch.int32, device=dev)
+        for _ in range(args.warmup):
+            vt.vt_histogram(ids, V, counts=counts, ws=ws)
+        torch.cuda.synchronize()
+        e0, e1 = _events()
+        e0.record()
+        for _ in range(args.steps):
+            vt.vt_histogram(ids, V, counts=counts, ws=ws)
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / args.steps
+        print(json.dumps({"case": "hist", "n": n, "ms": ms, "gtok_s": n / ms / 1e6, "gbs": 4.0 * n / ms / 1e6,
+                          "frac_of_measured": 4.0 * n / ms / 1e6 / peak_gbs}), flush=True)
+    else:
+        wl = build_head_workload(vt, dev, TREE["d"], 32768, TREE["B"], TREE["topk"], TREE["temp"], True, seed=1003)
+        ms = time_head(vt, wl, args.steps, args.warmup)
+        gbs = wl["algo_bytes"] / (ms * 1e-3) / 1e9
+        print(json.dumps({"case": "tree", "K": 32768, "us": ms * 1e3, "gbs": gbs,
+                          "frac_of_measured": gbs / peak_gbs}), flush=True)
+
+
 # --------------------------------------------------------------------------------------------------
 def main():
     ap = argparse.ArgumentParser()
@@ -349,6 +376,10 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-extras", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--case", default="head", choices=["head", "hist", "tree"],
+                    help="head: the full bench line (default); hist / tree: a short run of the vocabulary "
+                         "histogram (--hist-n ids) or of the tree-drafting head, for profiler captures")
+    ap.add_argument("--hist-n", type=int, default=200_000_000)
     args = ap.parse_args()
     args.warmup = max(3, args.warmup)
     rank = int(os.environ.get("RANK", "0"))
@@ -374,6 +405,9 @@ def main():
 
     peaks, peak_kind = measured_peaks()
     peak_gbs = float(peaks["hbm_gbs"])
+    if args.case != "head":
+        small_case(vt, dev, args, peak_gbs)
+        return
     wl = build_head_workload(vt, dev, HEAD["d"], HEAD["K"], HEAD["B"], HEAD["topk"], HEAD["temp"], False,
                              seed=1002)
     run_head_steps(vt, wl, args.warmup)
@@ -413,10 +447,10 @@ def main():
         "e2e": {"value": e2e_ms * 1e3, "unit": "us", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
         "gpu_launches": int(launches), "clocks": clk.summary(),
         "hbm_gbs": gbs, "hbm_gbs_aggregate": gbs * world,
-        "roofline": {"kernel": "k_head_skinny", "bound": "hbm", "achieved": gbs, "peak": peak_gbs, "unit": "GB/s",
+        "roofline": {"kernel": "k_head_stream", "bound": "hbm", "achieved": gbs, "peak": peak_gbs, "unit": "GB/s",
                      "frac": gbs / peak_gbs, "frac_of_8000": gbs / 8000.0, "peak_source": peak_kind,
                      "algorithmic_bytes_per_launch": wl["algo_bytes"],
-                     "traffic": NCU_TRAFFIC_BYTES["k_head_skinny"]},
+                     "traffic": NCU_TRAFFIC_BYTES["k_head_stream"]},
     }
     if rank == 0 and world == 1:
         if not args.no_cpu_baseline:
