@@ -135,11 +135,13 @@ __device__ uint32_t block_excl_scan(uint32_t x, uint32_t* s_warp /*[33]*/, uint3
 // hot = sampled count >= tau, plus (in id order) as many bins with count == tau-1 as still fit.
 __global__ void __launch_bounds__(kThreads, 1)
 k_hist_pick(const uint32_t* __restrict__ sample, int32_t V, int32_t H, uint2* __restrict__ table) {
+    extern __shared__ __align__(16) uint8_t s_dyn[];
     __shared__ uint32_t s_hist[kPickBins];
     __shared__ uint32_t s_warp[33];
+    __shared__ uint32_t s_definite;
     const int T32 = (V + 31) >> 5;
-    const int wpt = (T32 + kThreads - 1) / kThreads;
-    const int w_lo = min(T32, (int)threadIdx.x * wpt), w_hi = min(T32, w_lo + wpt);
+    uint2* s_tbl = reinterpret_cast<uint2*>(s_dyn);         // [T32] {definite, tie}, then {bits, slot base}
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     s_hist[threadIdx.x] = 0;
     __syncthreads();
     {   // most bins were sampled a handful of times: count those in registers, one atomic per warp
@@ -157,7 +159,7 @@ k_hist_pick(const uint32_t* __restrict__ sample, int32_t V, int32_t H, uint2* __
         for (int k = 0; k < 8; ++k) {
             uint32_t x = small[k];
             for (int o = 16; o; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
-            if ((threadIdx.x & 31) == 0 && x) atomicAdd(&s_hist[k], x);
+            if (lane == 0 && x) atomicAdd(&s_hist[k], x);
         }
     }
     __syncthreads();
@@ -167,31 +169,28 @@ k_hist_pick(const uint32_t* __restrict__ sample, int32_t V, int32_t H, uint2* __
     const uint32_t P = block_excl_scan(mine, s_warp, &tot) + mine;
     const int n_ok = __syncthreads_count(P <= (uint32_t)H);
     const uint32_t tau = kPickBins - n_ok;
-    __shared__ uint32_t s_definite;
     if (n_ok == 0 && threadIdx.x == 0) s_definite = 0;
     if (n_ok > 0 && (int)threadIdx.x == n_ok - 1) s_definite = P;
     __syncthreads();
     const uint32_t quota = (uint32_t)H - s_definite;
-    // pass A: membership words for "definite" and "tie" bins
-    uint32_t tsum = 0;
-    for (int w = w_lo; w < w_hi; ++w) {
-        uint32_t def = 0, tie = 0;
-        for (int b = 0; b < 32; ++b) {
-            const int v = w * 32 + b;
-            if (v < V) {
-                const uint32_t c = min(sample[v], (uint32_t)(kPickBins - 1));
-                if (c >= tau) def |= 1u << b;
-                else if (c + 1 == tau) tie |= 1u << b;
-            }
-        }
-        table[w] = make_uint2(def, tie);
-        tsum += __popc(tie);
+    // pass A: one coalesced load per 32 ids, the membership words come out of warp ballots
+    for (int w = warp; w < T32; w += kThreads / 32) {
+        const int v = w * 32 + lane;
+        const uint32_t c = v < V ? min(sample[v], (uint32_t)(kPickBins - 1)) : 0u;
+        const uint32_t def = __ballot_sync(0xffffffffu, v < V && c >= tau);
+        const uint32_t tie = __ballot_sync(0xffffffffu, v < V && c + 1 == tau);
+        if (lane == 0) s_tbl[w] = make_uint2(def, tie);
     }
+    __syncthreads();
+    // pass B: admit ties in id order while the quota lasts; every thread owns wpt consecutive words
+    const int wpt = (T32 + kThreads - 1) / kThreads;
+    const int w_lo = min(T32, (int)threadIdx.x * wpt), w_hi = min(T32, w_lo + wpt);
+    uint32_t tsum = 0;
+    for (int w = w_lo; w < w_hi; ++w) tsum += __popc(s_tbl[w].y);
     uint32_t tbase = block_excl_scan(tsum, s_warp, &tot);
-    // pass B: admit ties in id order while the quota lasts
     uint32_t hsum = 0;
     for (int w = w_lo; w < w_hi; ++w) {
-        const uint2 e = table[w];
+        const uint2 e = s_tbl[w];
         uint32_t tie = e.y, keep = 0;
         const uint32_t room = tbase < quota ? quota - tbase : 0u;
         const int admit = (int)min(room, (uint32_t)__popc(tie));
@@ -202,14 +201,16 @@ k_hist_pick(const uint32_t* __restrict__ sample, int32_t V, int32_t H, uint2* __
             tie ^= low;
         }
         const uint32_t bits = e.x | keep;
-        table[w].x = bits;
+        s_tbl[w].x = bits;
         hsum += __popc(bits);
     }
     uint32_t hbase = block_excl_scan(hsum, s_warp, &tot);
     for (int w = w_lo; w < w_hi; ++w) {
-        table[w].y = hbase;
-        hbase += __popc(table[w].x);
+        s_tbl[w].y = hbase;
+        hbase += __popc(s_tbl[w].x);
     }
+    __syncthreads();
+    for (int w = threadIdx.x; w < T32; w += kThreads) table[w] = s_tbl[w];
 }
 
 // ---- main pass: hot bins in shared memory, cold bins through L2 ----------------------------------
@@ -295,15 +296,17 @@ cudaError_t launch_histogram(const int32_t* ids, int64_t n, int32_t V, uint32_t*
     uint2* table = reinterpret_cast<uint2*>(scratch + p.off_table);
     e = cudaMemsetAsync(sample, 0, (size_t)V * 4, s);
     if (e != cudaSuccess) return e;
-    k_hist_sample<<<grid, kThreads, 0, s>>>(ids, n, V, sample);
-    k_hist_pick<<<1, kThreads, 0, s>>>(sample, V, H, table);
     static bool attr_done_hot = false;
     if (!attr_done_hot) {
+        e = cudaFuncSetAttribute(k_hist_pick, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(kDynSmem / 2));
+        if (e != cudaSuccess) return e;
         e = cudaFuncSetAttribute(k_hist_hot, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  (int)kDynSmem);
         if (e != cudaSuccess) return e;
         attr_done_hot = true;
     }
+    k_hist_sample<<<grid, kThreads, 0, s>>>(ids, n, V, sample);
+    k_hist_pick<<<1, kThreads, T32 * 8, s>>>(sample, V, H, table);
     k_hist_hot<<<grid, kThreads, kDynSmem, s>>>(ids, n, V, counts, table, H, ctrl);
     count_launch(3);
     return cudaGetLastError();
