@@ -165,7 +165,9 @@ vt_status vt_trim_head(const uint16_t *W_full, const int32_t *map, uint16_t *W_t
  *                                   columns 1.. = candidates in descending z, ties to lower index
  *   out_logprobs [B, 1+topk] fp32 : log softmax(logits/T_b) of the id in the same column
  * Uniforms are clamped to [2^-24, 1-2^-24].  Limits: d % 8 == 0, 1 <= topk <= min(K, 64),
- * 1 <= B <= 256, and d <= 8192 (B <= 8) or d <= 4096 (B <= 16) on the streaming path.
+ * 1 <= B <= 256.  B <= 16 with d <= 8192 (B <= 8) or d <= 4096 runs the streaming kernel; every
+ * other shape runs the dense tensor-core kernel, which keeps its top-k lists in registers and
+ * takes topk <= 16 (VT_ERR_UNSUPPORTED beyond).
  */
 vt_status vt_draft_head(const uint16_t *h, const uint16_t *W_trim, const int32_t *map, int32_t B,
                         int32_t K, int32_t d, const float *temp, int32_t topk,

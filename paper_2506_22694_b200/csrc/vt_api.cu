@@ -42,7 +42,7 @@ bool hist_shape_ok(int32_t V) {
 bool head_shape_ok(int32_t B, int32_t K, int32_t d, int32_t topk) {
     if (B < 1 || B > 256 || K < 1 || d < 8 || (d & 7) || topk < 1 || topk > VT_MAX_TOPK || topk > K)
         return false;
-    return head_skinny_supported(B, d) || head_dense_supported(B, K, d);
+    return head_skinny_supported(B, d) || (head_dense_supported(B, K, d) && head_dense_topk_ok(topk));
 }
 
 size_t head_scratch(int32_t B, int32_t K, int32_t d, int32_t topk) {

@@ -61,6 +61,7 @@ size_t head_skinny_scratch_bytes(int32_t B, int32_t K, int32_t topk);
 cudaError_t launch_head_skinny(const HeadArgs& a, Ctrl* ctrl, uint8_t* scratch, cudaStream_t s);
 
 bool head_dense_supported(int32_t B, int32_t K, int32_t d);
+bool head_dense_topk_ok(int32_t topk);
 size_t head_dense_scratch_bytes(int32_t B, int32_t K, int32_t topk);
 cudaError_t launch_head_dense(const HeadArgs& a, Ctrl* ctrl, uint8_t* scratch, cudaStream_t s);
 

@@ -170,3 +170,68 @@ def test_config3_tree_drafting_sweep(K):
         slack += check_head(ref, gi, gl, T, m, lg, lse)
     assert slack <= 0.02 * depths * B * (1 + topk)
     assert ws.read_status() == (0, 0, 0)
+
+
+# ---- dense tensor-core path (more than 16 hidden rows, or shapes the streaming kernel does not take) ----
+@pytest.mark.parametrize("B,K,d,topk,sample", [
+    (17, 300, 72, 5, True), (40, 1000, 256, 8, True), (64, 128, 64, 1, False), (130, 515, 200, 16, True),
+    (256, 2048, 512, 8, True), (128, 4099, 1024, 4, True), (12, 700, 4104, 6, True), (200, 9, 8, 9, True),
+])
+def test_dense_path_small_shapes_and_ragged_tails(B, K, d, topk, sample):
+    W = vt_inputs.gaussian_bf16((K, d), 0.02, seed=K + d, device=DEV)
+    h = vt_inputs.gaussian_bf16((B, d), 1.0, seed=B + 17, device=DEV)
+    T = vt_inputs.temperatures(B, 0.5, 1.5, seed=K, device=DEV)
+    u = vt_inputs.uniforms((B, K), seed=d + 1, device=DEV) if sample else None
+    m = torch.randperm(K * 3, device=DEV)[:K].to(torch.int32)
+    ws = vt.Workspace(vt.workspace_bytes(vt.VT_OP_DRAFT_HEAD, 0, 0, K, d, B, topk))
+    gi, gl, lg, lse = _run(h, W, m, T, topk, u, ws=ws)
+    ref = oracle_head(h, W, m, T, topk, u)
+    check_head(ref, gi, gl, T, m, lg, lse, sampled=sample)
+    assert ws.read_status() == (0, 0, 0)
+    # the timed entry point (no logits written) must give the same ids, twice in a row
+    a = _run(h, W, m, T, topk, u, debug=False, ws=ws)
+    b = _run(h, W, m, T, topk, u, debug=False, ws=ws)
+    assert torch.equal(a[0], gi) and torch.equal(b[0], gi) and torch.equal(a[1], b[1])
+
+
+def test_dense_path_rejects_long_candidate_lists():
+    W = vt_inputs.gaussian_bf16((256, 64), 0.02, seed=1, device=DEV)
+    h = vt_inputs.gaussian_bf16((32, 64), 1.0, seed=2, device=DEV)
+    assert vt.workspace_bytes(vt.VT_OP_DRAFT_HEAD, 0, 0, 256, 64, 32, 17) == 0
+    with pytest.raises((vt.VocabTrimError, ValueError)):
+        vt.vt_draft_head(h, W, None, torch.ones(32, device=DEV), 17, None)
+
+
+def test_config4_batched_serving_dense_head():
+    """64 sequences x 4 tree nodes = 256 rows, d=4096, V=128256, K=32768, per-row T in [0.5,1.5],
+    top-8, Gumbel sampling.  The oracle checks every row on a 4096-row slice of the trimmed head
+    (all logits) and a sample of rows on the full K (ids, log-probs)."""
+    d, K, B, topk = 4096, 32768, 256, 8
+    m, _ = _vocab_map(V3, K, seed=1104)
+    W = vt_inputs.gaussian_bf16((V3, d), 0.02, seed=1004, device=DEV)
+    Wt = vt.vt_trim_head(W, m)
+    del W
+    h = vt_inputs.gaussian_bf16((B, d), 1.0, seed=5000, device=DEV)
+    T = vt_inputs.temperatures(B, 0.5, 1.5, seed=5001, device=DEV)
+    u = vt_inputs.uniforms((B, K), seed=5002, device=DEV)
+    ws = vt.Workspace(vt.workspace_bytes(vt.VT_OP_DRAFT_HEAD, 0, 0, K, d, B, topk))
+    # slice: all 256 rows against the first 4096 vocabulary rows, logits included
+    Ks = 4096
+    us = u[:, :Ks].contiguous()
+    gi, gl, lg, lse = _run(h, Wt[:Ks], m[:Ks], T, topk, us, ws=ws)
+    ref = oracle_head(h, Wt[:Ks], m[:Ks], T, topk, us)
+    slack = check_head(ref, gi, gl, T, m[:Ks], lg, lse)
+    assert slack <= 0.02 * B * (1 + topk)
+    # full size, launch configuration of the benchmark: sampled rows against the oracle
+    gi, gl = _run(h, Wt, m, T, topk, u, debug=False, ws=ws)
+    rows = [0, 1, 31, 32, 127, 128, 200, 255]
+    ref = oracle_head(h[rows], Wt, m, T[rows], topk, u[rows])
+    check_head(ref, gi[rows], gl[rows], T[rows], m)
+    # every row: ids are members of the map, candidates distinct and ordered by log-prob
+    mm = set(m.cpu().numpy().tolist())
+    ids, lps = gi.cpu().numpy(), gl.cpu().numpy()
+    for b in range(B):
+        assert all(int(x) in mm for x in ids[b])
+        assert len(set(ids[b, 1:].tolist())) == topk
+        assert np.all(np.diff(lps[b, 1:]) <= 1e-6)
+    assert ws.read_status() == (0, 0, 0)
