@@ -290,6 +290,7 @@ def extras(vt, dev, peak_gbs):
         torch.cuda.empty_cache()
     out["tree_head_k_sweep"] = {"workload": "config3: d=4096 B=10 topk=10 T=0.7 Gumbel sampling, cold L2",
                                 "points": sweep}
+    out["batched_head"] = dense_case(vt, dev)
     wl = build_head_workload(vt, dev, HEAD["d"], V, HEAD["B"], HEAD["topk"], HEAD["temp"], False, seed=1002)
     ms = time_head(vt, wl, 300, 20)
     gbs = wl["algo_bytes"] / (ms * 1e-3) / 1e9
@@ -340,6 +341,31 @@ def extras(vt, dev, peak_gbs):
     return out
 
 
+DENSE = dict(d=4096, K=32768, B=256, topk=8)                   # BASELINE config 4 (batched serving)
+
+
+def dense_case(vt, dev, steps=200, warmup=20):
+    """Config 4: 256 rows x K=32768 x d=4096 on the tensor-core path, per-row temperatures, Gumbel sampling."""
+    peaks, _ = measured_peaks()
+    d, K, B, topk = DENSE["d"], DENSE["K"], DENSE["B"], DENSE["topk"]
+    wl = build_head_workload(vt, dev, d, K, B, topk, 1.0, True, seed=1004, pool=4)
+    wl["T"] = vt_inputs.temperatures(B, 0.5, 1.5, seed=5001, device=dev)
+    ms = time_head(vt, wl, steps, warmup)
+    st, flags, _ = wl["ws"].read_status()
+    flops = 2.0 * B * K * d
+    tf = flops / (ms * 1e-3) / 1e12
+    gbs = wl["algo_bytes"] / (ms * 1e-3) / 1e9
+    t_tensor = flops / (float(peaks["bf16_tflops"]) * 1e12) * 1e6
+    t_hbm = wl["algo_bytes"] / (float(peaks["hbm_gbs"]) * 1e9) * 1e6
+    return {"workload": "config4: 64 seq x 4 nodes = 256 rows, d=4096, K=32768, T_b~U[0.5,1.5], top-8, Gumbel, cold L2",
+            "us_per_step": ms * 1e3, "tflops": tf, "gbs": gbs, "status": st,
+            "frac_of_bf16_burst": tf / float(peaks["bf16_tflops"]),
+            "frac_of_bf16_sustained": tf / float(peaks["bf16_tflops_sustained"]),
+            "frac_of_hbm": gbs / float(peaks["hbm_gbs"]),
+            "bound_us": {"tensor_burst": t_tensor, "hbm": t_hbm},
+            "frac_of_lower_bound": max(t_tensor, t_hbm) / (ms * 1e3)}
+
+
 def small_case(vt, dev, args, peak_gbs):
     """Short single-kernel runs sized for profiler captures (inputs larger than L2, a few launches)."""
     if args.case == "hist":
@@ -359,6 +385,8 @@ def small_case(vt, dev, args, peak_gbs):
         ms = e0.elapsed_time(e1) / args.steps
         print(json.dumps({"case": "hist", "n": n, "ms": ms, "gtok_s": n / ms / 1e6, "gbs": 4.0 * n / ms / 1e6,
                           "frac_of_measured": 4.0 * n / ms / 1e6 / peak_gbs}), flush=True)
+    elif args.case == "dense":
+        print(json.dumps(dict(case="dense", **dense_case(vt, dev, args.steps, args.warmup))), flush=True)
     else:
         wl = build_head_workload(vt, dev, TREE["d"], 32768, TREE["B"], TREE["topk"], TREE["temp"], True, seed=1003)
         ms = time_head(vt, wl, args.steps, args.warmup)
@@ -376,7 +404,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-extras", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--case", default="head", choices=["head", "hist", "tree"],
+    ap.add_argument("--case", default="head", choices=["head", "hist", "tree", "dense"],
                     help="head: the full bench line (default); hist / tree: a short run of the vocabulary "
                          "histogram (--hist-n ids) or of the tree-drafting head, for profiler captures")
     ap.add_argument("--hist-n", type=int, default=200_000_000)

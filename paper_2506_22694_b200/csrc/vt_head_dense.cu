@@ -75,6 +75,11 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* b, uint32_t parity, volatile
         if (global_ns() - t0 > kWaitLimitNs) { *abort_flag = 1; return false; }
     }
 }
+// Same, called by all 32 lanes of a warp: the outcome is voted on so the lanes never part ways
+// before a warp-collective instruction.
+__device__ __forceinline__ bool mbar_wait_warp(uint64_t* b, uint32_t parity, volatile int* abort_flag) {
+    return __all_sync(0xffffffffu, mbar_wait(b, parity, abort_flag));
+}
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm, int x, int y, uint64_t* bar) {
     asm volatile(
         "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
@@ -125,6 +130,8 @@ struct DenseGeo {
     int n_mt;         // M tiles: 1 (B <= 128) or 2
 };
 
+// KT: capacity of the register top-k list (8 or kMaxTopk)
+template <int KT>
 __global__ void __launch_bounds__(kThreads, 1)
 k_head_dense(const HeadArgs a, Ctrl* ctrl, float* __restrict__ recs, const DenseGeo geo,
              const __grid_constant__ CUtensorMap tm_h, const __grid_constant__ CUtensorMap tm_w) {
@@ -230,64 +237,106 @@ k_head_dense(const HeadArgs a, Ctrl* ctrl, float* __restrict__ recs, const Dense
         }
         float st_m = -CUDART_INF_F, st_s = 0.f, gb_s = -CUDART_INF_F, gb_z = 0.f, thr = -CUDART_INF_F;
         int gb_j = -1;
-        float tv[kMaxTopk];
-        int tj[kMaxTopk];
+        float tv[KT];
+        int tj[KT];
 #pragma unroll
-        for (int i = 0; i < kMaxTopk; ++i) { tv[i] = -CUDART_INF_F; tj[i] = -1; }
+        for (int i = 0; i < KT; ++i) { tv[i] = -CUDART_INF_F; tj[i] = -1; }
         const bool vec_u = a.uniforms && ((K & 3) == 0);
+        // 32 uniforms of row b starting at column j0 (only called with j0 < K)
+        auto load_u = [&](int j0, float (&uu)[32]) {
+            const float* up = a.uniforms + (size_t)b * K + j0;
+            if (vec_u && j0 + 32 <= K) {
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const float4 q = __ldg(reinterpret_cast<const float4*>(up) + i);
+                    uu[4 * i] = q.x; uu[4 * i + 1] = q.y; uu[4 * i + 2] = q.z; uu[4 * i + 3] = q.w;
+                }
+            } else {
+#pragma unroll
+                for (int i = 0; i < 32; ++i) uu[i] = (j0 + i < K) ? __ldg(up + i) : 0.5f;
+            }
+        };
+        const bool use_u = row_live && a.uniforms != nullptr;
+        float u[32];
+#pragma unroll
+        for (int i = 0; i < 32; ++i) u[i] = 0.5f;
         int t_local = 0;
         for (int tile = blockIdx.x; tile < geo.n_tiles; tile += gridDim.x, ++t_local) {
             const int as = t_local & 1;
-            if (!mbar_wait(&s_acc_full[as], (uint32_t)((t_local >> 1) & 1), abort_flag)) break;
+            if (!mbar_wait_warp(&s_acc_full[as], (uint32_t)((t_local >> 1) & 1), abort_flag)) break;
             tc_fence_after();
             if (mt < geo.n_mt) {
 #pragma unroll 1
                 for (int ch = 0; ch < kBN / 32; ++ch) {
+                    const int j0 = tile * kBN + ch * 32;
+                    // this chunk's uniforms are requested first (they are needed last), and the next
+                    // chunk's line is pulled into L2 meanwhile
+                    if (use_u && j0 < K) load_u(j0, u);
+                    const int jn = (ch + 1 < kBN / 32) ? j0 + 32 : (tile + (int)gridDim.x) * kBN;
+                    if (use_u && jn < K)
+                        asm volatile("prefetch.global.L2 [%0];" ::"l"(a.uniforms + (size_t)b * K + jn));
                     uint32_t r[32];
                     tc_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(as * 2 * kBN + mt * kBN + ch * 32), r);
-                    const int j0 = tile * kBN + ch * 32;
-                    if (!row_live || j0 >= K) continue;
-                    float u[32];
-                    if (a.uniforms) {
-                        const float* up = a.uniforms + (size_t)b * K + j0;
-                        if (vec_u && j0 + 32 <= K) {
+                    // Warp-uniform from here on (j0 and K are): rows that do not exist simply carry nv = 0,
+                    // i.e. 32 columns of -inf, so the warp votes below always see all 32 lanes.
+                    if (j0 < K) {
+                        const int nv = row_live ? min(32, K - j0) : 0;
+                        float z[32];
+                        float cmax = -CUDART_INF_F;
 #pragma unroll
-                            for (int i = 0; i < 8; ++i) {
-                                const float4 q = __ldg(reinterpret_cast<const float4*>(up) + i);
-                                u[4 * i] = q.x; u[4 * i + 1] = q.y; u[4 * i + 2] = q.z; u[4 * i + 3] = q.w;
-                            }
-                        } else {
-#pragma unroll
-                            for (int i = 0; i < 32; ++i) u[i] = (j0 + i < K) ? __ldg(up + i) : 0.5f;
+                        for (int i = 0; i < 32; ++i) {
+                            z[i] = (i < nv) ? __uint_as_float(r[i]) * invT : -CUDART_INF_F;
+                            cmax = fmaxf(cmax, z[i]);
                         }
-                    }
+                        if (a.dbg_logits && row_live) {
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) {
-                        const int j = j0 + i;
-                        const float x = __uint_as_float(r[i]);
-                        const bool valid = j < K;
-                        if (a.dbg_logits && valid) a.dbg_logits[(size_t)b * K + j] = x;
-                        const float z = x * invT;
-                        const float zz = valid ? z : -CUDART_INF_F;
-                        const float m_new = fmaxf(st_m, zz);
+                            for (int i = 0; i < 32; ++i)
+                                if (i < nv) a.dbg_logits[(size_t)b * K + j0 + i] = __uint_as_float(r[i]);
+                        }
+                        // running max / sum-exp: one rescale per chunk, 32 independent exponentials
+                        const float m_new = fmaxf(st_m, cmax);
                         const float m_ref = (m_new == -CUDART_INF_F) ? 0.f : m_new;
-                        st_s = st_s * __expf(st_m - m_ref) + __expf(zz - m_ref);
+                        float acc = 0.f;
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) acc += __expf(z[i] - m_ref);
+                        st_s = st_s * __expf(st_m - m_ref) + acc;
                         st_m = m_new;
                         if (a.uniforms) {
-                            const float uc = fminf(fmaxf(u[i], 0x1p-24f), 1.f - 0x1p-24f);
-                            const float sc = z - logf(-logf(uc));
-                            const bool win = valid && sc > gb_s;
-                            gb_s = win ? sc : gb_s;
-                            gb_j = win ? j : gb_j;
-                            gb_z = win ? z : gb_z;
-                        }
-                        if (valid && z > thr) {               // rare once the list is warm
-                            float cv = z;
-                            int cj = j;
 #pragma unroll
-                            for (int p = 0; p < kMaxTopk; ++p) {
+                            for (int i = 0; i < 32; ++i) {
+                                // g = -log(-log u): -log u from a short series in 1-u near 1 (where the fast
+                                // logarithm's absolute error would dominate), fast logarithms elsewhere
+                                const float uc = fminf(fmaxf(u[i], 0x1p-24f), 1.f - 0x1p-24f);
+                                const float t = 1.f - uc;
+                                const float lp = t * (1.f + t * (0.5f + t * (0.33333334f + t * (0.25f + t * 0.2f))));
+                                const float L = uc > 0.95f ? lp : -__logf(uc);
+                                const float sc = z[i] - __logf(L);
+                                const bool win = sc > gb_s;               // invalid columns carry z = -inf
+                                gb_s = win ? sc : gb_s;
+                                gb_j = win ? j0 + i : gb_j;
+                                gb_z = win ? z[i] : gb_z;
+                            }
+                        }
+                        // top-k: pull the chunk's maxima out in descending order while they beat the list's
+                        // last entry.  The loop is warp-uniform (it runs while any row of the warp still has
+                        // a candidate) and everything inside is select-based: one row's insertions never
+                        // make the other 31 rows branch.
+                        float mx = z[0];
+                        int mi = 0;
+#pragma unroll
+                        for (int i = 1; i < 32; ++i) {
+                            const bool gt = z[i] > mx;                    // strict: ties keep the lower column
+                            mx = gt ? z[i] : mx;
+                            mi = gt ? i : mi;
+                        }
+                        while (__any_sync(0xffffffffu, mx > thr)) {
+                            const bool take = mx > thr;
+                            float cv = take ? mx : -CUDART_INF_F;
+                            int cj = j0 + mi;
+#pragma unroll
+                            for (int p = 0; p < KT; ++p) {
                                 if (p < topk) {
-                                    const bool sw = cv > tv[p];       // equal values keep the earlier (lower) index first
+                                    const bool sw = cv > tv[p];           // equal values keep the lower index first
                                     const float ov = tv[p];
                                     const int oj = tj[p];
                                     tv[p] = sw ? cv : ov;
@@ -299,11 +348,23 @@ k_head_dense(const HeadArgs a, Ctrl* ctrl, float* __restrict__ recs, const Dense
                             float nt = -CUDART_INF_F;
                             int nj = -1;
 #pragma unroll
-                            for (int p = 0; p < kMaxTopk; ++p) {
+                            for (int p = 0; p < KT; ++p) {
                                 nt = (p == topk - 1) ? tv[p] : nt;
                                 nj = (p == topk - 1) ? tj[p] : nj;
                             }
-                            thr = nj >= 0 ? nt : -CUDART_INF_F;   // a threshold only once the list is full
+                            thr = nj >= 0 ? nt : -CUDART_INF_F;           // a threshold only once the list is full
+                            // drop the extracted element, find the next maximum
+                            float nmx = -CUDART_INF_F;
+                            int nmi = 0;
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) {
+                                z[i] = (take && i == mi) ? -CUDART_INF_F : z[i];
+                                const bool gt = z[i] > nmx;
+                                nmx = gt ? z[i] : nmx;
+                                nmi = gt ? i : nmi;
+                            }
+                            mx = nmx;
+                            mi = nmi;
                         }
                     }
                 }
@@ -322,7 +383,7 @@ k_head_dense(const HeadArgs a, Ctrl* ctrl, float* __restrict__ recs, const Dense
             irecs[rec_at(b, 3, topk) + c] = gb_j;
             recs[rec_at(b, 4, topk) + c] = gb_z;
 #pragma unroll
-            for (int p = 0; p < kMaxTopk; ++p)
+            for (int p = 0; p < KT; ++p)
                 if (p < topk) {
                     recs[rec_at(b, 5 + p, topk) + c] = tv[p];
                     irecs[rec_at(b, 5 + topk + p, topk) + c] = tj[p];
@@ -409,12 +470,15 @@ cudaError_t launch_head_dense(const HeadArgs& a, Ctrl* ctrl, uint8_t* scratch, c
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev < 0 || dev >= 64 || !attr_done[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(k_head_dense, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kDynSmem);
+        cudaError_t e = cudaFuncSetAttribute(k_head_dense<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kDynSmem);
+        if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(k_head_dense<kMaxTopk>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kDynSmem);
         if (e != cudaSuccess) return e;
         if (dev >= 0 && dev < 64) attr_done[dev] = 1;
     }
     float* recs = reinterpret_cast<float*>(scratch);
-    k_head_dense<<<grid, kThreads, kDynSmem, s>>>(a, ctrl, recs, geo, tm_h, tm_w);
+    if (a.topk <= 8) k_head_dense<8><<<grid, kThreads, kDynSmem, s>>>(a, ctrl, recs, geo, tm_h, tm_w);
+    else k_head_dense<kMaxTopk><<<grid, kThreads, kDynSmem, s>>>(a, ctrl, recs, geo, tm_h, tm_w);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     k_head_merge<<<a.B, 32, 0, s>>>(a, ctrl, recs, grid);

@@ -76,17 +76,21 @@ __device__ __forceinline__ unsigned long long global_ns() {
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
     return t;
 }
-// Bounded wait; false when the CTA is aborting or the time limit expired (which starts an abort).
+// Bounded wait, called by all 32 lanes of a warp; false when the CTA is aborting or the time limit
+// expired (which starts an abort).  The outcome is voted on, so the lanes of a warp never part ways
+// before a warp-collective instruction (mma, shuffle, ballot).
 __device__ __forceinline__ bool mbar_wait(uint64_t* b, uint32_t parity, volatile int* abort_flag) {
-    if (mbar_try(b, parity)) return true;
-    const unsigned long long t0 = global_ns();
-    for (;;) {
+    bool ok = mbar_try(b, parity);
+    if (!ok) {
+        const unsigned long long t0 = global_ns();
+        for (;;) {
 #pragma unroll 1
-        for (int i = 0; i < 128; ++i)
-            if (mbar_try(b, parity)) return true;
-        if (*abort_flag) return false;
-        if (global_ns() - t0 > kWaitLimitNs) { *abort_flag = 1; return false; }
+            for (int i = 0; i < 128 && !ok; ++i) ok = mbar_try(b, parity);
+            if (ok || *abort_flag) break;
+            if (global_ns() - t0 > kWaitLimitNs) { *abort_flag = 1; break; }
+        }
     }
+    return __all_sync(0xffffffffu, ok);
 }
 __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint64_t* bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
