@@ -395,6 +395,23 @@ def small_case(vt, dev, args, peak_gbs):
                           "frac_of_measured": gbs / peak_gbs}), flush=True)
 
 
+def max_over_ranks(ms: float, dist, dev) -> float:
+    """The slowest rank's time: every rank runs an independent replica of the step (the path has no
+    exchange step), so the job's time per step is the maximum over ranks.  `dist` is
+    torch.distributed or None for a single process."""
+    t = torch.tensor([ms], dtype=torch.float64, device=dev)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_line(line: dict, world: int) -> dict:
+    """Whole-job figures for N replicas: time per step is the slowest rank's, bandwidth adds up."""
+    line["n_gpus"] = world
+    line["hbm_gbs_aggregate"] = line["hbm_gbs"] * world
+    return line
+
+
 # --------------------------------------------------------------------------------------------------
 def main():
     ap = argparse.ArgumentParser()
@@ -453,16 +470,9 @@ def main():
     launches = vt.launch_count() - launches0
     if dist:
         dist.barrier()
-    ms_total = e0.elapsed_time(e1)
-    t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
-    if dist:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_step = float(t.item()) / args.steps
+    ms_step = max_over_ranks(e0.elapsed_time(e1), dist, dev) / args.steps
     e2e_ms, h2d, d2h = time_head_e2e(vt, wl, max(200, min(args.steps, 5000)), 50)
-    t2 = torch.tensor([e2e_ms], dtype=torch.float64, device=dev)
-    if dist:
-        dist.all_reduce(t2, op=dist.ReduceOp.MAX)
-    e2e_ms = float(t2.item())
+    e2e_ms = max_over_ranks(e2e_ms, dist, dev)
     st, flags, _ = wl["ws"].read_status()
     if st != 0:
         raise SystemExit("device-side status after the timed region: %s (flags %d)" % (vt.status_str(st), flags))
@@ -474,12 +484,13 @@ def main():
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": head_config(),
         "e2e": {"value": e2e_ms * 1e3, "unit": "us", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
         "gpu_launches": int(launches), "clocks": clk.summary(),
-        "hbm_gbs": gbs, "hbm_gbs_aggregate": gbs * world,
+        "hbm_gbs": gbs,
         "roofline": {"kernel": "k_head_stream", "bound": "hbm", "achieved": gbs, "peak": peak_gbs, "unit": "GB/s",
                      "frac": gbs / peak_gbs, "frac_of_8000": gbs / 8000.0, "peak_source": peak_kind,
                      "algorithmic_bytes_per_launch": wl["algo_bytes"],
                      "traffic": NCU_TRAFFIC_BYTES["k_head_stream"]},
     }
+    line = aggregate_line(line, world)
     if rank == 0 and world == 1:
         if not args.no_cpu_baseline:
             us, rows, threads, reps = oracle_head_rate(wl, seconds=12.0)
