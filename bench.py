@@ -147,14 +147,19 @@ def build_head_workload(vt, dev, d, K, B, topk, temp, sample, seed, use_map=True
                 algo_bytes=K * d * 2 + B * d * 2 + (B * K * 4 if sample else 0) + 2 * B * (1 + topk) * 4)
 
 
-def run_head_steps(vt, wl, steps, start=0):
+def run_head_steps(vt, wl, steps, start=0, overlapped=True):
+    """`steps` draft steps back to back on the current stream.  The weights are static during drafting,
+    so the steps use vt_draft_head_overlapped: a step may start fetching W_trim while the previous
+    step's last CTA is still merging.  (The very first call after the weights were written is a plain
+    vt_draft_head: see time_head.)"""
     copies, hs, us = wl["copies"], wl["hs"], wl["us"]
     for i in range(start, start + steps):
         vt.vt_draft_head(hs[i % len(hs)], copies[i % len(copies)], wl["map"], wl["T"], wl["topk"],
-                         us[i % len(us)] if us else None, ws=wl["ws"], out=wl["out"])
+                         us[i % len(us)] if us else None, ws=wl["ws"], out=wl["out"], overlapped=overlapped)
 
 
 def time_head(vt, wl, steps, warmup):
+    torch.cuda.synchronize()                    # the weights were written earlier: they are final from here on
     run_head_steps(vt, wl, warmup)
     torch.cuda.synchronize()
     e0, e1 = _events()
@@ -270,6 +275,7 @@ def head_config():
                         "T=1 greedy+top-8 (chain drafting, one vt_draft_head per step)",
             "V": V, "d": HEAD["d"], "K": HEAD["K"], "B": HEAD["B"], "topk": HEAD["topk"],
             "cold_l2": "W_trim rotated over distinct copies (>= 8x L2 streamed between reuses)",
+            "launch": "vt_draft_head_overlapped (programmatic dependent launch between consecutive steps)",
             "parallelism": "replicas"}
 
 
@@ -455,6 +461,7 @@ def main():
         return
     wl = build_head_workload(vt, dev, HEAD["d"], HEAD["K"], HEAD["B"], HEAD["topk"], HEAD["temp"], False,
                              seed=1002)
+    torch.cuda.synchronize()
     run_head_steps(vt, wl, args.warmup)
     torch.cuda.synchronize()
     if dist:

@@ -174,6 +174,21 @@ vt_status vt_draft_head(const uint16_t *h, const uint16_t *W_trim, const int32_t
                         const float *uniforms, int32_t *out_ids, float *out_logprobs, void *ws,
                         size_t ws_bytes, void *stream);
 
+/*
+ * vt_draft_head for drafting loops (Algorithm 2's inner loop runs the head once per draft token):
+ * same arguments and results, but the kernel is launched so that it may become resident and start
+ * fetching W_trim while work enqueued earlier on the stream is still finishing (programmatic
+ * dependent launch); it reads h, temp, uniforms, map and the workspace only after that earlier work
+ * has completed.  The caller promises that W_trim was not written by work still pending on the
+ * stream -- weights are static while drafting; after vt_trim_head, synchronise or make one plain
+ * vt_draft_head call first.  Streaming kernel only (B <= 16 shapes); other shapes behave exactly
+ * like vt_draft_head.
+ */
+vt_status vt_draft_head_overlapped(const uint16_t *h, const uint16_t *W_trim, const int32_t *map,
+                                   int32_t B, int32_t K, int32_t d, const float *temp, int32_t topk,
+                                   const float *uniforms, int32_t *out_ids, float *out_logprobs,
+                                   void *ws, size_t ws_bytes, void *stream);
+
 /* Parity-only variant of vt_draft_head: also writes the fp32 logits [B,K] and lse [B]
  * (log sum exp of z) when those pointers are non-NULL.  Never used for timing. */
 vt_status vt_draft_head_debug(const uint16_t *h, const uint16_t *W_trim, const int32_t *map,

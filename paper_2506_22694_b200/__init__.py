@@ -32,6 +32,7 @@ EXPORTS = (
     "vt_last_cuda_error",
     "vt_histogram", "vt_select_topk", "vt_build_vocab", "vt_build_vocab_host", "vt_trim_head",
     "vt_draft_head", "vt_draft_head_debug", "vt_draft_head_host", "vt_select_topk_static",
+    "vt_draft_head_overlapped",
 )
 
 
@@ -71,6 +72,7 @@ def lib() -> ctypes.CDLL:
         head = [c_void_p, c_void_p, c_void_p, c_int32, c_int32, c_int32, c_void_p, c_int32, c_void_p,
                 c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
         L.vt_draft_head.argtypes = head
+        L.vt_draft_head_overlapped.argtypes = head
         L.vt_draft_head_host.argtypes = head
         L.vt_draft_head_debug.argtypes = head + [c_void_p, c_void_p]
         _lib = L
@@ -221,9 +223,10 @@ def vt_trim_head(W_full: torch.Tensor, map_: torch.Tensor, W_trim: torch.Tensor 
 
 def vt_draft_head(h: torch.Tensor, W_trim: torch.Tensor, map_: torch.Tensor | None, temp: torch.Tensor,
                   topk: int, uniforms: torch.Tensor | None = None, ws: Workspace | None = None,
-                  out=None, debug: bool = False):
+                  out=None, debug: bool = False, overlapped: bool = False):
     """Algorithm 2, lines 5-6 (head part).  Returns (out_ids int32 [B,1+topk], out_logprobs fp32
-    [B,1+topk]); with debug=True also (logits fp32 [B,K], lse fp32 [B])."""
+    [B,1+topk]); with debug=True also (logits fp32 [B,K], lse fp32 [B]).  overlapped=True uses
+    vt_draft_head_overlapped (drafting loops with static weights; see the header)."""
     _dev(h, torch.bfloat16, "h")
     _dev(W_trim, torch.bfloat16, "W_trim")
     _dev(temp, torch.float32, "temp")
@@ -247,7 +250,10 @@ def vt_draft_head(h: torch.Tensor, W_trim: torch.Tensor, map_: torch.Tensor | No
         lse = torch.empty(B, dtype=torch.float32, device=h.device)
         _check("vt_draft_head_debug", lib().vt_draft_head_debug(*args, _ptr(logits), _ptr(lse)))
         return ids, lps, logits, lse
-    _check("vt_draft_head", lib().vt_draft_head(*args))
+    if overlapped:
+        _check("vt_draft_head_overlapped", lib().vt_draft_head_overlapped(*args))
+    else:
+        _check("vt_draft_head", lib().vt_draft_head(*args))
     return ids, lps
 
 

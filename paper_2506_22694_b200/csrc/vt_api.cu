@@ -261,11 +261,11 @@ vt_status vt_trim_head(const uint16_t* W_full, const int32_t* map, uint16_t* W_t
                                         as_stream(stream)));
 }
 
-vt_status vt_draft_head_debug(const uint16_t* h, const uint16_t* W_trim, const int32_t* map,
-                              int32_t B, int32_t K, int32_t d, const float* temp, int32_t topk,
-                              const float* uniforms, int32_t* out_ids, float* out_logprobs,
-                              void* ws, size_t ws_bytes, void* stream, float* out_logits,
-                              float* out_lse) {
+static vt_status draft_head_impl(const uint16_t* h, const uint16_t* W_trim, const int32_t* map,
+                                 int32_t B, int32_t K, int32_t d, const float* temp, int32_t topk,
+                                 const float* uniforms, int32_t* out_ids, float* out_logprobs,
+                                 void* ws, size_t ws_bytes, void* stream, float* out_logits,
+                                 float* out_lse, int overlap) {
     if (!h || !W_trim || !temp || !out_ids || !out_logprobs) return VT_ERR_INVALID_ARG;
     if (B < 1 || K < 1 || d < 8 || (d & 7) || topk < 1 || topk > VT_MAX_TOPK || topk > K)
         return VT_ERR_INVALID_ARG;
@@ -274,7 +274,7 @@ vt_status vt_draft_head_debug(const uint16_t* h, const uint16_t* W_trim, const i
     vt_status st = check_ws(ws, ws_bytes, vt_workspace_bytes(VT_OP_DRAFT_HEAD, 0, 0, K, d, B, topk));
     if (st != VT_OK) return st;
     uint8_t* base = static_cast<uint8_t*>(ws);
-    HeadArgs a{h, W_trim, map, B, K, d, temp, topk, uniforms, out_ids, out_logprobs, out_logits, out_lse};
+    HeadArgs a{h, W_trim, map, B, K, d, temp, topk, uniforms, out_ids, out_logprobs, out_logits, out_lse, overlap};
     if (head_skinny_supported(B, d))
         return from_cuda(launch_head_skinny(a, reinterpret_cast<Ctrl*>(base), base + VT_CTRL_BYTES,
                                             as_stream(stream)));
@@ -282,12 +282,29 @@ vt_status vt_draft_head_debug(const uint16_t* h, const uint16_t* W_trim, const i
                                        as_stream(stream)));
 }
 
+vt_status vt_draft_head_debug(const uint16_t* h, const uint16_t* W_trim, const int32_t* map,
+                              int32_t B, int32_t K, int32_t d, const float* temp, int32_t topk,
+                              const float* uniforms, int32_t* out_ids, float* out_logprobs,
+                              void* ws, size_t ws_bytes, void* stream, float* out_logits,
+                              float* out_lse) {
+    return draft_head_impl(h, W_trim, map, B, K, d, temp, topk, uniforms, out_ids, out_logprobs, ws, ws_bytes,
+                           stream, out_logits, out_lse, 0);
+}
+
 vt_status vt_draft_head(const uint16_t* h, const uint16_t* W_trim, const int32_t* map, int32_t B,
                         int32_t K, int32_t d, const float* temp, int32_t topk,
                         const float* uniforms, int32_t* out_ids, float* out_logprobs, void* ws,
                         size_t ws_bytes, void* stream) {
-    return vt_draft_head_debug(h, W_trim, map, B, K, d, temp, topk, uniforms, out_ids, out_logprobs,
-                               ws, ws_bytes, stream, nullptr, nullptr);
+    return draft_head_impl(h, W_trim, map, B, K, d, temp, topk, uniforms, out_ids, out_logprobs, ws, ws_bytes,
+                           stream, nullptr, nullptr, 0);
+}
+
+vt_status vt_draft_head_overlapped(const uint16_t* h, const uint16_t* W_trim, const int32_t* map, int32_t B,
+                                   int32_t K, int32_t d, const float* temp, int32_t topk,
+                                   const float* uniforms, int32_t* out_ids, float* out_logprobs, void* ws,
+                                   size_t ws_bytes, void* stream) {
+    return draft_head_impl(h, W_trim, map, B, K, d, temp, topk, uniforms, out_ids, out_logprobs, ws, ws_bytes,
+                           stream, nullptr, nullptr, 1);
 }
 
 vt_status vt_draft_head_host(const uint16_t* h_host, const uint16_t* W_trim, const int32_t* map,

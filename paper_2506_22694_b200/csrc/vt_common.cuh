@@ -55,6 +55,7 @@ struct HeadArgs {
     float* out_logprobs;
     float* dbg_logits;
     float* dbg_lse;
+    int32_t overlap;       // launch with programmatic stream serialization (weights may be fetched early)
 };
 bool head_skinny_supported(int32_t B, int32_t d);
 size_t head_skinny_scratch_bytes(int32_t B, int32_t K, int32_t topk);

@@ -240,6 +240,12 @@ k_head_stream(const HeadArgs a, Ctrl* ctrl, float* __restrict__ recs, const Geo 
     };
     for (int i = 0; i < S && f_item < n_items; ++i) fetch_next();          // fill the ring (no waits)
 
+    // Programmatic dependent launch (a no-op unless the launch asked for it): the next kernel on the
+    // stream may become resident as soon as SMs free up, and this kernel goes no further than
+    // fetching weights until everything enqueued before it has completed and is visible.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+
     // ---- h fragments of this warp's columns, straight from global memory into registers ----------
     uint4 hl[NCH][KBC], hh[NCH][KBC];
 #pragma unroll
@@ -489,6 +495,20 @@ cudaError_t launch_variant(const HeadArgs& a, Ctrl* ctrl, float* recs, int grid,
                                              cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit);
         if (e != cudaSuccess) return e;
         if (dev >= 0 && dev < 64) attr_done[dev] = 1;
+    }
+    if (a.overlap) {
+        cudaLaunchConfig_t cfg{};
+        cfg.gridDim = dim3((unsigned)grid);
+        cfg.blockDim = dim3(kThreads);
+        cfg.dynamicSmemBytes = smem;
+        cfg.stream = s;
+        cudaLaunchAttribute attr{};
+        attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr.val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = &attr;
+        cfg.numAttrs = 1;
+        count_launch();
+        return cudaLaunchKernelEx(&cfg, k_head_stream<NCH, KBC, TWO>, a, ctrl, recs, geo);
     }
     k_head_stream<NCH, KBC, TWO><<<grid, kThreads, smem, s>>>(a, ctrl, recs, geo);
     count_launch();

@@ -235,3 +235,41 @@ def test_config4_batched_serving_dense_head():
         assert len(set(ids[b, 1:].tolist())) == topk
         assert np.all(np.diff(lps[b, 1:]) <= 1e-6)
     assert ws.read_status() == (0, 0, 0)
+
+
+def test_overlapped_launch_matches_plain_launch_over_a_chain_of_steps():
+    """vt_draft_head_overlapped lets a step fetch weights while the previous step is finishing; the
+    results must be those of plain calls, step after step, with the workspace shared."""
+    K, d, topk = 20_000, 3072, 8
+    Ws = [vt_inputs.gaussian_bf16((K, d), 0.02, seed=50 + i, device=DEV) for i in range(3)]
+    T = vt_inputs.temperatures(1, 1.0, 1.0, 0, device=DEV)
+    hs = [vt_inputs.gaussian_bf16((1, d), 1.0, seed=60 + i, device=DEV) for i in range(12)]
+    ws = vt.Workspace(vt.workspace_bytes(vt.VT_OP_DRAFT_HEAD, 0, 0, K, d, 1, topk))
+    plain = []
+    for i, h in enumerate(hs):
+        ids, lps = vt.vt_draft_head(h, Ws[i % 3], None, T, topk, None, ws=ws)
+        plain.append((ids.clone(), lps.clone()))
+    torch.cuda.synchronize()                                   # weights are final from here on
+    outs = [(torch.empty_like(plain[0][0]), torch.empty_like(plain[0][1])) for _ in hs]
+    for i, h in enumerate(hs):                                 # back to back, nothing in between
+        vt.vt_draft_head(h, Ws[i % 3], None, T, topk, None, ws=ws, out=outs[i], overlapped=True)
+    torch.cuda.synchronize()
+    for (pi, pl), (oi, ol) in zip(plain, outs):
+        assert torch.equal(pi, oi) and torch.equal(pl, ol)
+    # tree-drafting shape with sampling and a map
+    B, topk = 10, 10
+    W = vt_inputs.gaussian_bf16((K, 4096), 0.02, seed=70, device=DEV)
+    m = torch.randperm(K * 2, device=DEV)[:K].to(torch.int32)
+    T = vt_inputs.temperatures(B, 0.7, 0.7, 0, device=DEV)
+    ws = vt.Workspace(vt.workspace_bytes(vt.VT_OP_DRAFT_HEAD, 0, 0, K, 4096, B, topk))
+    hs = [vt_inputs.gaussian_bf16((B, 4096), 1.0, seed=80 + i, device=DEV) for i in range(6)]
+    us = [vt_inputs.uniforms((B, K), seed=90 + i, device=DEV) for i in range(6)]
+    plain = [tuple(t.clone() for t in vt.vt_draft_head(h, W, m, T, topk, u, ws=ws)) for h, u in zip(hs, us)]
+    torch.cuda.synchronize()
+    outs = [(torch.empty_like(plain[0][0]), torch.empty_like(plain[0][1])) for _ in hs]
+    for i in range(6):
+        vt.vt_draft_head(hs[i], W, m, T, topk, us[i], ws=ws, out=outs[i], overlapped=True)
+    torch.cuda.synchronize()
+    for (pi, pl), (oi, ol) in zip(plain, outs):
+        assert torch.equal(pi, oi) and torch.equal(pl, ol)
+    assert ws.read_status() == (0, 0, 0)
