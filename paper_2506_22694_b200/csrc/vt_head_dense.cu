@@ -11,7 +11,7 @@
 // described in place by shared-memory descriptors and the accumulators in tensor memory: two
 // accumulator stages of 2 x 128 columns, so the epilogue of tile t overlaps the MMAs of tile t+1.
 // Eight epilogue warps read the accumulators back with tcgen05.ld -- TMEM lane = hidden row, so every
-// thread owns one hidden row and walks its 128 logits of the tile: running max / sum-exp of
+// thread owns one hidden row and walks its 128 logits of the tile, 16 at a time: running max / sum-exp of
 // z = logit / T_b, Gumbel-max candidate from the caller's uniforms, and a sorted top-k list kept in
 // registers.  Logits never go to HBM.  Per CTA and hidden row one record goes to scratch; a second
 // small kernel (one warp per hidden row) merges the records, applies the index mapper and writes
@@ -36,6 +36,7 @@ constexpr int kTileBytes = kBM * kBK * 2; // 16 KB: one operand tile of a stage
 constexpr int kStageBytes = 3 * kTileBytes;
 constexpr int kEpiWarps = 8;
 constexpr int kThreads = (2 + kEpiWarps) * 32;
+constexpr int kCh = 16;                   // accumulator columns per epilogue step (keeps the row state in registers)
 constexpr int kTmemCols = 512;            // 2 accumulator stages x 2 M tiles x 128 columns
 constexpr int kMaxTopk = 16;              // top-k list lives in registers
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
@@ -96,16 +97,12 @@ __device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t a_desc, uint64_
         "{ .reg .pred p; setp.ne.b32 p, %4, 0; tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p; }"
         ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(acc) : "memory");
 }
-// 32 consecutive accumulator columns of this thread's TMEM lane
-__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+// 16 consecutive accumulator columns of this thread's TMEM lane
+__device__ __forceinline__ void tc_ld16(uint32_t taddr, uint32_t (&r)[16]) {
     asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,"
-        "%28,%29,%30,%31}, [%32];"
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
         : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
-          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
-          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
         : "r"(taddr));
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
@@ -240,26 +237,14 @@ k_head_dense(const HeadArgs a, Ctrl* ctrl, float* __restrict__ recs, const Dense
         float tv[KT];
         int tj[KT];
 #pragma unroll
-        for (int i = 0; i < KT; ++i) { tv[i] = -CUDART_INF_F; tj[i] = -1; }
+        // the list sits at the END of the arrays (slots KT-topk .. KT-1, descending), behind +inf
+        // sentinels: its last entry -- the insertion threshold -- is then always slot KT-1, a register
+        for (int i = 0; i < KT; ++i) { tv[i] = (i < KT - topk) ? CUDART_INF_F : -CUDART_INF_F; tj[i] = -1; }
         const bool vec_u = a.uniforms && ((K & 3) == 0);
-        // 32 uniforms of row b starting at column j0 (only called with j0 < K)
-        auto load_u = [&](int j0, float (&uu)[32]) {
-            const float* up = a.uniforms + (size_t)b * K + j0;
-            if (vec_u && j0 + 32 <= K) {
-#pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    const float4 q = __ldg(reinterpret_cast<const float4*>(up) + i);
-                    uu[4 * i] = q.x; uu[4 * i + 1] = q.y; uu[4 * i + 2] = q.z; uu[4 * i + 3] = q.w;
-                }
-            } else {
-#pragma unroll
-                for (int i = 0; i < 32; ++i) uu[i] = (j0 + i < K) ? __ldg(up + i) : 0.5f;
-            }
-        };
         const bool use_u = row_live && a.uniforms != nullptr;
-        float u[32];
+        float u[kCh];
 #pragma unroll
-        for (int i = 0; i < 32; ++i) u[i] = 0.5f;
+        for (int i = 0; i < kCh; ++i) u[i] = 0.5f;
         int t_local = 0;
         for (int tile = blockIdx.x; tile < geo.n_tiles; tile += gridDim.x, ++t_local) {
             const int as = t_local & 1;
@@ -267,43 +252,55 @@ k_head_dense(const HeadArgs a, Ctrl* ctrl, float* __restrict__ recs, const Dense
             tc_fence_after();
             if (mt < geo.n_mt) {
 #pragma unroll 1
-                for (int ch = 0; ch < kBN / 32; ++ch) {
-                    const int j0 = tile * kBN + ch * 32;
+                for (int ch = 0; ch < kBN / kCh; ++ch) {
+                    const int j0 = tile * kBN + ch * kCh;
                     // this chunk's uniforms are requested first (they are needed last), and the next
                     // chunk's line is pulled into L2 meanwhile
-                    if (use_u && j0 < K) load_u(j0, u);
-                    const int jn = (ch + 1 < kBN / 32) ? j0 + 32 : (tile + (int)gridDim.x) * kBN;
-                    if (use_u && jn < K)
+                    if (use_u && j0 < K) {
+                        const float* up = a.uniforms + (size_t)b * K + j0;
+                        if (vec_u && j0 + kCh <= K) {
+#pragma unroll
+                            for (int i = 0; i < kCh / 4; ++i) {
+                                const float4 q = __ldg(reinterpret_cast<const float4*>(up) + i);
+                                u[4 * i] = q.x; u[4 * i + 1] = q.y; u[4 * i + 2] = q.z; u[4 * i + 3] = q.w;
+                            }
+                        } else {
+#pragma unroll
+                            for (int i = 0; i < kCh; ++i) u[i] = (j0 + i < K) ? __ldg(up + i) : 0.5f;
+                        }
+                    }
+                    const int jn = (ch + 2 < kBN / kCh) ? j0 + 2 * kCh : (tile + (int)gridDim.x) * kBN;
+                    if (use_u && jn < K && (ch & 1) == 0)
                         asm volatile("prefetch.global.L2 [%0];" ::"l"(a.uniforms + (size_t)b * K + jn));
-                    uint32_t r[32];
-                    tc_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(as * 2 * kBN + mt * kBN + ch * 32), r);
+                    uint32_t r[kCh];
+                    tc_ld16(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(as * 2 * kBN + mt * kBN + ch * kCh), r);
                     // Warp-uniform from here on (j0 and K are): rows that do not exist simply carry nv = 0,
-                    // i.e. 32 columns of -inf, so the warp votes below always see all 32 lanes.
+                    // i.e. columns of -inf, so the warp votes below always see all 32 lanes.
                     if (j0 < K) {
-                        const int nv = row_live ? min(32, K - j0) : 0;
-                        float z[32];
+                        const int nv = row_live ? min(kCh, K - j0) : 0;
+                        float z[kCh];
                         float cmax = -CUDART_INF_F;
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) {
+                        for (int i = 0; i < kCh; ++i) {
                             z[i] = (i < nv) ? __uint_as_float(r[i]) * invT : -CUDART_INF_F;
                             cmax = fmaxf(cmax, z[i]);
                         }
                         if (a.dbg_logits && row_live) {
 #pragma unroll
-                            for (int i = 0; i < 32; ++i)
+                            for (int i = 0; i < kCh; ++i)
                                 if (i < nv) a.dbg_logits[(size_t)b * K + j0 + i] = __uint_as_float(r[i]);
                         }
-                        // running max / sum-exp: one rescale per chunk, 32 independent exponentials
+                        // running max / sum-exp: one rescale per chunk, independent exponentials
                         const float m_new = fmaxf(st_m, cmax);
                         const float m_ref = (m_new == -CUDART_INF_F) ? 0.f : m_new;
                         float acc = 0.f;
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) acc += __expf(z[i] - m_ref);
+                        for (int i = 0; i < kCh; ++i) acc += __expf(z[i] - m_ref);
                         st_s = st_s * __expf(st_m - m_ref) + acc;
                         st_m = m_new;
                         if (a.uniforms) {
 #pragma unroll
-                            for (int i = 0; i < 32; ++i) {
+                            for (int i = 0; i < kCh; ++i) {
                                 // g = -log(-log u): -log u from a short series in 1-u near 1 (where the fast
                                 // logarithm's absolute error would dominate), fast logarithms elsewhere
                                 const float uc = fminf(fmaxf(u[i], 0x1p-24f), 1.f - 0x1p-24f);
@@ -324,7 +321,7 @@ k_head_dense(const HeadArgs a, Ctrl* ctrl, float* __restrict__ recs, const Dense
                         float mx = z[0];
                         int mi = 0;
 #pragma unroll
-                        for (int i = 1; i < 32; ++i) {
+                        for (int i = 1; i < kCh; ++i) {
                             const bool gt = z[i] > mx;                    // strict: ties keep the lower column
                             mx = gt ? z[i] : mx;
                             mi = gt ? i : mi;
@@ -334,30 +331,21 @@ k_head_dense(const HeadArgs a, Ctrl* ctrl, float* __restrict__ recs, const Dense
                             float cv = take ? mx : -CUDART_INF_F;
                             int cj = j0 + mi;
 #pragma unroll
-                            for (int p = 0; p < KT; ++p) {
-                                if (p < topk) {
-                                    const bool sw = cv > tv[p];           // equal values keep the lower index first
-                                    const float ov = tv[p];
-                                    const int oj = tj[p];
-                                    tv[p] = sw ? cv : ov;
-                                    tj[p] = sw ? cj : oj;
-                                    cv = sw ? ov : cv;
-                                    cj = sw ? oj : cj;
-                                }
+                            for (int p = 0; p < KT; ++p) {                // the +inf sentinels in front never move
+                                const bool sw = cv > tv[p];               // equal values keep the lower index first
+                                const float ov = tv[p];
+                                const int oj = tj[p];
+                                tv[p] = sw ? cv : ov;
+                                tj[p] = sw ? cj : oj;
+                                cv = sw ? ov : cv;
+                                cj = sw ? oj : cj;
                             }
-                            float nt = -CUDART_INF_F;
-                            int nj = -1;
-#pragma unroll
-                            for (int p = 0; p < KT; ++p) {
-                                nt = (p == topk - 1) ? tv[p] : nt;
-                                nj = (p == topk - 1) ? tj[p] : nj;
-                            }
-                            thr = nj >= 0 ? nt : -CUDART_INF_F;           // a threshold only once the list is full
+                            thr = tj[KT - 1] >= 0 ? tv[KT - 1] : -CUDART_INF_F;   // a threshold only once the list is full
                             // drop the extracted element, find the next maximum
                             float nmx = -CUDART_INF_F;
                             int nmi = 0;
 #pragma unroll
-                            for (int i = 0; i < 32; ++i) {
+                            for (int i = 0; i < kCh; ++i) {
                                 z[i] = (take && i == mi) ? -CUDART_INF_F : z[i];
                                 const bool gt = z[i] > nmx;
                                 nmx = gt ? z[i] : nmx;
@@ -384,9 +372,9 @@ k_head_dense(const HeadArgs a, Ctrl* ctrl, float* __restrict__ recs, const Dense
             recs[rec_at(b, 4, topk) + c] = gb_z;
 #pragma unroll
             for (int p = 0; p < KT; ++p)
-                if (p < topk) {
-                    recs[rec_at(b, 5 + p, topk) + c] = tv[p];
-                    irecs[rec_at(b, 5 + topk + p, topk) + c] = tj[p];
+                if (p >= KT - topk) {
+                    recs[rec_at(b, 5 + p - (KT - topk), topk) + c] = tv[p];
+                    irecs[rec_at(b, 5 + topk + p - (KT - topk), topk) + c] = tj[p];
                 }
         }
     }
