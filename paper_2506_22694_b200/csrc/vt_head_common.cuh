@@ -11,7 +11,8 @@ namespace {
 constexpr int kMaxGrid = 160;                    // merge: each lane owns at most kMaxOwn CTA records
 constexpr int kMaxOwn = kMaxGrid / 32;
 constexpr int kMergeDepth = 4;                   // list entries per CTA staged on chip by the merge
-constexpr int kMergeStageWords = 2 * kMergeDepth * kMaxGrid;   // staging floats per merging warp
+constexpr int kSelCap = 128;                     // entries the merge's direct selection can rank
+constexpr int kMergeStageWords = 2 * kMergeDepth * kMaxGrid + 2 * kSelCap + 64;   // staging floats per merging warp
 
 __host__ __device__ inline int rec_fields(int topk) { return 5 + 2 * topk; }
 
@@ -107,6 +108,72 @@ __device__ __noinline__ void merge_records(const int32_t* map, int32_t* out_ids,
         if (gj2 >= 0 && (GJ < 0 || better(gs2, gj2, GS, GJ))) { GS = gs2; GJ = gj2; GZ = gz2; }
     }
     const float lse = M + logf(Ssum);
+    float res_v[2] = {0.f, 0.f};
+    int res_j[2] = {-1, -1};
+    bool done = false;
+    if (topk <= 32) {
+        // Direct selection.  tau = the topk-th largest of the 32 lanes' best list heads is a lower
+        // bound of the topk-th best entry overall, so only staged entries >= tau can matter: a few
+        // dozen at most.  They are compacted into shared memory and every one finds its output
+        // position as its rank -- no sequential rounds.  Falls back to the rounds below when a list
+        // might hold qualifying entries beyond the staged ones, or when too many qualify.
+        unsigned lh = 0u;
+#pragma unroll
+        for (int o = 0; o < kMaxOwn; ++o) {
+            const bool live = (lane + 32 * o < G) && ej[0][o] >= 0;
+            const unsigned h = live ? f2ord(ev[0][o]) : 0u;
+            lh = h > lh ? h : lh;
+        }
+        int rk = 0;
+#pragma unroll
+        for (int sl = 0; sl < 32; ++sl) {
+            const unsigned oh = __shfl_sync(0xffffffffu, lh, sl);
+            rk += (oh > lh || (oh == lh && sl < lane)) ? 1 : 0;
+        }
+        const unsigned at = __ballot_sync(0xffffffffu, rk == topk - 1);
+        const unsigned tau = __shfl_sync(0xffffffffu, lh, __ffs(at) - 1);
+        unsigned long long* sel = reinterpret_cast<unsigned long long*>(stv + 2 * kMergeDepth * kMaxGrid);
+        unsigned long long* outk = sel + kSelCap;
+        outk[lane] = 0ull;
+        int n = 0;
+        bool deep = false;
+#pragma unroll
+        for (int r = 0; r < kMergeDepth; ++r)
+#pragma unroll
+            for (int o = 0; o < kMaxOwn; ++o) {
+                const bool in = (lane + 32 * o < G) && r < depth && ej[r][o] >= 0 && f2ord(ev[r][o]) >= tau;
+                const unsigned bm = __ballot_sync(0xffffffffu, in);
+                if (in) {
+                    const int pos = n + __popc(bm & lanemask_lt());
+                    if (pos < kSelCap) sel[pos] = key64(ev[r][o], ej[r][o]);
+                }
+                n += __popc(bm);
+                deep = deep || (in && r == depth - 1 && depth < topk);
+            }
+        if (n <= kSelCap && !__any_sync(0xffffffffu, deep)) {
+            __syncwarp();
+            unsigned long long mine[kSelCap / 32];
+            int rk4[kSelCap / 32];
+#pragma unroll
+            for (int i = 0; i < kSelCap / 32; ++i) {
+                mine[i] = (lane + 32 * i < n) ? sel[lane + 32 * i] : 0ull;
+                rk4[i] = 0;
+            }
+            for (int e = 0; e < n; ++e) {
+                const unsigned long long k = sel[e];
+#pragma unroll
+                for (int i = 0; i < kSelCap / 32; ++i) rk4[i] += (k > mine[i]) ? 1 : 0;
+            }
+#pragma unroll
+            for (int i = 0; i < kSelCap / 32; ++i)
+                if (lane + 32 * i < n && rk4[i] < topk) outk[rk4[i]] = mine[i];
+            __syncwarp();
+            const unsigned long long k = outk[lane];
+            if (k != 0ull) { res_v[0] = key_val(k); res_j[0] = key_idx(k); }
+            done = true;
+        }
+    }
+    if (!done) {
     // heads of the lists: entry r of CTA c at stv[r * kMaxGrid + c]
     int* stj = reinterpret_cast<int*>(stv) + kMergeDepth * kMaxGrid;
 #pragma unroll
@@ -127,8 +194,6 @@ __device__ __noinline__ void merge_records(const int32_t* map, int32_t* out_ids,
         const bool live = (lane + 32 * o < G) && ej[0][o] >= 0;
         ck[o] = live ? key64(ev[0][o], ej[0][o]) : 0ull;
     }
-    float res_v[2] = {0.f, 0.f};
-    int res_j[2] = {-1, -1};
     for (int r = 0; r < topk; ++r) {
         unsigned long long lk = ck[0];
 #pragma unroll
@@ -158,6 +223,7 @@ __device__ __noinline__ void merge_records(const int32_t* map, int32_t* out_ids,
             if (r < 32) { res_v[0] = key_val(win); res_j[0] = key_idx(win); }
             else { res_v[1] = key_val(win); res_j[1] = key_idx(win); }
         }
+    }
     }
     const int row_w = 1 + topk;
     int* oid = a.out_ids + (size_t)b * row_w;

@@ -479,7 +479,7 @@ Geo make_geo(int B, int K, int d, int topk, size_t* smem_bytes) {
     g.S = S;
     g.ring_bytes = (int)(S * stage);
     *smem_bytes = g.ring_bytes + fixed;
-    const size_t merge_bytes = (size_t)B * 2 * kMergeDepth * kMaxGrid * 4;   // staging area of the merge
+    const size_t merge_bytes = (size_t)B * kMergeStageWords * 4;            // staging area of the merge
     if (*smem_bytes < merge_bytes) *smem_bytes = merge_bytes;
     return g;
 }

@@ -273,3 +273,19 @@ def test_overlapped_launch_matches_plain_launch_over_a_chain_of_steps():
     for (pi, pl), (oi, ol) in zip(plain, outs):
         assert torch.equal(pi, oi) and torch.equal(pl, ol)
     assert ws.read_status() == (0, 0, 0)
+
+
+def test_all_candidates_in_one_slab_of_the_vocabulary():
+    """The cross-CTA merge first tries a direct selection over the few best entries of every CTA's
+    list; when one CTA holds most of the global candidates that shortcut must notice and fall back."""
+    B, K, d, topk = 3, 8192, 128, 10
+    W = vt_inputs.gaussian_bf16((K, d), 0.02, seed=77, device=DEV)
+    h = vt_inputs.gaussian_bf16((B, d), 1.0, seed=78, device=DEV)
+    W[3:19] = (h[0].float() * 0.05).to(torch.bfloat16)         # 16 neighbouring rows aligned with h[0]: huge logits
+    W[5] = (h[0].float() * 0.06).to(torch.bfloat16)
+    T = vt_inputs.temperatures(B, 1.0, 1.0, 0, device=DEV)
+    u = vt_inputs.uniforms((B, K), seed=79, device=DEV)
+    gi, gl, lg, lse = _run(h, W, None, T, topk, u)
+    ref = oracle_head(h, W, None, T, topk, u)
+    check_head(ref, gi, gl, T, None, lg, lse)
+    assert set(gi[0, 1:].tolist()) <= set(range(3, 19))
