@@ -297,6 +297,21 @@ def extras(vt, dev, peak_gbs):
     out["tree_head_k_sweep"] = {"workload": "config3: d=4096 B=10 topk=10 T=0.7 Gumbel sampling, cold L2",
                                 "points": sweep}
     out["batched_head"] = dense_case(vt, dev)
+    # the paper's other drafter and task: independent 314M drafter (d=1024) and the function-calling
+    # vocabulary of about 5K tokens -- heads of 10-67 MB, where the fixed cost of a launch dominates
+    small = []
+    for name, d_, K_ in (("independent drafter d=1024 K=32768", 1024, 32768), ("independent drafter d=1024 K=5000", 1024, 5000),
+                         ("EAGLE d=3072 K=5000 (function calling)", 3072, 5000)):
+        wl = build_head_workload(vt, dev, d_, K_, 1, 8, 1.0, False, seed=1007)
+        ms = time_head(vt, wl, 2000, 50)
+        gbs = wl["algo_bytes"] / (ms * 1e-3) / 1e9
+        warm = dict(wl, copies=wl["copies"][:1])                      # one copy: the head stays in L2
+        ms_w = time_head(vt, warm, 2000, 50)
+        small.append({"workload": name + ", B=1, top-8", "mbytes": wl["algo_bytes"] / 1e6, "us_per_step_cold": ms * 1e3,
+                      "gbs_cold": gbs, "frac_of_measured_cold": gbs / peak_gbs, "us_per_step_l2_resident": ms_w * 1e3})
+        del wl, warm
+        torch.cuda.empty_cache()
+    out["small_heads"] = small
     wl = build_head_workload(vt, dev, HEAD["d"], V, HEAD["B"], HEAD["topk"], HEAD["temp"], False, seed=1002)
     ms = time_head(vt, wl, 300, 20)
     gbs = wl["algo_bytes"] / (ms * 1e-3) / 1e9
