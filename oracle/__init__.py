@@ -101,6 +101,33 @@ def select_topk(counts, K: int):
     return m, inv
 
 
+def select_topp(counts, p: float):
+    """Top-P variant of the selection (Method section).  Returns (K, map int32 [V] full ranking, inv_map [V])."""
+    counts = _c(counts, np.uint64)
+    V = counts.size
+    m = np.empty(V, dtype=np.int32)
+    inv = np.empty(V, dtype=np.int32)
+    _load().orc_select_topp.restype = c_int32
+    K = _load().orc_select_topp(_p(counts, c_uint64), c_int32(V), c_double(float(p)), _p(m, c_int32), _p(inv, c_int32))
+    if K < 0:
+        raise ValueError("select_topp: invalid arguments")
+    return int(K), m, inv
+
+
+def select_minfreq(counts, min_count: int):
+    """Minimum-frequency variant of the selection (Method section).  Returns (K, map [V], inv_map [V])."""
+    counts = _c(counts, np.uint64)
+    V = counts.size
+    m = np.empty(V, dtype=np.int32)
+    inv = np.empty(V, dtype=np.int32)
+    _load().orc_select_minfreq.restype = c_int32
+    K = _load().orc_select_minfreq(_p(counts, c_uint64), c_int32(V), c_uint64(int(min_count)), _p(m, c_int32),
+                                   _p(inv, c_int32))
+    if K < 0:
+        raise ValueError("select_minfreq: invalid arguments")
+    return int(K), m, inv
+
+
 def build_vocab(ids, V: int, K: int):
     counts, bad = histogram(ids, V)
     m, inv = select_topk(counts, K)

@@ -113,6 +113,70 @@ int orc_select_topk(const uint64_t *counts, int32_t V, int32_t K, int32_t *map,
     return 0;
 }
 
+/*
+ * Selection variants the Method section names next to Top-K: "Top-P" and "minimum frequency of
+ * tokens".  Both cut the same ranking (count descending, id ascending) at a data-dependent K:
+ *   Top-P:        the smallest K whose K most frequent ids hold at least ceil(p * total) of all
+ *                 counted tokens (p in (0,1]; total = sum of counts);
+ *   min frequency: K = number of ids with count >= min_count.
+ * Readings where the paper is silent: the target is ceil(p*total) evaluated in fp64; K is never
+ * below 1 (an empty vocabulary is useless).  map receives the FULL ranking [V]; inv_map is -1
+ * for ranks >= K.  Returns K, or -1 on invalid arguments.
+ */
+static int32_t orc_cut_ranking(const uint64_t *counts, int32_t V, int32_t K, const orc_pair *p,
+                               int32_t *map, int32_t *inv_map) {
+    (void)counts;
+    if (K < 1) K = 1;
+    if (K > V) K = V;
+    for (int32_t j = 0; j < V; ++j) {
+        map[j] = p[j].id;
+        inv_map[p[j].id] = j < K ? j : -1;
+    }
+    return K;
+}
+
+static orc_pair *orc_rank_all(const uint64_t *counts, int32_t V) {
+    orc_pair *p = (orc_pair *)malloc(sizeof(orc_pair) * (size_t)V);
+    if (!p) return NULL;
+    for (int32_t v = 0; v < V; ++v) {
+        p[v].count = counts[v];
+        p[v].id = v;
+    }
+    qsort(p, (size_t)V, sizeof(orc_pair), orc_pair_cmp);
+    return p;
+}
+
+int32_t orc_select_topp(const uint64_t *counts, int32_t V, double pfrac, int32_t *map,
+                        int32_t *inv_map) {
+    if (V <= 0 || !(pfrac > 0.0) || pfrac > 1.0) return -1;
+    orc_pair *p = orc_rank_all(counts, V);
+    if (!p) return -1;
+    uint64_t total = 0;
+    for (int32_t v = 0; v < V; ++v) total += counts[v];
+    const double target = ceil(pfrac * (double)total);
+    uint64_t cum = 0;
+    int32_t K = V;
+    for (int32_t j = 0; j < V; ++j) {
+        cum += p[j].count;
+        if ((double)cum >= target) { K = j + 1; break; }
+    }
+    K = orc_cut_ranking(counts, V, K, p, map, inv_map);
+    free(p);
+    return K;
+}
+
+int32_t orc_select_minfreq(const uint64_t *counts, int32_t V, uint64_t min_count, int32_t *map,
+                           int32_t *inv_map) {
+    if (V <= 0) return -1;
+    orc_pair *p = orc_rank_all(counts, V);
+    if (!p) return -1;
+    int32_t K = 0;
+    for (int32_t v = 0; v < V; ++v) K += counts[v] >= min_count;
+    K = orc_cut_ranking(counts, V, K, p, map, inv_map);
+    free(p);
+    return K;
+}
+
 /* Eq. 1, second line: W_trim = W[Top-K(c,k), :] -- a row gather, bit copy of bf16 words. */
 void orc_trim_head(const uint16_t *W_full, const int32_t *map, int32_t K, int32_t d,
                    uint16_t *W_trim) {

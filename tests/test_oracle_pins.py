@@ -321,3 +321,63 @@ def test_draft_head_rejects_bad_shapes():
     h = np.zeros((1, 8), dtype=np.uint16)
     with pytest.raises(ValueError):
         oracle.draft_head(h, W, None, np.ones(1, dtype=np.float32), 5, None)
+
+
+# ---- selection variants named in the Method section: Top-P and minimum frequency -----------------------
+def _brute_topp(counts, p):
+    """Definition written out: rank ids by (count desc, id asc); smallest K whose prefix holds >= ceil(p*total)."""
+    order = sorted(range(len(counts)), key=lambda v: (-int(counts[v]), v))
+    total = int(sum(int(c) for c in counts))
+    target = int(np.ceil(p * total))
+    cum = 0
+    for j, v in enumerate(order):
+        cum += int(counts[v])
+        if cum >= target:
+            return max(1, j + 1), order
+    return len(counts), order
+
+
+def test_select_topp_hand_example_and_definition_on_random_counts():
+    c = np.array([5, 0, 3, 3, 9, 0, 1], dtype=np.uint64)          # total 21; ranking 4,0,2,3,6,1,5
+    K, m, inv = oracle.select_topp(c, 0.5)                           # ceil(10.5) = 11 -> 9 + 5
+    assert K == 2 and m.tolist() == [4, 0, 2, 3, 6, 1, 5] and inv.tolist() == [1, -1, -1, -1, 0, -1, -1]
+    assert oracle.select_topp(c, 9 / 21)[0] == 1                     # exactly the top id's share
+    assert oracle.select_topp(c, 1.0)[0] == 5                        # all ids that were ever seen
+    rng = np.random.default_rng(7)
+    for _ in range(200):
+        V = int(rng.integers(1, 40))
+        counts = rng.integers(0, 6, V).astype(np.uint64)
+        p = float(rng.uniform(0.01, 1.0))
+        K, m, inv = oracle.select_topp(counts, p)
+        Kb, order = _brute_topp(counts, p)
+        assert K == Kb and m.tolist() == order
+        assert [int(inv[v]) for v in order] == [j if j < K else -1 for j in range(V)]
+
+
+def test_select_topp_is_minimal_and_monotone_in_p():
+    rng = np.random.default_rng(8)
+    counts = np.sort(rng.zipf(1.3, 5000).astype(np.uint64))[::-1].copy()
+    rng.shuffle(counts)
+    total = int(counts.sum())
+    last = 0
+    for p in (0.1, 0.5, 0.9, 0.99, 1.0):
+        K, m, _ = oracle.select_topp(counts, p)
+        cum = np.cumsum(counts[m].astype(np.int64))
+        target = int(np.ceil(p * total))
+        assert cum[K - 1] >= target and (K == 1 or cum[K - 2] < target)
+        assert K >= last
+        last = K
+
+
+def test_select_minfreq_counts_ids_at_or_above_the_threshold():
+    c = np.array([5, 0, 3, 3, 9, 0, 1], dtype=np.uint64)
+    assert oracle.select_minfreq(c, 3)[0] == 4 and oracle.select_minfreq(c, 0)[0] == 7
+    assert oracle.select_minfreq(c, 10)[0] == 1                      # never an empty vocabulary
+    rng = np.random.default_rng(9)
+    counts = rng.integers(0, 50, 3000).astype(np.uint64)
+    for f in (1, 7, 25, 49):
+        K, m, inv = oracle.select_minfreq(counts, f)
+        assert K == int((counts >= f).sum())
+        assert np.all(counts[m[:K]] >= f) and np.all(counts[m[K:]] < f)
+        ref_m, ref_inv = oracle.select_topk(counts, K)                # the same cut of the same ranking
+        assert np.array_equal(m[:K], ref_m) and np.array_equal(inv, ref_inv)
