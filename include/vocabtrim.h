@@ -112,6 +112,21 @@ vt_status vt_select_topk(const uint32_t *counts, int32_t V, int32_t K, int32_t *
                          int32_t *inv_map, void *ws, size_t ws_bytes, void *stream);
 
 /*
+ * Section 3 (Method) names two selection rules besides Top-K: Top-P and a minimum token frequency.
+ * Both cut the same ranking (count descending, id ascending) at a K found from the data:
+ *   vt_select_topp    : smallest K whose K most frequent ids hold at least ceil(p * total) of all
+ *                       counted tokens, 0 < p <= 1 (evaluated in fp64);
+ *   vt_select_minfreq : K = number of ids with count >= min_count.
+ * K is clamped to [1, V] and written to the DEVICE int32 *k_out.  map receives the FULL ranking
+ * ([V], the first K entries are the trimmed vocabulary), inv_map [V] is -1 for ranks >= K.
+ * Workspace: vt_workspace_bytes(VT_OP_SELECT_TOPK, 0, V, V, ...).  Integer work: exact and unique.
+ */
+vt_status vt_select_topp(const uint32_t *counts, int32_t V, double p, int32_t *map, int32_t *inv_map,
+                         int32_t *k_out, void *ws, size_t ws_bytes, void *stream);
+vt_status vt_select_minfreq(const uint32_t *counts, int32_t V, uint32_t min_count, int32_t *map,
+                            int32_t *inv_map, int32_t *k_out, void *ws, size_t ws_bytes, void *stream);
+
+/*
  * vt_select_topk without a workspace.  (The paper has no counterpart: this entry point exists for
  * the sake of callers, not of the method.)  Same result as vt_select_topk, for callers that cannot
  * allocate device memory or pass scratch along: code living inside another runtime's memory pool,

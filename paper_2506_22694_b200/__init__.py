@@ -13,7 +13,7 @@ from __future__ import annotations
 
 import ctypes
 import os
-from ctypes import c_char_p, c_float, c_int, c_int32, c_int64, c_size_t, c_uint32, c_uint64, c_void_p
+from ctypes import c_char_p, c_double, c_float, c_int, c_int32, c_int64, c_size_t, c_uint32, c_uint64, c_void_p
 
 import torch
 
@@ -32,7 +32,7 @@ EXPORTS = (
     "vt_last_cuda_error",
     "vt_histogram", "vt_select_topk", "vt_build_vocab", "vt_build_vocab_host", "vt_trim_head",
     "vt_draft_head", "vt_draft_head_debug", "vt_draft_head_host", "vt_select_topk_static",
-    "vt_draft_head_overlapped",
+    "vt_draft_head_overlapped", "vt_select_topp", "vt_select_minfreq",
 )
 
 
@@ -65,6 +65,8 @@ def lib() -> ctypes.CDLL:
         L.vt_histogram.argtypes = [c_void_p, c_int64, c_int32, c_void_p, c_int, c_void_p, c_size_t, c_void_p]
         L.vt_select_topk.argtypes = [c_void_p, c_int32, c_int32, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
         L.vt_select_topk_static.argtypes = [c_void_p, c_int32, c_int32, c_void_p, c_void_p, c_void_p]
+        L.vt_select_topp.argtypes = [c_void_p, c_int32, c_double, c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
+        L.vt_select_minfreq.argtypes = [c_void_p, c_int32, c_uint32, c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
         L.vt_build_vocab.argtypes = [c_void_p, c_int64, c_int32, c_int32, c_void_p, c_void_p, c_void_p,
                                      c_size_t, c_void_p]
         L.vt_build_vocab_host.argtypes = L.vt_build_vocab.argtypes
@@ -162,6 +164,28 @@ def vt_select_topk(counts: torch.Tensor, K: int, ws: Workspace | None = None):
     _check("vt_select_topk", lib().vt_select_topk(_ptr(counts), V, K, _ptr(map_), _ptr(inv), c_void_p(ws.ptr),
                                                   ws.nbytes, _stream()))
     return map_, inv
+
+
+def _select_cut(counts: torch.Tensor, ws, call, *arg):
+    _dev(counts, torch.int32, "counts")
+    V = counts.numel()
+    map_ = torch.empty(V, dtype=torch.int32, device=counts.device)
+    inv = torch.empty(V, dtype=torch.int32, device=counts.device)
+    k_out = torch.empty(1, dtype=torch.int32, device=counts.device)
+    ws = _ws(ws, workspace_bytes(VT_OP_SELECT_TOPK, 0, V, V), counts)
+    fn = getattr(lib(), call)
+    _check(call, fn(_ptr(counts), V, *arg, _ptr(map_), _ptr(inv), _ptr(k_out), c_void_p(ws.ptr), ws.nbytes, _stream()))
+    return k_out, map_, inv
+
+
+def vt_select_topp(counts: torch.Tensor, p: float, ws: Workspace | None = None):
+    """Top-P selection (Method section): returns (K device int32 [1], map [V] full ranking, inv_map [V])."""
+    return _select_cut(counts, ws, "vt_select_topp", c_double(float(p)))
+
+
+def vt_select_minfreq(counts: torch.Tensor, min_count: int, ws: Workspace | None = None):
+    """Minimum-frequency selection (Method section): returns (K device int32 [1], map [V], inv_map [V])."""
+    return _select_cut(counts, ws, "vt_select_minfreq", c_uint32(int(min_count)))
 
 
 def vt_select_topk_static(counts: torch.Tensor, K: int, out=None):

@@ -180,6 +180,29 @@ vt_status vt_select_topk(const uint32_t* counts, int32_t V, int32_t K, int32_t* 
                                         as_stream(stream)));
 }
 
+static vt_status select_cut_impl(const uint32_t* counts, int32_t V, int mode, double p, uint32_t min_count,
+                                 int32_t* map, int32_t* inv_map, int32_t* k_out, void* ws, size_t ws_bytes,
+                                 void* stream) {
+    if (!counts || !map || !inv_map || !k_out || V < 1) return VT_ERR_INVALID_ARG;
+    if (mode == 0 && (!(p > 0.0) || p > 1.0)) return VT_ERR_INVALID_ARG;
+    vt_status st = check_ws(ws, ws_bytes, vt_workspace_bytes(VT_OP_SELECT_TOPK, 0, V, V, 0, 0, 0));
+    if (st != VT_OK) return st;
+    uint8_t* base = static_cast<uint8_t*>(ws);
+    cudaError_t e = launch_select_topk(counts, V, V, map, inv_map, base + VT_CTRL_BYTES, as_stream(stream));
+    if (e != cudaSuccess) return from_cuda(e);
+    return from_cuda(launch_select_cut(counts, V, mode, p, min_count, map, inv_map, k_out, as_stream(stream)));
+}
+
+vt_status vt_select_topp(const uint32_t* counts, int32_t V, double p, int32_t* map, int32_t* inv_map,
+                         int32_t* k_out, void* ws, size_t ws_bytes, void* stream) {
+    return select_cut_impl(counts, V, 0, p, 0u, map, inv_map, k_out, ws, ws_bytes, stream);
+}
+
+vt_status vt_select_minfreq(const uint32_t* counts, int32_t V, uint32_t min_count, int32_t* map,
+                            int32_t* inv_map, int32_t* k_out, void* ws, size_t ws_bytes, void* stream) {
+    return select_cut_impl(counts, V, 1, 1.0, min_count, map, inv_map, k_out, ws, ws_bytes, stream);
+}
+
 vt_status vt_build_vocab(const int32_t* ids, int64_t n, int32_t V, int32_t K, int32_t* map,
                          int32_t* inv_map, void* ws, size_t ws_bytes, void* stream) {
     if (n < 0 || n >= ((int64_t)1 << 32) || V < 1 || K < 1 || K > V || !map || !inv_map || (n > 0 && !ids))

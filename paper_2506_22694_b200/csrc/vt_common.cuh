@@ -40,6 +40,9 @@ size_t select_scratch_bytes(int32_t V);
 cudaError_t launch_select_topk(const uint32_t* counts, int32_t V, int32_t K, int32_t* map,
                                int32_t* inv_map, uint8_t* scratch, cudaStream_t s);
 
+cudaError_t launch_select_cut(const uint32_t* counts, int32_t V, int mode, double pfrac, uint32_t min_count,
+                              const int32_t* map, int32_t* inv_map, int32_t* k_out, cudaStream_t s);
+
 cudaError_t launch_gather_rows(const uint16_t* W_full, const int32_t* map, uint16_t* W_trim,
                                int32_t V, int32_t K, int32_t d, Ctrl* ctrl, cudaStream_t s);
 

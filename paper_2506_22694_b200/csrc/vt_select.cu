@@ -140,7 +140,62 @@ k_select_sort(const uint32_t* counts, int32_t V, int32_t K, int32_t* map, int32_
     }
 }
 
+// Cut of a full ranking at a data-dependent K (the Method section's Top-P and minimum-frequency
+// variants of the selection).  `map` holds all V ids in rank order.  mode 0: smallest K whose prefix
+// of counts reaches ceil(p * total); mode 1: K = number of ids with count >= min_count.  K is clamped
+// to [1, V]; inv_map entries of ranks >= K become -1.  One CTA: V is about 1e5, this is latency.
+__global__ void __launch_bounds__(kThreads, 1)
+k_select_cut(const uint32_t* __restrict__ counts, int32_t V, int mode, double pfrac, uint32_t min_count,
+             const int32_t* __restrict__ map, int32_t* __restrict__ inv_map, int32_t* __restrict__ k_out) {
+    __shared__ unsigned long long s_part[kThreads];
+    __shared__ unsigned long long s_total;
+    __shared__ int s_k;
+    const int per = (V + kThreads - 1) / kThreads;                 // consecutive ranks per thread
+    const int j0 = min(V, (int)threadIdx.x * per), j1 = min(V, j0 + per);
+    unsigned long long sum = 0;
+    int ge = 0;
+    for (int j = j0; j < j1; ++j) {
+        const uint32_t c = counts[map[j]];
+        sum += c;
+        ge += c >= min_count;
+    }
+    s_part[threadIdx.x] = mode == 0 ? sum : (unsigned long long)ge;
+    if (threadIdx.x == 0) s_k = V;
+    __syncthreads();
+    if (threadIdx.x == 0) {                                        // exclusive scan of 1024 partials: trivial serially
+        unsigned long long run = 0;
+        for (int t = 0; t < kThreads; ++t) {
+            const unsigned long long x = s_part[t];
+            s_part[t] = run;
+            run += x;
+        }
+        s_total = run;
+    }
+    __syncthreads();
+    if (mode == 0) {
+        const double target = ceil(pfrac * (double)s_total);
+        unsigned long long cum = s_part[threadIdx.x];
+        for (int j = j0; j < j1; ++j) {
+            cum += counts[map[j]];
+            if ((double)cum >= target) { atomicMin(&s_k, j + 1); break; }
+        }
+    } else if (threadIdx.x == 0) {
+        s_k = (int)s_total;
+    }
+    __syncthreads();
+    const int K = max(1, min(V, s_k));
+    if (threadIdx.x == 0) *k_out = K;
+    for (int j = K + (int)threadIdx.x; j < V; j += kThreads) inv_map[map[j]] = -1;
+}
+
 }  // namespace
+
+cudaError_t launch_select_cut(const uint32_t* counts, int32_t V, int mode, double pfrac, uint32_t min_count,
+                              const int32_t* map, int32_t* inv_map, int32_t* k_out, cudaStream_t s) {
+    k_select_cut<<<1, kThreads, 0, s>>>(counts, V, mode, pfrac, min_count, map, inv_map, k_out);
+    count_launch();
+    return cudaGetLastError();
+}
 
 size_t select_scratch_bytes(int32_t V) { return 4 * align_up((size_t)V * 4, 256); }
 

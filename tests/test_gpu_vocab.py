@@ -166,3 +166,58 @@ def test_config5_corpus_scale_build_and_gather():
         Wt = vt.vt_trim_head(W, m)
         assert np.array_equal(vt_inputs.bf16_bits(Wt).cpu().numpy().view(np.uint16), oracle.trim_head(Wbits, rm))
     _assert_clean(ws)
+
+
+def _counts_for_cut(V, n, seed):
+    ids = vt_inputs.zipf_ids(n, V, 1.1, seed=seed, noise_frac=0.05)
+    ref, _ = oracle.histogram(ids.numpy(), V)
+    return ref
+
+
+@pytest.mark.parametrize("V,n", [(128256, 3_000_000), (50_000, 200_003), (1000, 5000), (33, 10)])
+@pytest.mark.parametrize("p", [1e-9, 0.25, 0.5, 0.9, 0.99, 0.999999, 1.0])
+def test_select_topp_matches_oracle(V, n, p):
+    ref = _counts_for_cut(V, n, seed=V % 101 + 3)
+    counts = torch.from_numpy(ref.astype(np.uint32).view(np.int32)).to(DEV)
+    ws = vt.Workspace(vt.workspace_bytes(vt.VT_OP_SELECT_TOPK, 0, V, V))
+    k_out, map_, inv = vt.vt_select_topp(counts, p, ws=ws)
+    K, rmap, rinv = oracle.select_topp(ref, p)
+    assert int(k_out.item()) == K
+    assert np.array_equal(map_.cpu().numpy(), rmap)
+    assert np.array_equal(inv.cpu().numpy(), rinv)
+    _assert_clean(ws)
+
+
+@pytest.mark.parametrize("V,n", [(128256, 3_000_000), (4096, 100_000), (33, 10)])
+@pytest.mark.parametrize("f", [0, 1, 2, 5, 100, 10_000, 2**31])
+def test_select_minfreq_matches_oracle(V, n, f):
+    ref = _counts_for_cut(V, n, seed=V % 89 + 5)
+    counts = torch.from_numpy(ref.astype(np.uint32).view(np.int32)).to(DEV)
+    ws = vt.Workspace(vt.workspace_bytes(vt.VT_OP_SELECT_TOPK, 0, V, V))
+    k_out, map_, inv = vt.vt_select_minfreq(counts, f, ws=ws)
+    K, rmap, rinv = oracle.select_minfreq(ref, f)
+    assert int(k_out.item()) == K
+    assert np.array_equal(map_.cpu().numpy(), rmap)
+    assert np.array_equal(inv.cpu().numpy(), rinv)
+    _assert_clean(ws)
+
+
+def test_select_cut_degenerate_counts_and_bad_arguments():
+    V = 4096
+    ws = vt.Workspace(vt.workspace_bytes(vt.VT_OP_SELECT_TOPK, 0, V, V))
+    zero = torch.zeros(V, dtype=torch.int32, device=DEV)
+    for call, arg in ((vt.vt_select_topp, 0.5), (vt.vt_select_minfreq, 1)):
+        k_out, map_, inv = call(zero, arg, ws=ws)
+        K, rmap, rinv = (oracle.select_topp if call is vt.vt_select_topp else oracle.select_minfreq)(
+            np.zeros(V, dtype=np.uint64), arg)
+        assert int(k_out.item()) == K
+        assert np.array_equal(map_.cpu().numpy(), rmap) and np.array_equal(inv.cpu().numpy(), rinv)
+    big = np.full(V, 2**32 - 1, dtype=np.uint64)            # prefix sums need 64 bits
+    counts = torch.from_numpy(big.astype(np.uint32).view(np.int32)).to(DEV)
+    k_out, map_, inv = vt.vt_select_topp(counts, 0.75, ws=ws)
+    K, rmap, rinv = oracle.select_topp(big, 0.75)
+    assert int(k_out.item()) == K == 3072
+    assert np.array_equal(inv.cpu().numpy(), rinv)
+    for p in (0.0, -0.1, 1.5, float("nan")):
+        with pytest.raises(vt.VocabTrimError):
+            vt.vt_select_topp(zero, p, ws=ws)
