@@ -5,8 +5,9 @@ product package never does.  It compiles the C file with gcc on first use and ca
 ctypes on numpy arrays.  Nothing here touches CUDA.
 
 Parity pins: see the header of vt_oracle.c -- pinned to definitions, invariants, library special
-cases and brute force by the CPU tests; parity with paper-printed values is unpinned because
-the paper prints no numeric example for this path.
+cases and brute force by the CPU tests; parity with paper-printed values is unpinned for the head
+and the vocabulary build because the paper prints no numeric example for them; `mbsu` is pinned to
+the (block efficiency, speed-up) pairs of the paper's Table 1.
 """
 from __future__ import annotations
 
@@ -219,3 +220,39 @@ def draft_head(h, W_trim, map_, temp, topk: int, uniforms=None, want_full: bool 
     if rc:
         raise ValueError("draft_head: invalid shape arguments")
     return r
+
+
+def verify_greedy(token, parent, target):
+    """Greedy verification of S drafted blocks (Experiments section; Algorithm 2's accept loop).
+
+    token [S,N], parent [S,N] or None (chains), target [S,N+1].  Returns (n_accept int32 [S],
+    path int32 [S,N] padded with -1, emitted int32 [S,N+1] padded with -1)."""
+    token = _c(token, np.int32)
+    target = _c(target, np.int32)
+    S, N = token.shape
+    assert target.shape == (S, N + 1)
+    if parent is not None:
+        parent = _c(parent, np.int32)
+        assert parent.shape == (S, N)
+    n_acc = np.zeros(S, dtype=np.int32)
+    path = np.full((S, N), -1, dtype=np.int32)
+    emitted = np.full((S, N + 1), -1, dtype=np.int32)
+    fn = _load().orc_verify_greedy
+    fn.restype = c_int32
+    for s in range(S):
+        n_acc[s] = fn(_p(token[s], c_int32), _p(parent[s], c_int32) if parent is not None else None,
+                      _p(target[s], c_int32), c_int32(N), _p(path[s], c_int32), _p(emitted[s], c_int32))
+    return n_acc, path, emitted
+
+
+def block_efficiency(n_accept) -> float:
+    """tau: mean number of tokens a block yields = accepted drafts + the target's own token
+    (Performance Metrics paragraph)."""
+    n_accept = np.asarray(n_accept, dtype=np.float64)
+    return float(np.mean(n_accept + 1.0))
+
+
+def mbsu(tau: float, c: float, gamma: int) -> float:
+    """Memory-bound speed-up tau / (c * gamma + 1), c = draft / target parameter ratio
+    (Performance Metrics paragraph)."""
+    return float(tau) / (float(c) * float(gamma) + 1.0)

@@ -10,8 +10,10 @@
  * silent (tie rules, clamping of uniforms, order of the map) the reading is noted inline.
  *
  * Parity pins: every function here is pinned by CPU tests against closed forms, invariants,
- * library special cases and brute force.  The paper prints no worked numeric example for this
- * path, so parity with *paper-printed values* is unpinned; parity with the definitions is pinned.
+ * library special cases and brute force.  The paper prints no worked numeric example for the
+ * head or the vocabulary build, so parity with *paper-printed values* is unpinned there; parity
+ * with the definitions is pinned.  The speed-up formula of the Python face is pinned to the
+ * (block efficiency, speed-up) pairs the paper's Table 1 prints.
  *
  * Threading: the only parallel construct is an OpenMP "parallel for" over independent
  * vocabulary rows in orc_logits (each dot product is still summed in index order by one
@@ -320,4 +322,39 @@ int orc_draft_head(const uint16_t *h, const uint16_t *W_trim, const int32_t *map
     free(z);
     if (!logits_out) free(logits);
     return 0;
+}
+
+/*
+ * Greedy verification of one drafted block (Experiments section: the target decodes greedily and a
+ * draft token is accepted only when it equals the target's token; Algorithm 2's accept loop).
+ *   token[i]   drafted id of node i, already a full-vocabulary id (after the index mapper);
+ *   parent[i]  index of node i's parent, -1 for a child of the last committed token; a node whose
+ *              parent is not in [-1, i) can never be reached.  parent == NULL means a chain
+ *              (parent[i] = i - 1);
+ *   target[0]  the target's greedy token after the committed prefix, target[i + 1] the one after
+ *              the path ending in node i.
+ * Walk from the committed prefix: at the current node the target's token decides; the child that
+ * carries exactly this token (the lowest-indexed one, should several) is accepted and becomes the
+ * current node; with no such child the block ends.  The target's token at the last accepted node
+ * is emitted after the accepted ones, so a block yields n + 1 tokens, at most depth + 1.
+ * Returns n; path[0..n) = accepted node indices, emitted[0..n] = the tokens of the block.
+ */
+int32_t orc_verify_greedy(const int32_t *token, const int32_t *parent, const int32_t *target,
+                          int32_t N, int32_t *path, int32_t *emitted) {
+    int32_t cur = -1, n = 0;
+    for (;;) {
+        const int32_t want = target[cur + 1];
+        int32_t next = -1;
+        for (int32_t i = cur + 1; i < N && next < 0; ++i) {
+            const int32_t par = parent ? parent[i] : i - 1;
+            if (par == cur && token[i] == want) next = i;
+        }
+        if (next < 0) break;
+        path[n] = next;
+        emitted[n] = token[next];
+        ++n;
+        cur = next;
+    }
+    emitted[n] = target[cur + 1];
+    return n;
 }

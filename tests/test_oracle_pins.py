@@ -4,6 +4,7 @@ tiny inputs -- chosen so that a dropped term, a wrong sign or index, or a transp
 fails at least one of them.  No GPU is involved."""
 import itertools
 import math
+import os
 
 import numpy as np
 import pytest
@@ -381,3 +382,121 @@ def test_select_minfreq_counts_ids_at_or_above_the_threshold():
         assert np.all(counts[m[:K]] >= f) and np.all(counts[m[K:]] < f)
         ref_m, ref_inv = oracle.select_topk(counts, K)                # the same cut of the same ranking
         assert np.array_equal(m[:K], ref_m) and np.array_equal(inv, ref_inv)
+
+
+# ---- greedy verification, block efficiency, MBSU (Experiments section; Algorithm 2's accept loop)
+
+def _consistent_nodes(token, parent, target):
+    """Set formulation: a node is accepted iff its token is the target's token at its parent and the
+    parent is accepted (the committed prefix is).  With distinct sibling tokens this set is a path."""
+    N = len(token)
+    ok = np.zeros(N, dtype=bool)
+    for i in range(N):                                   # parents precede children
+        par = parent[i]
+        ok[i] = (par == -1 or ok[par]) and token[i] == target[par + 1]
+    return np.flatnonzero(ok)
+
+
+def test_verify_chain_is_the_first_mismatch():
+    rng = np.random.default_rng(5)
+    S, N = 200, 7
+    token = rng.integers(0, 4, size=(S, N)).astype(np.int32)
+    target = rng.integers(0, 4, size=(S, N + 1)).astype(np.int32)
+    target[:, :N] = np.where(rng.random((S, N)) < 0.7, token, target[:, :N])
+    n_acc, path, emitted = oracle.verify_greedy(token, None, target)
+    match = token == target[:, :N]
+    first_miss = np.where(match.all(1), N, np.argmin(match, axis=1))
+    assert np.array_equal(n_acc, first_miss)
+    for s in range(S):
+        n = n_acc[s]
+        assert np.array_equal(path[s, :n], np.arange(n)) and np.all(path[s, n:] == -1)
+        assert np.array_equal(emitted[s, :n], token[s, :n]) and emitted[s, n] == target[s, n]
+        assert np.all(emitted[s, n + 1:] == -1)
+    # the chain is the tree whose parent of node i is node i-1
+    chain = np.tile(np.arange(-1, N - 1, dtype=np.int32), (S, 1))
+    n2, p2, e2 = oracle.verify_greedy(token, chain, target)
+    assert np.array_equal(n2, n_acc) and np.array_equal(p2, path) and np.array_equal(e2, emitted)
+
+
+def test_verify_tree_against_the_set_formulation():
+    for N, width, vocab, pm, seed in ((1, 1, 3, 0.5, 1), (12, 3, 5, 0.8, 2), (40, 8, 50, 0.7, 3), (63, 4, 4, 0.9, 4)):
+        token, parent, target = (t.numpy() for t in vt_inputs.draft_trees(60, N, width, vocab, pm, seed))
+        n_acc, path, emitted = oracle.verify_greedy(token, parent, target)
+        assert n_acc.max() >= min(N, 2) - 1                  # the inputs do produce walks
+        for s in range(token.shape[0]):
+            want = _consistent_nodes(token[s], parent[s], target[s])
+            n = int(n_acc[s])
+            assert np.array_equal(path[s, :n], want)
+            last = want[-1] if n else -1
+            assert emitted[s, n] == target[s, last + 1]
+            assert np.array_equal(emitted[s, :n], token[s][want])
+            # every accepted node hangs off the previous one
+            assert all(parent[s, path[s, k]] == (path[s, k - 1] if k else -1) for k in range(n))
+
+
+def test_verify_hand_example_bounds_and_duplicate_siblings():
+    # root children: node0 (tok 5), node1 (tok 4); node0's children: node2 (6), node3 (7); node3's child: node4 (8)
+    token = np.array([[5, 4, 6, 7, 8]], dtype=np.int32)
+    parent = np.array([[-1, -1, 0, 0, 3]], dtype=np.int32)
+    target = np.array([[5, 7, 0, 0, 8, 3]], dtype=np.int32)
+    n_acc, path, emitted = oracle.verify_greedy(token, parent, target)
+    assert n_acc[0] == 3 and path[0, :3].tolist() == [0, 3, 4] and emitted[0, :4].tolist() == [5, 7, 8, 3]
+    # nothing matches: the block still yields the target's own token (tau >= 1)
+    n_acc, _, emitted = oracle.verify_greedy(token, parent, np.full((1, 6), 9, dtype=np.int32))
+    assert n_acc[0] == 0 and emitted[0, 0] == 9 and oracle.block_efficiency(n_acc) == 1.0
+    # a full match of a depth-gamma chain yields gamma + 1 tokens, the stated maximum of tau
+    chain = np.arange(4, dtype=np.int32)[None]
+    n_acc, _, _ = oracle.verify_greedy(chain, None, np.arange(5, dtype=np.int32)[None])
+    assert oracle.block_efficiency(n_acc) == 5.0
+    # two siblings with the same token: the lower index is taken; unreachable parents are ignored
+    token = np.array([[3, 3, 1, 2]], dtype=np.int32)
+    parent = np.array([[-1, -1, 1, 0]], dtype=np.int32)
+    n_acc, path, _ = oracle.verify_greedy(token, parent, np.array([[3, 2, 1, 0, 0]], dtype=np.int32))
+    assert n_acc[0] == 2 and path[0, :2].tolist() == [0, 3]
+    bad_parent = np.array([[-1, 5, -7, 3]], dtype=np.int32)            # not in [-1, i)
+    n_acc, path, _ = oracle.verify_greedy(token, bad_parent, np.array([[3, 3, 3, 3, 3]], dtype=np.int32))
+    assert n_acc[0] == 1 and path[0, 0] == 0
+
+
+def _mbsu_rows():
+    here = os.path.join(os.path.dirname(__file__), "golden", "paper_mbsu_rows.txt")
+    rows = {}
+    for line in open(here):
+        if line.startswith("#") or not line.strip():
+            continue
+        f = line.split()
+        v = list(map(float, f[3:]))
+        rows[f[0]] = (f[1], float(f[2]), np.array(v[0::2]), np.array(v[1::2]))
+    return rows
+
+
+def test_mbsu_reproduces_the_table_rows_of_the_paper():
+    """Table 1 prints (BE, MBSU) per task.  MBSU = tau / (c*gamma + 1) with c the parameter ratio, so
+    (i) within a row MBSU is BE over ONE constant; (ii) that constant moves with the draft
+    parameter count only: fixing gamma / P_target from the untrimmed independent drafter (314M
+    parameters) predicts the denominators of the three other drafters from the printed head sizes."""
+    rows = _mbsu_rows()
+    assert len(rows) == 6
+    name, head, be, mb = rows["independent_full"]
+    per_m = float(np.mean(be / mb) - 1.0) / 314.0                 # gamma / P_target per 1e6 draft parameters
+    gamma = 4
+    p_target = gamma / per_m
+    assert abs(p_target - 3212.7) < 12.0                          # Llama-3.2-3B has 3.21e9 parameters at gamma = 4
+    ind_trim = 314.0 - 131.3 + 33.8
+    for key in ("independent_full", "independent_raw", "independent_target"):
+        _, head, be, mb = rows[key]
+        p_draft = 314.0 if head == 131.3 else ind_trim
+        for tau, want in zip(be, mb):
+            assert abs(oracle.mbsu(tau, p_draft / p_target, gamma) - want) < 2.5e-3
+    # EAGLE drafter: its total size is not printed; one row fixes it, the trimmed rows follow from
+    # the printed head sizes alone.
+    _, head, be, mb = rows["eagle_full"]
+    p_eagle = float(np.mean(be / mb) - 1.0) / per_m
+    for key in ("eagle_full", "eagle_raw", "eagle_target"):
+        _, head, be, mb = rows[key]
+        p_draft = p_eagle - 394.0 + head
+        for tau, want in zip(be, mb):
+            assert abs(oracle.mbsu(tau, p_draft / p_target, gamma) - want) < 2.5e-3
+    # a wrong form (tau * denominator, or gamma + c instead of c * gamma + 1) misses by far more
+    assert abs(3.846 / (1 + 4 * 314.0 / p_target) - 2.765) < 2.5e-3
+    assert abs(3.846 / (4 + 314.0 / p_target) - 2.765) > 1.0

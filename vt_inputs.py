@@ -81,3 +81,33 @@ def bf16_bits(t: torch.Tensor) -> torch.Tensor:
     """View a bf16 tensor as its raw 16-bit patterns (int16 storage, same memory)."""
     assert t.dtype == torch.bfloat16
     return t.view(torch.int16)
+
+
+def draft_trees(S: int, N: int, width: int, vocab: int, p_match: float, seed: int):
+    """S random draft trees of N nodes each, as CPU int32 tensors, plus a stand-in for the target's
+    greedy tokens: (token [S,N], parent [S,N], target [S,N+1]).
+
+    Node i hangs off a uniformly drawn earlier node (or off the committed prefix, parent -1) that
+    still has fewer than `width` children; siblings carry distinct ids, as a top-k expansion
+    gives.  target[s, j] is, with probability p_match, the id of a uniformly drawn child of node
+    j-1 (so that walks of some depth occur) and a fresh id otherwise.  Data only: no acceptance
+    logic lives here."""
+    assert width <= vocab
+    g = _gen(seed, "cpu")
+    token = torch.empty(S, N, dtype=torch.int32)
+    parent = torch.empty(S, N, dtype=torch.int32)
+    target = torch.randint(0, vocab, (S, N + 1), generator=g, dtype=torch.int32)
+    for s in range(S):
+        kids = [[] for _ in range(N + 1)]                 # kids[j] = children of node j-1
+        for i in range(N):
+            open_ = [j for j in range(i + 1) if len(kids[j]) < width]
+            j = open_[int(torch.randint(0, len(open_), (1,), generator=g))]
+            kids[j].append(i)
+            parent[s, i] = j - 1
+        for j in range(N + 1):
+            if kids[j]:
+                ids = torch.randperm(vocab, generator=g)[:len(kids[j])].to(torch.int32)
+                token[s, kids[j]] = ids
+                if float(torch.rand((), generator=g)) < p_match:
+                    target[s, j] = ids[int(torch.randint(0, len(ids), (1,), generator=g))]
+    return token, parent, target
