@@ -127,6 +127,36 @@ vt_status vt_select_minfreq(const uint32_t *counts, int32_t V, uint32_t min_coun
                             int32_t *inv_map, int32_t *k_out, void *ws, size_t ws_bytes, void *stream);
 
 /*
+ * Greedy verification of S drafted blocks (Section 4, Experiments: the target decodes greedily and a
+ * draft token is accepted only if it equals the target's token; the accept loop of Algorithm 2).
+ * All pointers are DEVICE pointers, row-major:
+ *   token  [S,N]   drafted ids, already full-vocabulary ids (after the index mapper);
+ *   parent [S,N]   parent node index, -1 = child of the last committed token; a node whose parent is
+ *                  not in [-1, i) is never reached.  NULL = chains (parent[i] = i - 1);
+ *   target [S,N+1] target[s,0] = the target's greedy token after the committed prefix,
+ *                  target[s,i+1] = its greedy token after the path that ends in node i.
+ * From the committed prefix the walk accepts the child of the current node that carries the
+ * target's token there (the lowest-indexed one if several do) until no child does.
+ *   n_accept [S]      accepted draft tokens per block;
+ *   path     [S,N]    accepted node indices, -1 beyond n_accept (may be NULL);
+ *   emitted  [S,N+1]  accepted tokens followed by the target's token at the last accepted node,
+ *                     -1 beyond (may be NULL); a block yields n_accept + 1 tokens;
+ *   tokens_total      DEVICE uint64 the call ADDS sum(n_accept + 1) to (may be NULL); divided by the
+ *                     number of blocks it is the block efficiency tau.
+ * Integer work: exact.  S = 0 is a no-op.  N < 1 or a NULL required pointer: VT_ERR_INVALID_ARG.
+ */
+vt_status vt_verify_greedy(const int32_t *token, const int32_t *parent, const int32_t *target, int32_t S,
+                           int32_t N, int32_t *n_accept, int32_t *path, int32_t *emitted,
+                           uint64_t *tokens_total, void *stream);
+
+/*
+ * Memory-bound speed-up of Section 4.1 (Performance Metrics): tau / (c * gamma + 1) with
+ * c = draft_params / target_params.  HOST arithmetic in fp64; NaN for arguments outside
+ * tau >= 0, draft_params >= 0, target_params > 0, gamma >= 0.
+ */
+double vt_mbsu(double tau, double draft_params, double target_params, int32_t gamma);
+
+/*
  * vt_select_topk without a workspace.  (The paper has no counterpart: this entry point exists for
  * the sake of callers, not of the method.)  Same result as vt_select_topk, for callers that cannot
  * allocate device memory or pass scratch along: code living inside another runtime's memory pool,

@@ -32,7 +32,7 @@ EXPORTS = (
     "vt_last_cuda_error",
     "vt_histogram", "vt_select_topk", "vt_build_vocab", "vt_build_vocab_host", "vt_trim_head",
     "vt_draft_head", "vt_draft_head_debug", "vt_draft_head_host", "vt_select_topk_static",
-    "vt_draft_head_overlapped", "vt_select_topp", "vt_select_minfreq",
+    "vt_draft_head_overlapped", "vt_select_topp", "vt_select_minfreq", "vt_verify_greedy", "vt_mbsu",
 )
 
 
@@ -67,6 +67,9 @@ def lib() -> ctypes.CDLL:
         L.vt_select_topk_static.argtypes = [c_void_p, c_int32, c_int32, c_void_p, c_void_p, c_void_p]
         L.vt_select_topp.argtypes = [c_void_p, c_int32, c_double, c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
         L.vt_select_minfreq.argtypes = [c_void_p, c_int32, c_uint32, c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
+        L.vt_verify_greedy.argtypes = [c_void_p, c_void_p, c_void_p, c_int32, c_int32, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]
+        L.vt_mbsu.argtypes = [c_double, c_double, c_double, c_int32]
+        L.vt_mbsu.restype = c_double
         L.vt_build_vocab.argtypes = [c_void_p, c_int64, c_int32, c_int32, c_void_p, c_void_p, c_void_p,
                                      c_size_t, c_void_p]
         L.vt_build_vocab_host.argtypes = L.vt_build_vocab.argtypes
@@ -186,6 +189,37 @@ def vt_select_topp(counts: torch.Tensor, p: float, ws: Workspace | None = None):
 def vt_select_minfreq(counts: torch.Tensor, min_count: int, ws: Workspace | None = None):
     """Minimum-frequency selection (Method section): returns (K device int32 [1], map [V], inv_map [V])."""
     return _select_cut(counts, ws, "vt_select_minfreq", c_uint32(int(min_count)))
+
+
+def vt_verify_greedy(token: torch.Tensor, parent: torch.Tensor | None, target: torch.Tensor,
+                     tokens_total: torch.Tensor | None = None):
+    """Greedy verification (Experiments section; Algorithm 2's accept loop) of S blocks.
+
+    token [S,N], parent [S,N] or None (chains), target [S,N+1], all int32 on the device.  Returns
+    (n_accept [S], path [S,N], emitted [S,N+1]); `tokens_total` (int64 [1], device) is added to."""
+    _dev(token, torch.int32, "token")
+    _dev(target, torch.int32, "target")
+    S, N = token.shape
+    if tuple(target.shape) != (S, N + 1):
+        raise ValueError("target must be [S, N+1]")
+    if parent is not None:
+        _dev(parent, torch.int32, "parent")
+        if tuple(parent.shape) != (S, N):
+            raise ValueError("parent must be [S, N]")
+    if tokens_total is not None:
+        _dev(tokens_total, torch.int64, "tokens_total")
+    n_accept = torch.empty(S, dtype=torch.int32, device=token.device)
+    path = torch.empty(S, N, dtype=torch.int32, device=token.device)
+    emitted = torch.empty(S, N + 1, dtype=torch.int32, device=token.device)
+    _check("vt_verify_greedy", lib().vt_verify_greedy(
+        _ptr(token), _ptr(parent) if parent is not None else None, _ptr(target), S, N, _ptr(n_accept),
+        _ptr(path), _ptr(emitted), _ptr(tokens_total) if tokens_total is not None else None, _stream()))
+    return n_accept, path, emitted
+
+
+def vt_mbsu(tau: float, draft_params: float, target_params: float, gamma: int) -> float:
+    """Memory-bound speed-up tau / (c*gamma + 1), c = draft_params / target_params (host arithmetic)."""
+    return float(lib().vt_mbsu(float(tau), float(draft_params), float(target_params), int(gamma)))
 
 
 def vt_select_topk_static(counts: torch.Tensor, K: int, out=None):

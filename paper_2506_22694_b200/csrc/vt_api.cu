@@ -4,6 +4,9 @@
 
 #include "vt_common.cuh"
 
+#include <cmath>
+#include <cstdint>
+
 namespace vt {
 
 static std::atomic<uint64_t> g_launches{0};
@@ -201,6 +204,22 @@ vt_status vt_select_topp(const uint32_t* counts, int32_t V, double p, int32_t* m
 vt_status vt_select_minfreq(const uint32_t* counts, int32_t V, uint32_t min_count, int32_t* map,
                             int32_t* inv_map, int32_t* k_out, void* ws, size_t ws_bytes, void* stream) {
     return select_cut_impl(counts, V, 1, 1.0, min_count, map, inv_map, k_out, ws, ws_bytes, stream);
+}
+
+vt_status vt_verify_greedy(const int32_t* token, const int32_t* parent, const int32_t* target, int32_t S,
+                           int32_t N, int32_t* n_accept, int32_t* path, int32_t* emitted,
+                           uint64_t* tokens_total, void* stream) {
+    if (S < 0 || N < 1 || N == INT32_MAX) return VT_ERR_INVALID_ARG;
+    if (S > 0 && (!token || !target || !n_accept)) return VT_ERR_INVALID_ARG;
+    return from_cuda(launch_verify_greedy(token, parent, target, S, N, n_accept, path, emitted,
+                                          reinterpret_cast<unsigned long long*>(tokens_total),
+                                          as_stream(stream)));
+}
+
+double vt_mbsu(double tau, double draft_params, double target_params, int32_t gamma) {
+    if (!(tau >= 0.0) || !(draft_params >= 0.0) || !(target_params > 0.0) || gamma < 0) return nan("");
+    const double c = draft_params / target_params;
+    return tau / (c * (double)gamma + 1.0);
 }
 
 vt_status vt_build_vocab(const int32_t* ids, int64_t n, int32_t V, int32_t K, int32_t* map,

@@ -86,3 +86,13 @@ def test_missing_library_fails_loudly(monkeypatch):
     monkeypatch.setattr(vt, "LIB_PATH", os.path.join(ROOT, "no_such_dir", "libvocabtrim.so"))
     with pytest.raises(RuntimeError, match="no fallback"):
         vt.lib()
+
+
+def test_mbsu_host_calculator_matches_a_table_cell_of_the_paper():
+    """Table 1, independent drafter (314M parameters, block size 4, 3.21e9-parameter target):
+    block efficiency 3.846 is printed with a memory-bound speed-up of 2.765."""
+    import math
+    import paper_2506_22694_b200 as vt
+    assert abs(vt.vt_mbsu(3.846, 314.0e6, 3212.7e6, 4) - 2.765) < 2.5e-3
+    assert vt.vt_mbsu(5.0, 0.0, 1.0, 4) == 5.0
+    assert math.isnan(vt.vt_mbsu(1.0, 1.0, 0.0, 4)) and math.isnan(vt.vt_mbsu(-1.0, 1.0, 1.0, 4))
