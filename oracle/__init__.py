@@ -256,3 +256,51 @@ def mbsu(tau: float, c: float, gamma: int) -> float:
     """Memory-bound speed-up tau / (c * gamma + 1), c = draft / target parameter ratio
     (Performance Metrics paragraph)."""
     return float(tau) / (float(c) * float(gamma) + 1.0)
+
+
+# ---- draft-tree construction.  The paper takes "draft trees construction ... following EAGLE-2"
+# (Settings) with depth 3, top-K = 8 and at most 32 draft tokens (60 in the depth ablation); the steps
+# below restate that published procedure.  Scores are cumulative log-probabilities kept in fp32, the
+# precision the GPU path keeps them in, because they decide integers (which nodes are taken).
+
+def _score_order(score, index):
+    """Order of preference: higher score first, lower node index on equal scores; NaN ranks last."""
+    s = np.where(np.isnan(score), -np.inf, score).astype(np.float32)
+    return np.lexsort((index, -s.astype(np.float64)))
+
+
+def tree_expand(cand_ids, cand_logprobs, frontier_nodes, pool_token, pool_parent, pool_score,
+                pool_base: int, n_front: int):
+    """One depth of the expansion.  Row b of cand_* holds the top-k ids / log-probs the head gave for
+    the node frontier_nodes[b] (None: the single row is the committed prefix, parent -1, score 0).
+    Every candidate becomes a pool node at pool_base + b*topk + j with
+    score = score(parent) + min(logprob, 0); the n_front best new nodes are the next frontier.
+    Mutates the pool arrays; returns the frontier's pool indices in order of preference."""
+    cand_ids = np.asarray(cand_ids, dtype=np.int32)
+    lp = np.asarray(cand_logprobs, dtype=np.float32)
+    B, topk = cand_ids.shape
+    for b in range(B):
+        par = -1 if frontier_nodes is None else int(frontier_nodes[b])
+        base_score = np.float32(0.0) if par < 0 else pool_score[par]
+        for j in range(topk):
+            node = pool_base + b * topk + j
+            pool_token[node] = cand_ids[b, j]
+            pool_parent[node] = par
+            step = lp[b, j] if np.isnan(lp[b, j]) else min(lp[b, j], np.float32(0.0))
+            pool_score[node] = np.float32(base_score + step)
+    new = np.arange(pool_base, pool_base + B * topk, dtype=np.int32)
+    order = _score_order(pool_score[new], new)
+    return new[order[:n_front]].copy()
+
+
+def tree_rerank(pool_token, pool_parent, pool_score, n: int, budget: int):
+    """Final selection: the `budget` best of the n pool nodes by cumulative score, listed in pool
+    order (parents precede children), parents renumbered into that list (-1 = committed prefix).
+    Returns (nodes, token, parent), each of length min(budget, n)."""
+    idx = np.arange(n, dtype=np.int32)
+    keep = np.sort(idx[_score_order(np.asarray(pool_score[:n], dtype=np.float32), idx)[:budget]])
+    pos = {int(node): k for k, node in enumerate(keep)}
+    token = np.array([pool_token[i] for i in keep], dtype=np.int32)
+    parent = np.array([-1 if pool_parent[i] < 0 else pos.get(int(pool_parent[i]), -2) for i in keep],
+                      dtype=np.int32)
+    return keep.astype(np.int32), token, parent

@@ -500,3 +500,87 @@ def test_mbsu_reproduces_the_table_rows_of_the_paper():
     # a wrong form (tau * denominator, or gamma + c instead of c * gamma + 1) misses by far more
     assert abs(3.846 / (1 + 4 * 314.0 / p_target) - 2.765) < 2.5e-3
     assert abs(3.846 / (4 + 314.0 / p_target) - 2.765) > 1.0
+
+
+# ---- draft-tree expansion and rerank (Settings: tree construction following EAGLE-2)
+
+def _grow(depth, topk, n_front, vocab, seed, tie_frac=0.0):
+    cap = topk + (depth - 1) * n_front * topk
+    tok = np.full(cap, -9, dtype=np.int32)
+    par = np.full(cap, -9, dtype=np.int32)
+    sc = np.full(cap, np.nan, dtype=np.float32)
+    steps = []
+    ids, lp = (t.numpy() for t in vt_inputs.head_candidates(1, topk, vocab, seed, tie_frac))
+    front = oracle.tree_expand(ids, lp, None, tok, par, sc, 0, n_front)
+    steps.append((ids, lp, None, 0, front))
+    base = topk
+    for dep in range(1, depth):
+        ids, lp = (t.numpy() for t in vt_inputs.head_candidates(len(front), topk, vocab, seed + dep, tie_frac))
+        nxt = oracle.tree_expand(ids, lp, front, tok, par, sc, base, n_front)
+        steps.append((ids, lp, front, base, nxt))
+        base += len(front) * topk
+        front = nxt
+    return tok, par, sc, base, steps
+
+
+def test_tree_scores_are_path_sums_and_frontier_is_the_brute_force_best():
+    for depth, topk, seed in ((3, 8, 1), (5, 10, 2), (2, 3, 3), (7, 4, 4)):
+        tok, par, sc, n, steps = _grow(depth, topk, topk, 1000, seed)
+        assert n == topk + (depth - 1) * topk * topk and not np.isnan(sc[:n]).any()
+        lp_of = {}
+        for ids, lp, front, base, nxt in steps:
+            B = ids.shape[0]
+            for b in range(B):
+                for j in range(topk):
+                    node = base + b * topk + j
+                    lp_of[node] = lp[b, j]
+                    assert tok[node] == ids[b, j] and par[node] == (-1 if front is None else front[b])
+            new = list(range(base, base + B * topk))
+            best = sorted(new, key=lambda i: (-float(sc[i]), i))[:len(nxt)]
+            assert best == nxt.tolist()
+        for i in range(n):                                   # cumulative score = sum over the path, root first
+            chain = []
+            j = i
+            while j >= 0:
+                chain.append(j)
+                j = par[j]
+            acc = np.float32(0.0)
+            for j in reversed(chain):
+                acc = np.float32(acc + lp_of[j])
+            assert acc == sc[i]
+            assert par[i] < i and (par[i] < 0 or sc[par[i]] >= sc[i])
+
+
+def test_tree_rerank_keeps_the_best_nodes_closed_under_parents():
+    for depth, topk, budget, seed, ties in ((3, 8, 32, 1, 0.0), (6, 10, 60, 2, 0.0), (4, 5, 17, 3, 0.8),
+                                            (2, 2, 100, 4, 0.5), (3, 4, 1, 5, 0.0)):
+        tok, par, sc, n, _ = _grow(depth, topk, topk, 500, seed, ties)
+        nodes, token, parent = oracle.tree_rerank(tok, par, sc, n, budget)
+        m = min(budget, n)
+        assert len(nodes) == m and np.all(np.diff(nodes) > 0)
+        brute = sorted(sorted(range(n), key=lambda i: (-float(sc[i]), i))[:m])
+        assert nodes.tolist() == brute
+        worst_kept = min(float(sc[i]) for i in nodes)
+        assert all(float(sc[i]) <= worst_kept for i in range(n) if i not in set(nodes.tolist()))
+        for k in range(m):                                   # parents are kept, precede their children, renumbered
+            assert token[k] == tok[nodes[k]]
+            if par[nodes[k]] < 0:
+                assert parent[k] == -1
+            else:
+                assert 0 <= parent[k] < k and nodes[parent[k]] == par[nodes[k]]
+
+
+def test_tree_hand_example_ties_positive_logprob_and_nan():
+    tok = np.zeros(6, dtype=np.int32); par = np.zeros(6, dtype=np.int32); sc = np.zeros(6, dtype=np.float32)
+    ids = np.array([[7, 9]], dtype=np.int32)
+    front = oracle.tree_expand(ids, np.array([[-0.5, -1.0]], dtype=np.float32), None, tok, par, sc, 0, 2)
+    assert front.tolist() == [0, 1] and sc[:2].tolist() == [-0.5, -1.0]
+    # children: of node 0: (-0.25, -2.0) -> -0.75, -2.5 ; of node 1: (+1e-7 clamps to 0, NaN) -> -1.0, NaN
+    lp = np.array([[-0.25, -2.0], [1e-7, np.nan]], dtype=np.float32)
+    front = oracle.tree_expand(np.array([[1, 2], [3, 4]], dtype=np.int32), lp, front, tok, par, sc, 2, 3)
+    assert sc[2] == np.float32(-0.75) and sc[3] == np.float32(-2.5) and sc[4] == np.float32(-1.0) and np.isnan(sc[5])
+    assert front.tolist() == [2, 4, 3]                        # NaN ranks last
+    assert par[2:6].tolist() == [0, 0, 1, 1] and tok[2:6].tolist() == [1, 2, 3, 4]
+    nodes, token, parent = oracle.tree_rerank(tok, par, sc, 6, 4)
+    # scores: -0.5, -1.0, -0.75, -2.5, -1.0, NaN : best four = 0, 2, then 1 before 4 on the tie
+    assert nodes.tolist() == [0, 1, 2, 4] and token.tolist() == [7, 9, 1, 3] and parent.tolist() == [-1, -1, 0, 1]

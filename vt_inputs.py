@@ -111,3 +111,19 @@ def draft_trees(S: int, N: int, width: int, vocab: int, p_match: float, seed: in
                 if float(torch.rand((), generator=g)) < p_match:
                     target[s, j] = ids[int(torch.randint(0, len(ids), (1,), generator=g))]
     return token, parent, target
+
+
+def head_candidates(B: int, topk: int, vocab: int, seed: int, tie_frac: float = 0.0):
+    """Stand-in for the head's per-row top-k output, as CPU tensors: ids int32 [B,topk] (distinct per
+    row) and log-probs fp32 [B,topk], descending per row and <= 0 (log of sorted Dirichlet-like
+    masses).  tie_frac > 0 rounds log-probs to a coarse grid so that equal scores occur."""
+    g = _gen(seed, "cpu")
+    ids = torch.stack([torch.randperm(vocab, generator=g)[:topk] for _ in range(B)]).to(torch.int32)
+    mass = torch.rand(B, topk + 1, generator=g, dtype=torch.float64) ** 3 + 1e-6
+    mass = mass / mass.sum(dim=1, keepdim=True)
+    lp = torch.log(mass[:, :topk]).sort(dim=1, descending=True).values.to(torch.float32)
+    if tie_frac > 0:
+        coarse = torch.round(lp * 2) / 2
+        pick = torch.rand(B, topk, generator=g) < tie_frac
+        lp = torch.where(pick, coarse, lp).sort(dim=1, descending=True).values
+    return ids, lp.clamp(max=0.0)
