@@ -127,6 +127,39 @@ vt_status vt_select_minfreq(const uint32_t *counts, int32_t V, uint32_t min_coun
                             int32_t *inv_map, int32_t *k_out, void *ws, size_t ws_bytes, void *stream);
 
 /*
+ * Draft-tree construction around the head.  Section 4.1 (Settings) adopts the draft-tree construction
+ * of EAGLE-2 with depth 3, top-K 8 and at most 32 draft tokens (60 in the depth ablation of the
+ * appendix).  The node pool is three caller-owned DEVICE arrays of pool_capacity entries: token id,
+ * parent node (-1 = the committed prefix) and cumulative log-probability (fp32).
+ *
+ * vt_tree_expand: one depth.  Row b of cand_ids / cand_logprobs (DEVICE, row stride ld, candidates in
+ * columns col0 .. col0+topk-1: the out_ids / out_logprobs of vt_draft_head fit with ld = 1+topk,
+ * col0 = 1) holds the head's top-k for the node frontier_nodes[b] (DEVICE [B], entries < pool_base;
+ * NULL, with B = 1, for the first depth whose single row is the committed prefix).  Candidate j of
+ * row b becomes node pool_base + b*topk + j with score(parent) + min(logprob, 0) (fp32 addition;
+ * score of the prefix is 0).  next_frontier (DEVICE [n_front]) receives the n_front best NEW nodes,
+ * best first: higher score, then lower node index; NaN scores rank last.  Hidden row r of the
+ * next depth belongs to next_frontier[r].
+ *
+ * vt_tree_rerank: the final draft.  Of pool nodes [0,n) the `budget` best by the same order are
+ * kept and listed in pool order (parents before children): out_nodes (pool index), out_token,
+ * out_parent (position in this list, -1 = committed prefix), each DEVICE [budget], padded with -1
+ * when n < budget.  Scores never rise along a path, so a kept node's parent is kept (-2 would mark
+ * a parent that is not).  The three outputs are the token / parent inputs of vt_verify_greedy.
+ *
+ * Limits: B*topk and n at most VT_TREE_MAX_NODES (VT_ERR_UNSUPPORTED beyond); n_front <= B*topk and
+ * pool_base + B*topk <= pool_capacity (VT_ERR_INVALID_ARG).  Integer results are exact.
+ */
+#define VT_TREE_MAX_NODES 4096
+vt_status vt_tree_expand(const int32_t *cand_ids, const float *cand_logprobs, int32_t B, int32_t topk,
+                         int32_t ld, int32_t col0, const int32_t *frontier_nodes, int32_t *pool_token,
+                         int32_t *pool_parent, float *pool_score, int32_t pool_base, int32_t pool_capacity,
+                         int32_t n_front, int32_t *next_frontier, void *stream);
+vt_status vt_tree_rerank(const int32_t *pool_token, const int32_t *pool_parent, const float *pool_score,
+                         int32_t n, int32_t budget, int32_t *out_nodes, int32_t *out_token, int32_t *out_parent,
+                         void *stream);
+
+/*
  * Greedy verification of S drafted blocks (Section 4, Experiments: the target decodes greedily and a
  * draft token is accepted only if it equals the target's token; the accept loop of Algorithm 2).
  * All pointers are DEVICE pointers, row-major:

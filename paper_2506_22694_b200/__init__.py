@@ -32,7 +32,7 @@ EXPORTS = (
     "vt_last_cuda_error",
     "vt_histogram", "vt_select_topk", "vt_build_vocab", "vt_build_vocab_host", "vt_trim_head",
     "vt_draft_head", "vt_draft_head_debug", "vt_draft_head_host", "vt_select_topk_static",
-    "vt_draft_head_overlapped", "vt_select_topp", "vt_select_minfreq", "vt_verify_greedy", "vt_mbsu",
+    "vt_draft_head_overlapped", "vt_select_topp", "vt_select_minfreq", "vt_verify_greedy", "vt_mbsu", "vt_tree_expand", "vt_tree_rerank",
 )
 
 
@@ -70,6 +70,8 @@ def lib() -> ctypes.CDLL:
         L.vt_verify_greedy.argtypes = [c_void_p, c_void_p, c_void_p, c_int32, c_int32, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]
         L.vt_mbsu.argtypes = [c_double, c_double, c_double, c_int32]
         L.vt_mbsu.restype = c_double
+        L.vt_tree_expand.argtypes = [c_void_p, c_void_p, c_int32, c_int32, c_int32, c_int32, c_void_p, c_void_p, c_void_p, c_void_p, c_int32, c_int32, c_int32, c_void_p, c_void_p]
+        L.vt_tree_rerank.argtypes = [c_void_p, c_void_p, c_void_p, c_int32, c_int32, c_void_p, c_void_p, c_void_p, c_void_p]
         L.vt_build_vocab.argtypes = [c_void_p, c_int64, c_int32, c_int32, c_void_p, c_void_p, c_void_p,
                                      c_size_t, c_void_p]
         L.vt_build_vocab_host.argtypes = L.vt_build_vocab.argtypes
@@ -189,6 +191,45 @@ def vt_select_topp(counts: torch.Tensor, p: float, ws: Workspace | None = None):
 def vt_select_minfreq(counts: torch.Tensor, min_count: int, ws: Workspace | None = None):
     """Minimum-frequency selection (Method section): returns (K device int32 [1], map [V], inv_map [V])."""
     return _select_cut(counts, ws, "vt_select_minfreq", c_uint32(int(min_count)))
+
+
+def tree_pool(capacity: int, device="cuda"):
+    """Caller-owned node pool of vt_tree_expand / vt_tree_rerank: (token, parent, score) tensors."""
+    return (torch.empty(capacity, dtype=torch.int32, device=device),
+            torch.empty(capacity, dtype=torch.int32, device=device),
+            torch.empty(capacity, dtype=torch.float32, device=device))
+
+
+def vt_tree_expand(cand_ids: torch.Tensor, cand_logprobs: torch.Tensor, frontier_nodes: torch.Tensor | None,
+                   pool, pool_base: int, n_front: int, col0: int = 0) -> torch.Tensor:
+    """One depth of the draft-tree expansion (Settings).  cand_* are [B, col0+topk] device tensors (the
+    head's outputs with col0=1); returns the next frontier's pool indices [n_front], best first."""
+    _dev(cand_ids, torch.int32, "cand_ids")
+    _dev(cand_logprobs, torch.float32, "cand_logprobs")
+    B, ld = cand_ids.shape
+    if tuple(cand_logprobs.shape) != (B, ld):
+        raise ValueError("cand_ids and cand_logprobs must have the same shape")
+    tok, par, sc = pool
+    _dev(tok, torch.int32, "pool token"), _dev(par, torch.int32, "pool parent"), _dev(sc, torch.float32, "pool score")
+    if frontier_nodes is not None and _dev(frontier_nodes, torch.int32, "frontier_nodes").numel() != B:
+        raise ValueError("frontier_nodes must have B entries")
+    nxt = torch.empty(n_front, dtype=torch.int32, device=cand_ids.device)
+    _check("vt_tree_expand", lib().vt_tree_expand(
+        _ptr(cand_ids), _ptr(cand_logprobs), B, ld - col0, ld, col0, _ptr(frontier_nodes), _ptr(tok), _ptr(par),
+        _ptr(sc), pool_base, min(tok.numel(), par.numel(), sc.numel()), n_front, _ptr(nxt), _stream()))
+    return nxt
+
+
+def vt_tree_rerank(pool, n: int, budget: int):
+    """Final draft of the tree (Settings): returns (nodes, token, parent), each int32 [budget]."""
+    tok, par, sc = pool
+    _dev(tok, torch.int32, "pool token"), _dev(par, torch.int32, "pool parent"), _dev(sc, torch.float32, "pool score")
+    if n > min(tok.numel(), par.numel(), sc.numel()):
+        raise ValueError("n exceeds the pool")
+    outs = [torch.empty(budget, dtype=torch.int32, device=tok.device) for _ in range(3)]
+    _check("vt_tree_rerank", lib().vt_tree_rerank(_ptr(tok), _ptr(par), _ptr(sc), n, budget, _ptr(outs[0]),
+                                                  _ptr(outs[1]), _ptr(outs[2]), _stream()))
+    return tuple(outs)
 
 
 def vt_verify_greedy(token: torch.Tensor, parent: torch.Tensor | None, target: torch.Tensor,

@@ -206,6 +206,33 @@ vt_status vt_select_minfreq(const uint32_t* counts, int32_t V, uint32_t min_coun
     return select_cut_impl(counts, V, 1, 1.0, min_count, map, inv_map, k_out, ws, ws_bytes, stream);
 }
 
+vt_status vt_tree_expand(const int32_t* cand_ids, const float* cand_logprobs, int32_t B, int32_t topk,
+                         int32_t ld, int32_t col0, const int32_t* frontier_nodes, int32_t* pool_token,
+                         int32_t* pool_parent, float* pool_score, int32_t pool_base, int32_t pool_capacity,
+                         int32_t n_front, int32_t* next_frontier, void* stream) {
+    if (!cand_ids || !cand_logprobs || !pool_token || !pool_parent || !pool_score || !next_frontier)
+        return VT_ERR_INVALID_ARG;
+    if (B < 1 || topk < 1 || col0 < 0 || ld < col0 + topk || pool_base < 0 || n_front < 1) return VT_ERR_INVALID_ARG;
+    if (!frontier_nodes && B != 1) return VT_ERR_INVALID_ARG;
+    const int64_t n_new = (int64_t)B * topk;
+    if (n_new > tree_max_nodes()) return VT_ERR_UNSUPPORTED;
+    if (n_front > n_new || pool_base + n_new > pool_capacity) return VT_ERR_INVALID_ARG;
+    return from_cuda(launch_tree_expand(cand_ids, cand_logprobs, B, topk, ld, col0, frontier_nodes, pool_token,
+                                        pool_parent, pool_score, pool_base, n_front, next_frontier,
+                                        as_stream(stream)));
+}
+
+vt_status vt_tree_rerank(const int32_t* pool_token, const int32_t* pool_parent, const float* pool_score,
+                         int32_t n, int32_t budget, int32_t* out_nodes, int32_t* out_token, int32_t* out_parent,
+                         void* stream) {
+    if (!pool_token || !pool_parent || !pool_score || !out_nodes || !out_token || !out_parent)
+        return VT_ERR_INVALID_ARG;
+    if (n < 1 || budget < 1) return VT_ERR_INVALID_ARG;
+    if (n > tree_max_nodes()) return VT_ERR_UNSUPPORTED;
+    return from_cuda(launch_tree_rerank(pool_token, pool_parent, pool_score, n, budget, out_nodes, out_token,
+                                        out_parent, as_stream(stream)));
+}
+
 vt_status vt_verify_greedy(const int32_t* token, const int32_t* parent, const int32_t* target, int32_t S,
                            int32_t N, int32_t* n_accept, int32_t* path, int32_t* emitted,
                            uint64_t* tokens_total, void* stream) {

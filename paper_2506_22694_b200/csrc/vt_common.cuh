@@ -47,6 +47,15 @@ cudaError_t launch_verify_greedy(const int32_t* token, const int32_t* parent, co
                                  int32_t N, int32_t* n_accept, int32_t* path, int32_t* emitted,
                                  unsigned long long* tokens_total, cudaStream_t st);
 
+int tree_max_nodes();
+cudaError_t launch_tree_expand(const int32_t* cand_ids, const float* cand_lp, int32_t B, int32_t topk, int32_t ld,
+                               int32_t col0, const int32_t* frontier, int32_t* pool_token, int32_t* pool_parent,
+                               float* pool_score, int32_t pool_base, int32_t n_front, int32_t* next_frontier,
+                               cudaStream_t st);
+cudaError_t launch_tree_rerank(const int32_t* pool_token, const int32_t* pool_parent, const float* pool_score,
+                               int32_t n, int32_t budget, int32_t* out_nodes, int32_t* out_token,
+                               int32_t* out_parent, cudaStream_t st);
+
 cudaError_t launch_gather_rows(const uint16_t* W_full, const int32_t* map, uint16_t* W_trim,
                                int32_t V, int32_t K, int32_t d, Ctrl* ctrl, cudaStream_t s);
 
