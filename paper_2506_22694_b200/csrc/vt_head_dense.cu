@@ -2,21 +2,28 @@
 // and runs on the 5th-generation tensor cores (Algorithm 2, lines 5-6, with many sequences and
 // tree nodes drafted at once).
 //
-//   D[b, j] = sum_i h[b, i] * W_trim[j, i]      M = hidden rows (128 per MMA, two M tiles),
-//                                               N = 128 vocabulary rows per tile, K-loop over d
+//   D[b, j] = sum_i h[b, i] * W_trim[j, i]      M = hidden rows (the TMEM lanes), N = vocabulary rows
+//                                               of a tile (TMEM columns), K-loop over d in 64-column steps
 //
-// One persistent CTA per SM walks vocabulary tiles.  Warp 0 feeds a 4-stage shared-memory ring with
-// TMA tensor copies (128-byte swizzle, no multicast): per 64-column step the two halves of h and one
-// tile of W_trim.  One thread of warp 1 issues tcgen05.mma (bf16 x bf16 -> fp32) with the operands
-// described in place by shared-memory descriptors and the accumulators in tensor memory: two
-// accumulator stages of 2 x 128 columns, so the epilogue of tile t overlaps the MMAs of tile t+1.
-// Eight epilogue warps read the accumulators back with tcgen05.ld -- TMEM lane = hidden row, so every
-// thread owns one hidden row and walks its 128 logits of the tile, 16 at a time: running max / sum-exp of
-// z = logit / T_b, Gumbel-max candidate from the caller's uniforms, and a sorted top-k list kept in
-// registers.  Logits never go to HBM.  Per CTA and hidden row one record goes to scratch; a second
-// small kernel (one warp per hidden row) merges the records, applies the index mapper and writes
-// the outputs.  Every wait is bounded; on expiry the CTA raises VT_FLAG_TIMEOUT and leaves after
-// releasing its tensor memory.
+// B <= 128: one persistent CTA per SM walks vocabulary tiles (M = 128, tcgen05.mma.cta_group::1).
+// B  > 128: the two CTAs of a cluster act as one MMA of M = 256 (cta_group::2).  Each CTA stages its
+// own 128 hidden rows and HALF of the tile's vocabulary rows; the tensor cores of both SMs read the
+// two halves of the B operand from both shared memories.  Per SM and flop this halves the operand
+// bytes staged and read compared with two M tiles in one CTA, which is what bounded that form.
+//
+// Warp 0 feeds a shared-memory ring with TMA tensor copies (128-byte swizzle, no multicast); in a pair
+// both CTAs' copies count their bytes on the leader's barrier.  One thread of warp 1 (of the leader)
+// issues the MMAs (bf16 x bf16 -> fp32) with the operands described in place by shared-memory
+// descriptors and the accumulators in tensor memory: two accumulator stages of up to 256 columns, so
+// the epilogue of tile t overlaps the MMAs of tile t+1.  tcgen05.commit releases ring stages and
+// publishes accumulators (to both CTAs of a pair).  Eight epilogue warps read the accumulators back
+// with tcgen05.ld -- TMEM lane = hidden row; warps 0-3 take the first half of a tile's columns, warps
+// 4-7 the second -- 16 columns at a time: running max / sum-exp of z = logit / T_b, Gumbel-max candidate
+// from the caller's uniforms, and a sorted top-k list kept in registers.  Logits never go to HBM.  The
+// two column halves of a row are merged through shared memory; per CTA (pair) and hidden row one
+// record goes to scratch; a second small kernel (one warp per hidden row) merges the records,
+// applies the index mapper and writes the outputs.  Every wait is bounded; on expiry the CTA raises
+// VT_FLAG_TIMEOUT and leaves after releasing its tensor memory.
 #include <cuda.h>
 
 #include <mutex>
@@ -28,19 +35,18 @@ namespace vt {
 
 namespace {
 
-constexpr int kBM = 128;                  // hidden rows per MMA (TMEM lanes)
-constexpr int kBN = 128;                  // vocabulary rows per tile (TMEM columns per accumulator)
+constexpr int kBM = 128;                  // hidden rows per CTA (TMEM lanes)
+constexpr int kMaxBN = 256;               // vocabulary rows per tile at most (TMEM columns per accumulator)
 constexpr int kBK = 64;                   // columns of d per ring stage: 128 bytes, one swizzle row
-constexpr int kStages = 4;
-constexpr int kTileBytes = kBM * kBK * 2; // 16 KB: one operand tile of a stage
-constexpr int kStageBytes = 3 * kTileBytes;
+constexpr int kMaxStages = 8;
+constexpr int kHTileBytes = kBM * kBK * 2; // 16 KB: the hidden-row operand of a stage
 constexpr int kEpiWarps = 8;
-constexpr int kThreads = (2 + kEpiWarps) * 32;
+constexpr int kThreads = (2 + kEpiWarps) * 32;   // TMA producer, MMA issuer, 8 epilogue warps
 constexpr int kCh = 16;                   // accumulator columns per epilogue step (keeps the row state in registers)
-constexpr int kTmemCols = 512;            // 2 accumulator stages x 2 M tiles x 128 columns
+constexpr int kTmemCols = 512;            // 2 accumulator stages x kMaxBN columns
 constexpr int kMaxTopk = 16;              // top-k list lives in registers
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
-constexpr size_t kDynSmem = (size_t)kStages * kStageBytes + 1024;   // + slack to align to 1024 bytes
+constexpr size_t kRingBudget = 225 * 1024;   // ring bytes at most (227 KB per CTA less alignment slack and statics)
 
 // ---- PTX wrappers ----------------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -76,10 +82,24 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* b, uint32_t parity, volatile
         if (global_ns() - t0 > kWaitLimitNs) { *abort_flag = 1; return false; }
     }
 }
-// Same, called by all 32 lanes of a warp: the outcome is voted on so the lanes never part ways
-// before a warp-collective instruction.
+// Same, called by all 32 lanes of a warp that expects to wait long (a whole tile of MMAs): lane 0
+// polls with pauses -- 256 spinning threads cost issue slots and power the tensor pipe wants -- then
+// every lane observes the completed phase itself.  The outcome is voted on so the lanes never part
+// ways before a warp-collective instruction.
 __device__ __forceinline__ bool mbar_wait_warp(uint64_t* b, uint32_t parity, volatile int* abort_flag) {
-    return __all_sync(0xffffffffu, mbar_wait(b, parity, abort_flag));
+    bool ok = true;
+    if ((threadIdx.x & 31) == 0 && !mbar_try(b, parity)) {
+        const unsigned long long t0 = global_ns();
+        for (;;) {
+            __nanosleep(128);
+            if (mbar_try(b, parity)) break;
+            if (*abort_flag) { ok = false; break; }
+            if (global_ns() - t0 > kWaitLimitNs) { *abort_flag = 1; ok = false; break; }
+        }
+    }
+    ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+    if (ok) ok = mbar_try(b, parity) || mbar_wait(b, parity, abort_flag);
+    return __all_sync(0xffffffffu, ok);
 }
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm, int x, int y, uint64_t* bar) {
     asm volatile(
@@ -121,268 +141,402 @@ __host__ __device__ constexpr uint32_t make_idesc(int M, int N) {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
 }
 
+// Programmatic dependent launch: let the next launch on the stream become resident / wait until the
+// work this launch depends on has completed and its writes are visible (no-ops in a plain launch).
+__device__ __forceinline__ void griddep_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+// ---- CTA-pair forms (cta_group::2): two CTAs of a cluster act as one 256-row MMA ---------------------
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// shared::cluster address of the same variable in CTA `rank` of this cluster
+__device__ __forceinline__ uint32_t mapa_u32(uint32_t addr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// tensor copy into THIS CTA's shared memory whose bytes are counted on a barrier of either CTA of the pair
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* tm, int x, int y, uint32_t bar_cluster) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(tm), "r"(bar_cluster), "r"(x), "r"(y) : "memory");
+}
+// arrives on the barrier at this shared-memory offset in both CTAs once the MMAs issued so far are done
+__device__ __forceinline__ void tc_commit_pair(uint64_t* bar) {
+    asm volatile(
+        "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+        ::"r"(smem_u32(bar)), "h"((uint16_t)3) : "memory");
+}
+// D[tmem of both CTAs] (+)= A * B^T, 256 x N x 16: each CTA supplies 128 rows of A and N/2 rows of B
+__device__ __forceinline__ void tc_mma_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t acc) {
+    const uint32_t z = 0;
+    asm volatile(
+        "{ .reg .pred p; setp.ne.b32 p, %4, 0;"
+        " tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5, %5, %5, %5, %5}, p; }"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(acc), "r"(z) : "memory");
+}
+
 struct DenseGeo {
-    int n_tiles;      // vocabulary tiles of kBN rows
+    int n_tiles;      // vocabulary tiles of bn rows
     int n_kc;         // ring steps per tile: ceil(d / kBK)
-    int n_mt;         // M tiles: 1 (B <= 128) or 2
+    int bn;           // vocabulary rows per tile (per CTA pair when paired); a multiple of 32, <= kMaxBN
+    int n_stages;     // ring depth
+    int stage_bytes;  // bytes one CTA stages per step: hidden rows + its share of the vocabulary rows
+    int n_groups;     // CTAs (or CTA pairs) walking the tiles round-robin
 };
 
-// KT: capacity of the register top-k list (8 or kMaxTopk)
+// Per-thread state of one hidden row over the columns the thread has seen.
 template <int KT>
+struct RowState {
+    float m, s;               // running max and sum of exp(z - m)
+    float gb_s, gb_z;         // best Gumbel score and its z
+    int gb_j;
+    float tv[KT];             // top-k list at the END of the arrays (slots KT-topk .. KT-1, descending)
+    int tj[KT];               // behind +inf sentinels: the insertion threshold is always slot KT-1
+};
+
+// Insert (cv, cj) into the sorted list with selects only; equal values keep the entry already there.
+template <int KT>
+__device__ __forceinline__ void list_insert(float (&tv)[KT], int (&tj)[KT], float cv, int cj) {
+#pragma unroll
+    for (int p = 0; p < KT; ++p) {
+        const bool sw = cv > tv[p];
+        const float ov = tv[p];
+        const int oj = tj[p];
+        tv[p] = sw ? cv : ov;
+        tj[p] = sw ? cj : oj;
+        cv = sw ? ov : cv;
+        cj = sw ? oj : cj;
+    }
+}
+
+// KT: capacity of the register top-k list (8 or kMaxTopk).  PAIR: two CTAs of a cluster form one MMA.
+template <int KT, bool PAIR>
 __global__ void __launch_bounds__(kThreads, 1)
 k_head_dense(const HeadArgs a, Ctrl* ctrl, float* __restrict__ recs, const DenseGeo geo,
              const __grid_constant__ CUtensorMap tm_h, const __grid_constant__ CUtensorMap tm_w) {
     extern __shared__ uint8_t s_dyn[];
-    __shared__ uint64_t s_full[kStages], s_empty[kStages], s_acc_full[2], s_acc_empty[2];
+    __shared__ uint64_t s_full[kMaxStages], s_empty[kMaxStages], s_acc_full[2], s_acc_empty[2];
     __shared__ uint32_t s_tmem_base;
     __shared__ int s_abort;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    // identical in both CTAs of a pair: the MMA addresses the peer's operands by the leader's offsets
     uint8_t* ring = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(s_dyn) + 1023) & ~(uintptr_t)1023);
     const uint32_t ring_u32 = smem_u32(ring);
     const int B = a.B, K = a.K, topk = a.topk;
+    const uint32_t rank = PAIR ? cluster_ctarank() : 0u;          // 0 = leader: issues the MMAs, owns the full barriers
+    const int group = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
+    const int bn = geo.bn, n_stages = geo.n_stages;
+    const int w_rows = PAIR ? bn / 2 : bn;                         // vocabulary rows this CTA stages per step
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kStages; ++s) { mbar_init(&s_full[s], 1); mbar_init(&s_empty[s], 1); }
-        for (int p = 0; p < 2; ++p) { mbar_init(&s_acc_full[p], 1); mbar_init(&s_acc_empty[p], kEpiWarps); }
+        for (int s = 0; s < kMaxStages; ++s) { mbar_init(&s_full[s], 1); mbar_init(&s_empty[s], 1); }
+        for (int p = 0; p < 2; ++p) { mbar_init(&s_acc_full[p], 1); mbar_init(&s_acc_empty[p], (PAIR ? 2 : 1) * kEpiWarps); }
         s_abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 1) {   // tensor memory: the whole SM's 512 columns (one CTA per SM by shared-memory size)
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                     ::"r"(smem_u32(&s_tmem_base)), "r"((uint32_t)kTmemCols) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    if (warp == 1) {   // tensor memory: all 512 columns of the SM (one CTA per SM by shared-memory size)
+        if (PAIR) {
+            asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
+                         ::"r"(smem_u32(&s_tmem_base)), "r"((uint32_t)kTmemCols) : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+        } else {
+            asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                         ::"r"(smem_u32(&s_tmem_base)), "r"((uint32_t)kTmemCols) : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        }
     }
     tc_fence_before();
-    __syncthreads();
+    if (PAIR) cluster_sync_all(); else __syncthreads();           // barriers initialised in both CTAs before any signal
     tc_fence_after();
     const uint32_t tmem_base = s_tmem_base;
     volatile int* abort_flag = &s_abort;
+    griddep_launch_dependents();                                  // the merge kernel may take its seats
 
     if (warp == 0) {
-        // ================= TMA producer ================================================================
+        // ================= TMA producer (both CTAs of a pair) ==========================================
         if (lane == 0) {
-            int s = 0, issued = 0;
-            uint32_t ph = 0;
-            const uint32_t bytes = (uint32_t)(geo.n_mt + 1) * kTileBytes;
-            bool alive = true;
-            for (int tile = blockIdx.x; tile < geo.n_tiles && alive; tile += gridDim.x) {
-                for (int kc = 0; kc < geo.n_kc; ++kc) {
-                    if (issued >= kStages && !mbar_wait(&s_empty[s], ph ^ 1, abort_flag)) { alive = false; break; }
-                    const uint32_t base = ring_u32 + (uint32_t)s * kStageBytes;
-                    mbar_expect_tx(&s_full[s], bytes);
-                    tma_load_2d(base, &tm_h, kc * kBK, 0, &s_full[s]);
-                    if (geo.n_mt == 2) tma_load_2d(base + kTileBytes, &tm_h, kc * kBK, kBM, &s_full[s]);
-                    tma_load_2d(base + 2 * kTileBytes, &tm_w, kc * kBK, tile * kBN, &s_full[s]);
-                    ++issued;
-                    if (++s == kStages) { s = 0; ph ^= 1; }
-                }
+            // fills are numbered g = 0 .. total-1 over (tile, step in d); fill g uses stage g % n_stages
+            const int my_tiles = (geo.n_tiles - group + geo.n_groups - 1) / geo.n_groups;
+            const int total = my_tiles * geo.n_kc;
+            const uint32_t bytes = (uint32_t)(PAIR ? 2 : 1) * (uint32_t)geo.stage_bytes;
+            const uint32_t full0 = PAIR ? mapa_u32(smem_u32(&s_full[0]), 0) : 0u;      // the leader's full barriers
+            auto load_w = [&](int g) {
+                const int s = g % n_stages, tile = group + (g / geo.n_kc) * geo.n_groups, kc = g % geo.n_kc;
+                const uint32_t dst = ring_u32 + (uint32_t)s * (uint32_t)geo.stage_bytes + kHTileBytes;
+                if (PAIR) tma_load_2d_pair(dst, &tm_w, kc * kBK, tile * bn + (int)rank * w_rows, full0 + (uint32_t)(s * sizeof(uint64_t)));
+                else tma_load_2d(dst, &tm_w, kc * kBK, tile * bn, &s_full[s]);
+            };
+            auto load_h = [&](int g) {
+                const int s = g % n_stages, kc = g % geo.n_kc;
+                const uint32_t dst = ring_u32 + (uint32_t)s * (uint32_t)geo.stage_bytes;
+                if (PAIR) tma_load_2d_pair(dst, &tm_h, kc * kBK, (int)rank * kBM, full0 + (uint32_t)(s * sizeof(uint64_t)));
+                else tma_load_2d(dst, &tm_h, kc * kBK, 0, &s_full[s]);
+            };
+            // The weights are static: the first ring of them is requested before the work this launch
+            // depends on has finished; everything that work may have produced is touched after the wait.
+            const int pre = min(n_stages, total);
+            for (int g = 0; g < pre; ++g) {
+                if (rank == 0) mbar_expect_tx(&s_full[g], bytes);
+                load_w(g);
             }
-            if (!alive || *abort_flag) {
-                // drain: every stage that was filled must have landed before the CTA may leave
-                const int back = min(issued, kStages);
-                for (int i = 1; i <= back; ++i) {
-                    const int it = issued - i;
-                    const unsigned long long t0 = global_ns();
-                    while (!mbar_try(&s_full[it % kStages], (uint32_t)((it / kStages) & 1)) &&
-                           global_ns() - t0 < kWaitLimitNs) {}
-                }
+            griddep_wait();
+            for (int g = 0; g < pre; ++g) load_h(g);
+            int done = pre;
+            for (int g = pre; g < total; ++g, ++done) {
+                const int s = g % n_stages;
+                if (!mbar_wait(&s_empty[s], (uint32_t)((g / n_stages) & 1) ^ 1u, abort_flag)) break;
+                if (rank == 0) mbar_expect_tx(&s_full[s], bytes);
+                load_h(g);
+                load_w(g);
+            }
+            if (done == total && !*abort_flag) {
+                // every fill consumed: all copies have landed and every commit aimed at this CTA's
+                // barriers has arrived before the CTA may leave
+                for (int g = max(0, total - n_stages); g < total; ++g)
+                    if (!mbar_wait(&s_empty[g % n_stages], (uint32_t)((g / n_stages) & 1), abort_flag)) break;
+            }
+            if (*abort_flag) {
+                // something timed out: give copies still in flight time to land before the memory goes away
+                const unsigned long long t0 = global_ns();
+                while (global_ns() - t0 < 200000ull) {}
             }
         }
     } else if (warp == 1) {
-        // ================= MMA issuer ==================================================================
-        if (lane == 0) {
-            const uint32_t idesc = make_idesc(kBM, kBN);
+        // ================= MMA issuer (leader CTA only) ================================================
+        if (lane == 0 && rank == 0) {
+            const uint32_t idesc = make_idesc(PAIR ? 2 * kBM : kBM, bn);
             int s = 0, t_local = 0;
             uint32_t ph = 0;
             bool alive = true;
-            for (int tile = blockIdx.x; tile < geo.n_tiles && alive; tile += gridDim.x, ++t_local) {
+            for (int tile = group; tile < geo.n_tiles && alive; tile += geo.n_groups, ++t_local) {
                 const int as = t_local & 1;
                 const uint32_t use = (uint32_t)(t_local >> 1);
-                if (t_local >= 2 && !mbar_wait(&s_acc_empty[as], (use - 1) & 1, abort_flag)) break;
+                if (t_local >= 2 && !mbar_wait(&s_acc_empty[as], (use - 1) & 1, abort_flag)) { alive = false; break; }
                 tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)(as * kMaxBN);
                 for (int kc = 0; kc < geo.n_kc; ++kc) {
                     if (!mbar_wait(&s_full[s], ph, abort_flag)) { alive = false; break; }
                     tc_fence_after();
-                    const uint32_t base = ring_u32 + (uint32_t)s * kStageBytes;
+                    const uint32_t base = ring_u32 + (uint32_t)s * (uint32_t)geo.stage_bytes;
 #pragma unroll
-                    for (int mt = 0; mt < 2; ++mt) {
-                        if (mt < geo.n_mt) {
-                            const uint32_t d_tmem = tmem_base + (uint32_t)(as * 2 * kBN + mt * kBN);
-#pragma unroll
-                            for (int k = 0; k < kBK / 16; ++k)
-                                tc_mma(d_tmem, make_desc(base + mt * kTileBytes + k * 32),
-                                       make_desc(base + 2 * kTileBytes + k * 32), idesc, (kc | k) != 0 ? 1u : 0u);
-                        }
+                    for (int k = 0; k < kBK / 16; ++k) {
+                        const uint64_t da = make_desc(base + k * 32), db = make_desc(base + kHTileBytes + k * 32);
+                        if (PAIR) tc_mma_pair(d_tmem, da, db, idesc, (kc | k) != 0 ? 1u : 0u);
+                        else tc_mma(d_tmem, da, db, idesc, (kc | k) != 0 ? 1u : 0u);
                     }
-                    tc_commit(&s_empty[s]);                  // the stage is free once these MMAs have read it
-                    if (++s == kStages) { s = 0; ph ^= 1; }
+                    // the stage is free (in both CTAs) once these MMAs have read it
+                    if (PAIR) tc_commit_pair(&s_empty[s]); else tc_commit(&s_empty[s]);
+                    if (++s == n_stages) { s = 0; ph ^= 1; }
                 }
-                if (alive) tc_commit(&s_acc_full[as]);       // accumulators of this tile are complete
+                if (alive) {                                      // accumulators of this tile are complete
+                    if (PAIR) tc_commit_pair(&s_acc_full[as]); else tc_commit(&s_acc_full[as]);
+                }
             }
+            // the last accumulators have been read (every arrival of the peer has landed) before leaving
+            for (int t = max(0, t_local - 2); t < t_local && alive; ++t)
+                if (!mbar_wait(&s_acc_empty[t & 1], (uint32_t)((t >> 1) & 1), abort_flag)) break;
         }
     } else {
-        // ================= epilogue warps: one hidden row per thread ===================================
+        // ================= epilogue warps: one hidden row and one half of the tile's columns per thread =
         const int ew = warp - 2;
         const int quad = warp & 3;                            // TMEM lanes this warp may read
-        const int mt = ew >> 2;
-        const int b = mt * kBM + quad * 32 + lane;
-        const bool row_live = b < B && mt < geo.n_mt;
+        const int half = ew >> 2;                             // which half of the tile's columns
+        const int cols_half = bn / 2, n_ch = cols_half / kCh;
+        const int b = (int)rank * kBM + quad * 32 + lane;
+        const bool row_live = b < B;
+        griddep_wait();                                       // temp, uniforms and the record scratch belong to earlier work until here
         float invT = 1.f;
         if (row_live) {
             const float T = a.temp[b];
             invT = (T > 0.f && T < CUDART_INF_F) ? 1.f / T : CUDART_NAN_F;
         }
-        float st_m = -CUDART_INF_F, st_s = 0.f, gb_s = -CUDART_INF_F, gb_z = 0.f, thr = -CUDART_INF_F;
-        int gb_j = -1;
-        float tv[KT];
-        int tj[KT];
+        RowState<KT> st;
+        st.m = -CUDART_INF_F; st.s = 0.f; st.gb_s = -CUDART_INF_F; st.gb_z = 0.f; st.gb_j = -1;
+        float thr = -CUDART_INF_F;
 #pragma unroll
-        // the list sits at the END of the arrays (slots KT-topk .. KT-1, descending), behind +inf
-        // sentinels: its last entry -- the insertion threshold -- is then always slot KT-1, a register
-        for (int i = 0; i < KT; ++i) { tv[i] = (i < KT - topk) ? CUDART_INF_F : -CUDART_INF_F; tj[i] = -1; }
+        for (int i = 0; i < KT; ++i) { st.tv[i] = (i < KT - topk) ? CUDART_INF_F : -CUDART_INF_F; st.tj[i] = -1; }
         const bool vec_u = a.uniforms && ((K & 3) == 0);
         const bool use_u = row_live && a.uniforms != nullptr;
+        const uint32_t acc_empty_bar = PAIR ? mapa_u32(smem_u32(&s_acc_empty[0]), 0) : 0u;
         float u[kCh];
 #pragma unroll
         for (int i = 0; i < kCh; ++i) u[i] = 0.5f;
         int t_local = 0;
-        for (int tile = blockIdx.x; tile < geo.n_tiles; tile += gridDim.x, ++t_local) {
+        for (int tile = group; tile < geo.n_tiles; tile += geo.n_groups, ++t_local) {
             const int as = t_local & 1;
             if (!mbar_wait_warp(&s_acc_full[as], (uint32_t)((t_local >> 1) & 1), abort_flag)) break;
             tc_fence_after();
-            if (mt < geo.n_mt) {
+            const int jt = tile * bn + half * cols_half;      // first vocabulary row of this thread's columns
 #pragma unroll 1
-                for (int ch = 0; ch < kBN / kCh; ++ch) {
-                    const int j0 = tile * kBN + ch * kCh;
-                    // this chunk's uniforms are requested first (they are needed last), and the next
-                    // chunk's line is pulled into L2 meanwhile
-                    if (use_u && j0 < K) {
-                        const float* up = a.uniforms + (size_t)b * K + j0;
-                        if (vec_u && j0 + kCh <= K) {
+            for (int ch = 0; ch < n_ch; ++ch) {
+                const int j0 = jt + ch * kCh;
+                // this chunk's uniforms are requested first (they are needed last), and a later
+                // chunk's line is pulled into L2 meanwhile
+                if (use_u && j0 < K) {
+                    const float* up = a.uniforms + (size_t)b * K + j0;
+                    if (vec_u && j0 + kCh <= K) {
 #pragma unroll
-                            for (int i = 0; i < kCh / 4; ++i) {
-                                const float4 q = __ldg(reinterpret_cast<const float4*>(up) + i);
-                                u[4 * i] = q.x; u[4 * i + 1] = q.y; u[4 * i + 2] = q.z; u[4 * i + 3] = q.w;
-                            }
-                        } else {
-#pragma unroll
-                            for (int i = 0; i < kCh; ++i) u[i] = (j0 + i < K) ? __ldg(up + i) : 0.5f;
+                        for (int i = 0; i < kCh / 4; ++i) {
+                            const float4 q = __ldg(reinterpret_cast<const float4*>(up) + i);
+                            u[4 * i] = q.x; u[4 * i + 1] = q.y; u[4 * i + 2] = q.z; u[4 * i + 3] = q.w;
                         }
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < kCh; ++i) u[i] = (j0 + i < K) ? __ldg(up + i) : 0.5f;
                     }
-                    const int jn = (ch + 2 < kBN / kCh) ? j0 + 2 * kCh : (tile + (int)gridDim.x) * kBN;
-                    if (use_u && jn < K && (ch & 1) == 0)
-                        asm volatile("prefetch.global.L2 [%0];" ::"l"(a.uniforms + (size_t)b * K + jn));
-                    uint32_t r[kCh];
-                    tc_ld16(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(as * 2 * kBN + mt * kBN + ch * kCh), r);
-                    // Warp-uniform from here on (j0 and K are): rows that do not exist simply carry nv = 0,
-                    // i.e. columns of -inf, so the warp votes below always see all 32 lanes.
-                    if (j0 < K) {
-                        const int nv = row_live ? min(kCh, K - j0) : 0;
-                        float z[kCh];
-                        float cmax = -CUDART_INF_F;
+                }
+                const int jn = (ch + 2 < n_ch) ? j0 + 2 * kCh : jt + geo.n_groups * bn;
+                if (use_u && jn < K && (ch & 1) == 0)
+                    asm volatile("prefetch.global.L2 [%0];" ::"l"(a.uniforms + (size_t)b * K + jn));
+                uint32_t r[kCh];
+                tc_ld16(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(as * kMaxBN + half * cols_half + ch * kCh), r);
+                // Warp-uniform from here on (j0 and K are): rows that do not exist simply carry nv = 0,
+                // i.e. columns of -inf, so the warp votes below always see all 32 lanes.
+                if (j0 < K) {
+                    const int nv = row_live ? min(kCh, K - j0) : 0;
+                    float z[kCh];
+                    float cmax = -CUDART_INF_F;
+#pragma unroll
+                    for (int i = 0; i < kCh; ++i) {
+                        z[i] = (i < nv) ? __uint_as_float(r[i]) * invT : -CUDART_INF_F;
+                        cmax = fmaxf(cmax, z[i]);
+                    }
+                    if (a.dbg_logits && row_live) {
+#pragma unroll
+                        for (int i = 0; i < kCh; ++i)
+                            if (i < nv) a.dbg_logits[(size_t)b * K + j0 + i] = __uint_as_float(r[i]);
+                    }
+                    // running max / sum-exp: one rescale per chunk, independent exponentials
+                    const float m_new = fmaxf(st.m, cmax);
+                    const float m_ref = (m_new == -CUDART_INF_F) ? 0.f : m_new;
+                    float acc = 0.f;
+#pragma unroll
+                    for (int i = 0; i < kCh; ++i) acc += __expf(z[i] - m_ref);
+                    st.s = st.s * __expf(st.m - m_ref) + acc;
+                    st.m = m_new;
+                    if (a.uniforms) {
 #pragma unroll
                         for (int i = 0; i < kCh; ++i) {
-                            z[i] = (i < nv) ? __uint_as_float(r[i]) * invT : -CUDART_INF_F;
-                            cmax = fmaxf(cmax, z[i]);
+                            // g = -log(-log u): -log u from a short series in 1-u near 1 (where the fast
+                            // logarithm's absolute error would dominate), fast logarithms elsewhere
+                            const float uc = fminf(fmaxf(u[i], 0x1p-24f), 1.f - 0x1p-24f);
+                            const float t = 1.f - uc;
+                            const float lp = t * (1.f + t * (0.5f + t * (0.33333334f + t * (0.25f + t * 0.2f))));
+                            const float L = uc > 0.95f ? lp : -__logf(uc);
+                            const float sc = z[i] - __logf(L);
+                            const bool win = sc > st.gb_s;            // invalid columns carry z = -inf
+                            st.gb_s = win ? sc : st.gb_s;
+                            st.gb_j = win ? j0 + i : st.gb_j;
+                            st.gb_z = win ? z[i] : st.gb_z;
                         }
-                        if (a.dbg_logits && row_live) {
+                    }
+                    // top-k: pull the chunk's maxima out in descending order while they beat the list's
+                    // last entry.  The loop is warp-uniform (it runs while any row of the warp still has
+                    // a candidate) and everything inside is select-based: one row's insertions never
+                    // make the other 31 rows branch.
+                    float mx = z[0];
+                    int mi = 0;
 #pragma unroll
-                            for (int i = 0; i < kCh; ++i)
-                                if (i < nv) a.dbg_logits[(size_t)b * K + j0 + i] = __uint_as_float(r[i]);
+                    for (int i = 1; i < kCh; ++i) {
+                        const bool gt = z[i] > mx;                    // strict: ties keep the lower column
+                        mx = gt ? z[i] : mx;
+                        mi = gt ? i : mi;
+                    }
+                    while (__any_sync(0xffffffffu, mx > thr)) {
+                        const bool take = mx > thr;
+                        list_insert<KT>(st.tv, st.tj, take ? mx : -CUDART_INF_F, j0 + mi);
+                        thr = st.tj[KT - 1] >= 0 ? st.tv[KT - 1] : -CUDART_INF_F;   // a threshold only once the list is full
+                        // drop the extracted element, find the next maximum
+                        float nmx = -CUDART_INF_F;
+                        int nmi = 0;
+#pragma unroll
+                        for (int i = 0; i < kCh; ++i) {
+                            z[i] = (take && i == mi) ? -CUDART_INF_F : z[i];
+                            const bool gt = z[i] > nmx;
+                            nmx = gt ? z[i] : nmx;
+                            nmi = gt ? i : nmi;
                         }
-                        // running max / sum-exp: one rescale per chunk, independent exponentials
-                        const float m_new = fmaxf(st_m, cmax);
-                        const float m_ref = (m_new == -CUDART_INF_F) ? 0.f : m_new;
-                        float acc = 0.f;
-#pragma unroll
-                        for (int i = 0; i < kCh; ++i) acc += __expf(z[i] - m_ref);
-                        st_s = st_s * __expf(st_m - m_ref) + acc;
-                        st_m = m_new;
-                        if (a.uniforms) {
-#pragma unroll
-                            for (int i = 0; i < kCh; ++i) {
-                                // g = -log(-log u): -log u from a short series in 1-u near 1 (where the fast
-                                // logarithm's absolute error would dominate), fast logarithms elsewhere
-                                const float uc = fminf(fmaxf(u[i], 0x1p-24f), 1.f - 0x1p-24f);
-                                const float t = 1.f - uc;
-                                const float lp = t * (1.f + t * (0.5f + t * (0.33333334f + t * (0.25f + t * 0.2f))));
-                                const float L = uc > 0.95f ? lp : -__logf(uc);
-                                const float sc = z[i] - __logf(L);
-                                const bool win = sc > gb_s;               // invalid columns carry z = -inf
-                                gb_s = win ? sc : gb_s;
-                                gb_j = win ? j0 + i : gb_j;
-                                gb_z = win ? z[i] : gb_z;
-                            }
-                        }
-                        // top-k: pull the chunk's maxima out in descending order while they beat the list's
-                        // last entry.  The loop is warp-uniform (it runs while any row of the warp still has
-                        // a candidate) and everything inside is select-based: one row's insertions never
-                        // make the other 31 rows branch.
-                        float mx = z[0];
-                        int mi = 0;
-#pragma unroll
-                        for (int i = 1; i < kCh; ++i) {
-                            const bool gt = z[i] > mx;                    // strict: ties keep the lower column
-                            mx = gt ? z[i] : mx;
-                            mi = gt ? i : mi;
-                        }
-                        while (__any_sync(0xffffffffu, mx > thr)) {
-                            const bool take = mx > thr;
-                            float cv = take ? mx : -CUDART_INF_F;
-                            int cj = j0 + mi;
-#pragma unroll
-                            for (int p = 0; p < KT; ++p) {                // the +inf sentinels in front never move
-                                const bool sw = cv > tv[p];               // equal values keep the lower index first
-                                const float ov = tv[p];
-                                const int oj = tj[p];
-                                tv[p] = sw ? cv : ov;
-                                tj[p] = sw ? cj : oj;
-                                cv = sw ? ov : cv;
-                                cj = sw ? oj : cj;
-                            }
-                            thr = tj[KT - 1] >= 0 ? tv[KT - 1] : -CUDART_INF_F;   // a threshold only once the list is full
-                            // drop the extracted element, find the next maximum
-                            float nmx = -CUDART_INF_F;
-                            int nmi = 0;
-#pragma unroll
-                            for (int i = 0; i < kCh; ++i) {
-                                z[i] = (take && i == mi) ? -CUDART_INF_F : z[i];
-                                const bool gt = z[i] > nmx;
-                                nmx = gt ? z[i] : nmx;
-                                nmi = gt ? i : nmi;
-                            }
-                            mx = nmx;
-                            mi = nmi;
-                        }
+                        mx = nmx;
+                        mi = nmi;
                     }
                 }
             }
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(&s_acc_empty[as]);
+            if (lane == 0) {
+                if (PAIR) mbar_arrive_cluster(acc_empty_bar + (uint32_t)(as * sizeof(uint64_t)));
+                else mbar_arrive(&s_acc_empty[as]);
+            }
         }
-        // ---- this CTA's record of hidden row b ---------------------------------------------------------
-        if (row_live && !*abort_flag) {
+        // ---- the two column halves of a row meet in shared memory (the ring is idle by now: the last
+        // accumulators were complete, so every MMA has read its operands and every copy has landed) ----
+        float* xch = reinterpret_cast<float*>(ring);
+        const int slot = quad * 32 + lane;                    // row within the CTA
+        const bool ok = !*abort_flag;
+        if (half == 1 && ok) {
+            float* x = xch + slot;                            // field-major: conflict-free
+            x[0 * kBM] = st.m; x[1 * kBM] = st.s; x[2 * kBM] = st.gb_s; x[3 * kBM] = __int_as_float(st.gb_j); x[4 * kBM] = st.gb_z;
+#pragma unroll
+            for (int p = 0; p < KT; ++p) { x[(5 + p) * kBM] = st.tv[p]; x[(5 + KT + p) * kBM] = __int_as_float(st.tj[p]); }
+        }
+        asm volatile("bar.sync 1, %0;" ::"n"(kEpiWarps * 32) : "memory");
+        if (half == 0 && ok && row_live) {
+            const float* x = xch + slot;
+            lse_merge(st.m, st.s, x[0 * kBM], x[1 * kBM]);
+            const float os = x[2 * kBM];
+            const int oj = __float_as_int(x[3 * kBM]);
+            if (better(os, oj, st.gb_s, st.gb_j) && oj >= 0) { st.gb_s = os; st.gb_j = oj; st.gb_z = x[4 * kBM]; }
+#pragma unroll
+            for (int p = 0; p < KT; ++p) {
+                // entries of the other half: equal values must still order by index, so compare keys
+                float cv = x[(5 + p) * kBM];
+                int cj = __float_as_int(x[(5 + KT + p) * kBM]);
+                if (p < KT - topk) continue;                  // its sentinels
+#pragma unroll
+                for (int q = 0; q < KT; ++q) {
+                    const bool sw = key64(cv, cj) > key64(st.tv[q], st.tj[q]) && q >= KT - topk;
+                    const float ov = st.tv[q];
+                    const int oj2 = st.tj[q];
+                    st.tv[q] = sw ? cv : ov;
+                    st.tj[q] = sw ? cj : oj2;
+                    cv = sw ? ov : cv;
+                    cj = sw ? oj2 : cj;
+                }
+            }
+            // ---- this CTA's record of hidden row b ---------------------------------------------------------
             int* irecs = reinterpret_cast<int*>(recs);
-            const int c = blockIdx.x;
-            recs[rec_at(b, 0, topk) + c] = st_m;
-            recs[rec_at(b, 1, topk) + c] = st_s;
-            recs[rec_at(b, 2, topk) + c] = gb_s;
-            irecs[rec_at(b, 3, topk) + c] = gb_j;
-            recs[rec_at(b, 4, topk) + c] = gb_z;
+            const int c = group;
+            recs[rec_at(b, 0, topk) + c] = st.m;
+            recs[rec_at(b, 1, topk) + c] = st.s;
+            recs[rec_at(b, 2, topk) + c] = st.gb_s;
+            irecs[rec_at(b, 3, topk) + c] = st.gb_j;
+            recs[rec_at(b, 4, topk) + c] = st.gb_z;
 #pragma unroll
             for (int p = 0; p < KT; ++p)
                 if (p >= KT - topk) {
-                    recs[rec_at(b, 5 + p - (KT - topk), topk) + c] = tv[p];
-                    irecs[rec_at(b, 5 + topk + p - (KT - topk), topk) + c] = tj[p];
+                    recs[rec_at(b, 5 + p - (KT - topk), topk) + c] = st.tv[p];
+                    irecs[rec_at(b, 5 + topk + p - (KT - topk), topk) + c] = st.tj[p];
                 }
         }
     }
     tc_fence_before();
-    __syncthreads();
+    __syncwarp();                                                 // lanes of the single-thread roles rejoin their warps
+    if (PAIR) cluster_sync_all(); else __syncthreads();           // nobody leaves while its peer may still signal it
     if (warp == 1) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)kTmemCols) : "memory");
+        if (PAIR) asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)kTmemCols) : "memory");
+        else asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)kTmemCols) : "memory");
     }
     if (threadIdx.x == 0 && s_abort) atomicOr(&ctrl->flags, (uint32_t)VT_FLAG_TIMEOUT);
 }
@@ -392,6 +546,8 @@ __global__ void __launch_bounds__(32)
 k_head_merge(const HeadArgs a, Ctrl* ctrl, const float* __restrict__ recs, int G) {
     __shared__ float s_stage[kMergeStageWords];
     const int b = blockIdx.x;
+    griddep_launch_dependents();                                  // the next step may start fetching its weights
+    griddep_wait();                                               // the records are complete
     const float T = a.temp[b];
     const bool row_ok = (T > 0.f) && (T < CUDART_INF_F);
     merge_records(a.map, a.out_ids, a.out_logprobs, a.dbg_lse, a.topk, a.uniforms != nullptr, ctrl, recs, b, row_ok, G,
@@ -430,6 +586,56 @@ bool encode_map(CUtensorMap* tm, const void* base, int rows, int cols, int box_r
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Tile width: the vocabulary is dealt to `groups` CTAs (pairs) in tiles of bn rows; the slowest group
+// works ceil(tiles / groups) * bn rows.  Smallest such makespan wins, the wider tile on equal terms
+// (fewer re-reads of the hidden rows).
+DenseGeo make_geo(int32_t K, int32_t d, bool pair, int max_groups) {
+    DenseGeo g{};
+    long best = -1;
+    for (int bn = kMaxBN; bn >= 32; bn -= 32) {
+        const long tiles = (K + bn - 1) / bn;
+        const long span = ((tiles + max_groups - 1) / max_groups) * bn;
+        if (best < 0 || span < best) { best = span; g.bn = bn; }
+    }
+    g.n_tiles = (K + g.bn - 1) / g.bn;
+    g.n_kc = (d + kBK - 1) / kBK;
+    g.n_groups = g.n_tiles < max_groups ? g.n_tiles : max_groups;
+    g.stage_bytes = kHTileBytes + (pair ? g.bn / 2 : g.bn) * kBK * 2;
+    g.n_stages = (int)(kRingBudget / (size_t)g.stage_bytes);
+    if (g.n_stages > kMaxStages) g.n_stages = kMaxStages;
+    return g;
+}
+
+template <int KT, bool PAIR>
+cudaError_t launch_variant(const HeadArgs& a, Ctrl* ctrl, float* recs, const DenseGeo& geo, const CUtensorMap& tm_h,
+                           const CUtensorMap& tm_w, cudaStream_t s) {
+    static int attr_done[64] = {0};
+    const size_t smem = (size_t)geo.n_stages * geo.stage_bytes + 1024;   // + slack to align the ring to 1024 bytes
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev < 0 || dev >= 64 || !attr_done[dev]) {
+        cudaError_t e = cudaFuncSetAttribute(k_head_dense<KT, PAIR>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             (int)(kRingBudget + 1024));
+        if (e != cudaSuccess) return e;
+        if (dev >= 0 && dev < 64) attr_done[dev] = 1;
+    }
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3((unsigned)(PAIR ? 2 * geo.n_groups : geo.n_groups));
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute at[2];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = PAIR ? 2 : 1;
+    at[0].val.clusterDim.y = 1;
+    at[0].val.clusterDim.z = 1;
+    at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = a.overlap ? 2 : 1;
+    return cudaLaunchKernelEx(&cfg, k_head_dense<KT, PAIR>, a, ctrl, recs, geo, tm_h, tm_w);
+}
+
 }  // namespace
 
 bool head_dense_supported(int32_t B, int32_t K, int32_t d) {
@@ -445,33 +651,33 @@ size_t head_dense_scratch_bytes(int32_t B, int32_t K, int32_t topk) {
 
 cudaError_t launch_head_dense(const HeadArgs& a, Ctrl* ctrl, uint8_t* scratch, cudaStream_t s) {
     if (!head_dense_supported(a.B, a.K, a.d) || !head_dense_topk_ok(a.topk)) return cudaErrorInvalidValue;
+    const bool pair = a.B > kBM;                       // more than one MMA's worth of hidden rows: CTA pairs
+    int max_groups = pair ? num_sms() / 2 : num_sms();
+    if (max_groups > kMaxGrid) max_groups = kMaxGrid;
+    if (max_groups < 1) return cudaErrorInvalidValue;
+    const DenseGeo geo = make_geo(a.K, a.d, pair, max_groups);
     CUtensorMap tm_h, tm_w;
-    if (!encode_map(&tm_h, a.h, a.B, a.d, kBM) || !encode_map(&tm_w, a.W, a.K, a.d, kBN)) return cudaErrorInvalidValue;
-    DenseGeo geo{};
-    geo.n_tiles = (a.K + kBN - 1) / kBN;
-    geo.n_kc = (a.d + kBK - 1) / kBK;
-    geo.n_mt = a.B > kBM ? 2 : 1;
-    int grid = num_sms();
-    if (grid > kMaxGrid) grid = kMaxGrid;
-    if (grid > geo.n_tiles) grid = geo.n_tiles;
-    static int attr_done[64] = {0};
-    int dev = 0;
-    cudaGetDevice(&dev);
-    if (dev < 0 || dev >= 64 || !attr_done[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(k_head_dense<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kDynSmem);
-        if (e != cudaSuccess) return e;
-        e = cudaFuncSetAttribute(k_head_dense<kMaxTopk>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kDynSmem);
-        if (e != cudaSuccess) return e;
-        if (dev >= 0 && dev < 64) attr_done[dev] = 1;
-    }
+    if (!encode_map(&tm_h, a.h, a.B, a.d, kBM) || !encode_map(&tm_w, a.W, a.K, a.d, pair ? geo.bn / 2 : geo.bn))
+        return cudaErrorInvalidValue;
     float* recs = reinterpret_cast<float*>(scratch);
-    if (a.topk <= 8) k_head_dense<8><<<grid, kThreads, kDynSmem, s>>>(a, ctrl, recs, geo, tm_h, tm_w);
-    else k_head_dense<kMaxTopk><<<grid, kThreads, kDynSmem, s>>>(a, ctrl, recs, geo, tm_h, tm_w);
-    cudaError_t e = cudaGetLastError();
+    cudaError_t e;
+    if (a.topk <= 8) e = pair ? launch_variant<8, true>(a, ctrl, recs, geo, tm_h, tm_w, s)
+                              : launch_variant<8, false>(a, ctrl, recs, geo, tm_h, tm_w, s);
+    else e = pair ? launch_variant<kMaxTopk, true>(a, ctrl, recs, geo, tm_h, tm_w, s)
+                  : launch_variant<kMaxTopk, false>(a, ctrl, recs, geo, tm_h, tm_w, s);
     if (e != cudaSuccess) return e;
-    k_head_merge<<<a.B, 32, 0, s>>>(a, ctrl, recs, grid);
+    // the merge always follows its own producer closely: it takes its seats early and waits on the device
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3((unsigned)a.B);
+    cfg.blockDim = dim3(32);
+    cfg.stream = s;
+    cudaLaunchAttribute at{};
+    at.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at.val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = &at;
+    cfg.numAttrs = 1;
     count_launch(2);
-    return cudaGetLastError();
+    return cudaLaunchKernelEx(&cfg, k_head_merge, a, ctrl, static_cast<const float*>(recs), geo.n_groups);
 }
 
 }  // namespace vt
