@@ -349,6 +349,10 @@ def extras(vt, dev, peak_gbs):
         vb["build_vocab_K%d_gtok_s" % K] = n / (ms_b * 1e-3) / 1e9
     ms_s = timed(lambda: vt.vt_select_topk(counts, 32768, ws=ws), reps=20)
     vb["select_topk_K32768_us"] = ms_s * 1e3
+    ms_p = timed(lambda: vt.vt_select_topp(counts, 0.99, ws=ws), reps=20)
+    vb["select_topp_p0.99_us"] = ms_p * 1e3
+    ms_f = timed(lambda: vt.vt_select_minfreq(counts, 100, ws=ws), reps=20)
+    vb["select_minfreq_100_us"] = ms_f * 1e3
     del ids
     torch.cuda.empty_cache()
     W_full = vt_inputs.gaussian_bf16((V, 4096), 0.02, seed=1006, device=dev)
@@ -359,7 +363,35 @@ def extras(vt, dev, peak_gbs):
     vb["trim_head_gbs"] = 2 * 32768 * 4096 * 2 / (ms_g * 1e-3) / 1e9
     vb["trim_head_frac_of_measured"] = vb["trim_head_gbs"] / peak_gbs
     out["vocab_build"] = vb
+    out["draft_block"] = draft_block_case(vt, dev, timed)
     return out
+
+
+def draft_block_case(vt, dev, timed):
+    """The on-chip select steps around the head in a drafting block, at the paper's tree settings
+    (depth 3, top-8, 32 draft tokens): three expansions + the rerank of one tree, and the greedy
+    verification of 64 such trees.  Latency-bound single-CTA / warp-per-sequence kernels."""
+    topk, depth, budget = 8, 3, 32
+    cands = [vt_inputs.head_candidates(1 if dep == 0 else topk, topk, V, seed=1010 + dep) for dep in range(depth)]
+    cands = [(i.to(dev), l.to(dev)) for i, l in cands]
+    cap = topk + (depth - 1) * topk * topk
+    pool = vt.tree_pool(cap, dev)
+
+    def build_tree():
+        front, base = None, 0
+        for ids_, lp_ in cands:
+            front = vt.vt_tree_expand(ids_, lp_, front, pool, base, topk)
+            base += ids_.shape[0] * topk
+        return vt.vt_tree_rerank(pool, base, budget)
+
+    ms_t = timed(build_tree, reps=200, warm=10)
+    tok, par, tgt = vt_inputs.draft_trees(64, budget, topk, V, 0.7, seed=1011)
+    tok, par, tgt = tok.to(dev), par.to(dev), tgt.to(dev)
+    total = torch.zeros(1, dtype=torch.int64, device=dev)
+    ms_v = timed(lambda: vt.vt_verify_greedy(tok, par, tgt, tokens_total=total), reps=200, warm=10)
+    return {"workload": "tree depth 3 / top-8 / 32 draft tokens; verification of 64 trees",
+            "tree_3_expansions_plus_rerank_us": ms_t * 1e3, "launches_per_tree": depth + 1,
+            "verify_64_trees_us": ms_v * 1e3}
 
 
 DENSE = dict(d=4096, K=32768, B=256, topk=8)                   # BASELINE config 4 (batched serving)
