@@ -45,7 +45,7 @@ FALLBACK_HBM_GBS = 6650.0
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the head kernel on the headline
 # workload, from the ncu capture summarised under profiles/ (None until a capture exists).
-NCU_TRAFFIC_BYTES = {"k_head_stream": 205_400_000, "k_hist_hot": None}
+NCU_TRAFFIC_BYTES = {"k_head_stream": 206_000_000, "k_hist_hot": None}
 
 
 def measured_peaks():
