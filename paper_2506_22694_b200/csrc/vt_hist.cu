@@ -146,13 +146,24 @@ k_hist_pick(const uint32_t* __restrict__ sample, int32_t V, int32_t H, uint2* __
     __syncthreads();
     {   // most bins were sampled a handful of times: count those in registers, one atomic per warp
         uint32_t small[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-        for (int v = threadIdx.x; v < V; v += kThreads) {
-            const uint32_t c = min(sample[v], (uint32_t)(kPickBins - 1));
-            if (c < 8) {
+        // eight loads in flight per thread: one CTA walking 128K counts one load at a time is all latency
+        for (int v0 = threadIdx.x; v0 < V; v0 += kThreads * 8) {
+            uint32_t cs[8];
 #pragma unroll
-                for (int k = 0; k < 8; ++k) small[k] += (c == (uint32_t)k);
-            } else {
-                atomicAdd(&s_hist[c], 1u);
+            for (int q = 0; q < 8; ++q) {
+                const int v = v0 + q * kThreads;
+                cs[q] = v < V ? __ldg(sample + v) : 0xffffffffu;
+            }
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+                if (cs[q] == 0xffffffffu) continue;                     // past the end (a count never gets there)
+                const uint32_t c = min(cs[q], (uint32_t)(kPickBins - 1));
+                if (c < 8) {
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) small[k] += (c == (uint32_t)k);
+                } else {
+                    atomicAdd(&s_hist[c], 1u);
+                }
             }
         }
 #pragma unroll
@@ -174,12 +185,22 @@ k_hist_pick(const uint32_t* __restrict__ sample, int32_t V, int32_t H, uint2* __
     __syncthreads();
     const uint32_t quota = (uint32_t)H - s_definite;
     // pass A: one coalesced load per 32 ids, the membership words come out of warp ballots
-    for (int w = warp; w < T32; w += kThreads / 32) {
-        const int v = w * 32 + lane;
-        const uint32_t c = v < V ? min(sample[v], (uint32_t)(kPickBins - 1)) : 0u;
-        const uint32_t def = __ballot_sync(0xffffffffu, v < V && c >= tau);
-        const uint32_t tie = __ballot_sync(0xffffffffu, v < V && c + 1 == tau);
-        if (lane == 0) s_tbl[w] = make_uint2(def, tie);
+    for (int w0 = warp; w0 < T32; w0 += (kThreads / 32) * 8) {          // again eight loads in flight
+        uint32_t cs[8];
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            const int v = (w0 + q * (kThreads / 32)) * 32 + lane;
+            cs[q] = v < V ? min(__ldg(sample + v), (uint32_t)(kPickBins - 1)) : 0xffffffffu;
+        }
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            const int w = w0 + q * (kThreads / 32);
+            if (w >= T32) break;                                        // warp-uniform
+            const bool in = cs[q] != 0xffffffffu;
+            const uint32_t def = __ballot_sync(0xffffffffu, in && cs[q] >= tau);
+            const uint32_t tie = __ballot_sync(0xffffffffu, in && cs[q] + 1 == tau);
+            if (lane == 0) s_tbl[w] = make_uint2(def, tie);
+        }
     }
     __syncthreads();
     // pass B: admit ties in id order while the quota lasts; every thread owns wpt consecutive words
