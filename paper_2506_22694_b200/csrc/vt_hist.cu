@@ -8,8 +8,8 @@
 //     hottest bins that fit (about 49.8 K of them), and the main pass keeps those in shared
 //     memory; the rare cold tokens go to L2 with one red.global each.  The hot set only steers
 //     traffic: counts are exact whichever bins were picked.
-//       hot lookup: table[id >> 5] = {32-bit membership word, slot of its first member};
-//       slot = base + popc(word & below(id)), one 8-byte shared load per token.
+//       hot lookup: entry[id >> 4] = {16 membership bits, 16-bit slot of the group's first member};
+//       slot = base + popc(bits & below(id)), one 4-byte shared load per token.
 #include "vt_common.cuh"
 
 namespace vt {
@@ -240,32 +240,39 @@ k_hist_hot(const int32_t* __restrict__ ids, int64_t n, int32_t V, uint32_t* __re
            const uint2* __restrict__ table, int32_t H, Ctrl* ctrl) {
     extern __shared__ __align__(16) uint8_t s_raw[];
     const int T32 = (V + 31) >> 5;
-    uint2* s_tbl = reinterpret_cast<uint2*>(s_raw);
+    // The lookup is repacked for the main pass: one 4-byte word per 16 ids = {16 membership bits,
+    // 16-bit slot of the first member} -- a 4-byte gather costs half the shared-memory wavefronts of
+    // an 8-byte one, and the lookup is one of the two shared-memory operations every token pays.
+    uint32_t* s_t16 = reinterpret_cast<uint32_t*>(s_raw);                       // [2 * T32]
     uint32_t* s_cnt = reinterpret_cast<uint32_t*>(s_raw + (size_t)T32 * 8);
-    for (int i = threadIdx.x; i < T32; i += kThreads) s_tbl[i] = table[i];
+    for (int i = threadIdx.x; i < T32; i += kThreads) {
+        const uint2 e = table[i];
+        s_t16[2 * i] = (e.x & 0xffffu) | (e.y << 16);
+        s_t16[2 * i + 1] = (e.x >> 16) | ((e.y + __popc(e.x & 0xffffu)) << 16);
+    }
     for (int i = threadIdx.x; i < H; i += kThreads) s_cnt[i] = 0;
     __syncthreads();
     unsigned long long bad = 0;
     stream_ids(ids, n, [&](uint32_t id) {
         if (id < (uint32_t)V) {
-            const uint2 e = s_tbl[id >> 5];
-            const uint32_t bit = 1u << (id & 31);
-            if (e.x & bit) atomicAdd(&s_cnt[e.y + __popc(e.x & (bit - 1))], 1u);
+            const uint32_t e = s_t16[id >> 4];
+            const uint32_t bit = 1u << (id & 15);
+            if (e & bit) atomicAdd(&s_cnt[(e >> 16) + __popc(e & (bit - 1))], 1u);
             else atomicAdd(&counts[id], 1u);
         } else {
             ++bad;
         }
     });
     __syncthreads();
-    for (int i = threadIdx.x; i < T32; i += kThreads) {
-        const int w = (i + blockIdx.x * 27) % T32;       // de-phase the CTAs' flushes
-        const uint2 e = s_tbl[w];
-        uint32_t bits = e.x, slot = e.y;
+    for (int i = threadIdx.x; i < 2 * T32; i += kThreads) {
+        const int g = (i + blockIdx.x * 53) % (2 * T32);   // de-phase the CTAs' flushes
+        const uint32_t e = s_t16[g];
+        uint32_t bits = e & 0xffffu, slot = e >> 16;
         while (bits) {
             const int b = __ffs(bits) - 1;
             bits &= bits - 1;
             const uint32_t c = s_cnt[slot++];
-            if (c) atomicAdd(&counts[w * 32 + b], c);
+            if (c) atomicAdd(&counts[g * 16 + b], c);
         }
     }
     report_bad(bad, ctrl);
@@ -312,7 +319,8 @@ cudaError_t launch_histogram(const int32_t* ids, int64_t n, int32_t V, uint32_t*
     }
     const size_t T32 = ((size_t)V + 31) / 32;
     if (T32 * 8 + 4096 > kDynSmem) return cudaErrorInvalidValue;   // rejected earlier by the API
-    const int32_t H = (int32_t)((kDynSmem - T32 * 8) / 4);
+    int32_t H = (int32_t)((kDynSmem - T32 * 8) / 4);
+    if (H > 65535) H = 65535;                          // slots are 16-bit in the main pass's lookup
     uint32_t* sample = reinterpret_cast<uint32_t*>(scratch + p.off_sample);
     uint2* table = reinterpret_cast<uint2*>(scratch + p.off_table);
     e = cudaMemsetAsync(sample, 0, (size_t)V * 4, s);
