@@ -22,6 +22,7 @@ constexpr int kSampleSlots = 4096;             // aggregating cache of the sampl
 constexpr int kSamplePerCta = 16384;           // ids sampled per CTA
 constexpr int kPickBins = 1024;                // sampled counts are clipped to kPickBins-1
 static_assert(kPickBins == kThreads, "one pick bin per thread");
+constexpr int kPickLoads = 16;                 // loads each thread of the one-CTA pick keeps in flight
 
 // ---- streaming loop shared by the counting kernels ---------------------------------------------
 // The CTA's share of the 16-byte-aligned body is read with four independent 128-bit loads per
@@ -146,16 +147,16 @@ k_hist_pick(const uint32_t* __restrict__ sample, int32_t V, int32_t H, uint2* __
     __syncthreads();
     {   // most bins were sampled a handful of times: count those in registers, one atomic per warp
         uint32_t small[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-        // eight loads in flight per thread: one CTA walking 128K counts one load at a time is all latency
-        for (int v0 = threadIdx.x; v0 < V; v0 += kThreads * 8) {
-            uint32_t cs[8];
+        // sixteen loads in flight per thread: one CTA walking 128K counts one load at a time is all latency
+        for (int v0 = threadIdx.x; v0 < V; v0 += kThreads * kPickLoads) {
+            uint32_t cs[kPickLoads];
 #pragma unroll
-            for (int q = 0; q < 8; ++q) {
+            for (int q = 0; q < kPickLoads; ++q) {
                 const int v = v0 + q * kThreads;
                 cs[q] = v < V ? __ldg(sample + v) : 0xffffffffu;
             }
 #pragma unroll
-            for (int q = 0; q < 8; ++q) {
+            for (int q = 0; q < kPickLoads; ++q) {
                 if (cs[q] == 0xffffffffu) continue;                     // past the end (a count never gets there)
                 const uint32_t c = min(cs[q], (uint32_t)(kPickBins - 1));
                 if (c < 8) {
@@ -185,15 +186,15 @@ k_hist_pick(const uint32_t* __restrict__ sample, int32_t V, int32_t H, uint2* __
     __syncthreads();
     const uint32_t quota = (uint32_t)H - s_definite;
     // pass A: one coalesced load per 32 ids, the membership words come out of warp ballots
-    for (int w0 = warp; w0 < T32; w0 += (kThreads / 32) * 8) {          // again eight loads in flight
-        uint32_t cs[8];
+    for (int w0 = warp; w0 < T32; w0 += (kThreads / 32) * kPickLoads) {          // again sixteen loads in flight
+        uint32_t cs[kPickLoads];
 #pragma unroll
-        for (int q = 0; q < 8; ++q) {
+        for (int q = 0; q < kPickLoads; ++q) {
             const int v = (w0 + q * (kThreads / 32)) * 32 + lane;
             cs[q] = v < V ? min(__ldg(sample + v), (uint32_t)(kPickBins - 1)) : 0xffffffffu;
         }
 #pragma unroll
-        for (int q = 0; q < 8; ++q) {
+        for (int q = 0; q < kPickLoads; ++q) {
             const int w = w0 + q * (kThreads / 32);
             if (w >= T32) break;                                        // warp-uniform
             const bool in = cs[q] != 0xffffffffu;
