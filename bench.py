@@ -389,9 +389,33 @@ def draft_block_case(vt, dev, timed):
     tok, par, tgt = tok.to(dev), par.to(dev), tgt.to(dev)
     total = torch.zeros(1, dtype=torch.int64, device=dev)
     ms_v = timed(lambda: vt.vt_verify_greedy(tok, par, tgt, tokens_total=total), reps=200, warm=10)
-    return {"workload": "tree depth 3 / top-8 / 32 draft tokens; verification of 64 trees",
-            "tree_3_expansions_plus_rerank_us": ms_t * 1e3, "launches_per_tree": depth + 1,
-            "verify_64_trees_us": ms_v * 1e3}
+    out = {"workload": "tree depth 3 / top-8 / 32 draft tokens; verification of 64 trees",
+           "tree_3_expansions_plus_rerank_us": ms_t * 1e3, "launches_per_tree": depth + 1,
+           "verify_64_trees_us": ms_v * 1e3}
+    # one tree depth of config 3 (B = 10 nodes, top-10, K = 32768): head + expansion as two launches and
+    # as the single launch of vt_draft_head_expand
+    wl = build_head_workload(vt, dev, TREE["d"], 32768, TREE["B"], TREE["topk"], TREE["temp"], True, seed=1003)
+    B, tk = TREE["B"], TREE["topk"]
+    pool2 = vt.tree_pool(64 + B * tk, dev)
+    pool2[2].zero_()
+    front = torch.arange(B, dtype=torch.int32, device=dev)
+    copies, hs, us = wl["copies"], wl["hs"], wl["us"]
+    state = {"i": 0}
+
+    def two_launches():
+        i = state["i"] = state["i"] + 1
+        ids_, lp_ = vt.vt_draft_head(hs[i % len(hs)], copies[i % len(copies)], wl["map"], wl["T"], tk,
+                                     us[i % len(us)], ws=wl["ws"], out=wl["out"], overlapped=True)
+        vt.vt_tree_expand(ids_, lp_, front, pool2, 64, tk, col0=1)
+
+    def one_launch():
+        i = state["i"] = state["i"] + 1
+        vt.vt_draft_head_expand(hs[i % len(hs)], copies[i % len(copies)], wl["map"], wl["T"], tk, us[i % len(us)],
+                                front, pool2, 64, tk, ws=wl["ws"], out=wl["out"])
+
+    out["config3_depth_K32768_head_then_expand_us"] = timed(two_launches, reps=300, warm=20) * 1e3
+    out["config3_depth_K32768_fused_us"] = timed(one_launch, reps=300, warm=20) * 1e3
+    return out
 
 
 DENSE = dict(d=4096, K=32768, B=256, topk=8)                   # BASELINE config 4 (batched serving)

@@ -267,6 +267,21 @@ vt_status vt_draft_head_overlapped(const uint16_t *h, const uint16_t *W_trim, co
                                    const float *uniforms, int32_t *out_ids, float *out_logprobs,
                                    void *ws, size_t ws_bytes, void *stream);
 
+/*
+ * One tree depth in one call: vt_draft_head_overlapped followed by vt_tree_expand on its candidates
+ * (out_ids / out_logprobs columns 1..topk), with the same arguments, results and limits as those two
+ * (Algorithm 2 lines 5-6 with the draft tree of Section 4.1).  For the streaming kernel's shapes
+ * (B <= 16) the expansion runs inside the head kernel, in the CTA that merges the rows, so a tree
+ * depth costs one launch; other shapes chain the expansion kernel behind the merge.  The caller's
+ * promise about W_trim is that of vt_draft_head_overlapped.
+ */
+vt_status vt_draft_head_expand(const uint16_t *h, const uint16_t *W_trim, const int32_t *map, int32_t B,
+                               int32_t K, int32_t d, const float *temp, int32_t topk,
+                               const float *uniforms, int32_t *out_ids, float *out_logprobs,
+                               const int32_t *frontier_nodes, int32_t *pool_token, int32_t *pool_parent,
+                               float *pool_score, int32_t pool_base, int32_t pool_capacity, int32_t n_front,
+                               int32_t *next_frontier, void *ws, size_t ws_bytes, void *stream);
+
 /* Parity-only variant of vt_draft_head: also writes the fp32 logits [B,K] and lse [B]
  * (log sum exp of z) when those pointers are non-NULL.  Never used for timing. */
 vt_status vt_draft_head_debug(const uint16_t *h, const uint16_t *W_trim, const int32_t *map,

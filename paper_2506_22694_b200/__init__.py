@@ -32,7 +32,7 @@ EXPORTS = (
     "vt_last_cuda_error",
     "vt_histogram", "vt_select_topk", "vt_build_vocab", "vt_build_vocab_host", "vt_trim_head",
     "vt_draft_head", "vt_draft_head_debug", "vt_draft_head_host", "vt_select_topk_static",
-    "vt_draft_head_overlapped", "vt_select_topp", "vt_select_minfreq", "vt_verify_greedy", "vt_mbsu", "vt_tree_expand", "vt_tree_rerank",
+    "vt_draft_head_overlapped", "vt_select_topp", "vt_select_minfreq", "vt_verify_greedy", "vt_mbsu", "vt_tree_expand", "vt_tree_rerank", "vt_draft_head_expand",
 )
 
 
@@ -71,6 +71,7 @@ def lib() -> ctypes.CDLL:
         L.vt_mbsu.argtypes = [c_double, c_double, c_double, c_int32]
         L.vt_mbsu.restype = c_double
         L.vt_tree_expand.argtypes = [c_void_p, c_void_p, c_int32, c_int32, c_int32, c_int32, c_void_p, c_void_p, c_void_p, c_void_p, c_int32, c_int32, c_int32, c_void_p, c_void_p]
+        L.vt_draft_head_expand.argtypes = [c_void_p, c_void_p, c_void_p, c_int32, c_int32, c_int32, c_void_p, c_int32, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_int32, c_int32, c_int32, c_void_p, c_void_p, c_size_t, c_void_p]
         L.vt_tree_rerank.argtypes = [c_void_p, c_void_p, c_void_p, c_int32, c_int32, c_void_p, c_void_p, c_void_p, c_void_p]
         L.vt_build_vocab.argtypes = [c_void_p, c_int64, c_int32, c_int32, c_void_p, c_void_p, c_void_p,
                                      c_size_t, c_void_p]
@@ -218,6 +219,39 @@ def vt_tree_expand(cand_ids: torch.Tensor, cand_logprobs: torch.Tensor, frontier
         _ptr(cand_ids), _ptr(cand_logprobs), B, ld - col0, ld, col0, _ptr(frontier_nodes), _ptr(tok), _ptr(par),
         _ptr(sc), pool_base, min(tok.numel(), par.numel(), sc.numel()), n_front, _ptr(nxt), _stream()))
     return nxt
+
+
+def vt_draft_head_expand(h: torch.Tensor, W_trim: torch.Tensor, map_: torch.Tensor | None, temp: torch.Tensor,
+                         topk: int, uniforms: torch.Tensor | None, frontier_nodes: torch.Tensor | None, pool,
+                         pool_base: int, n_front: int, ws: Workspace | None = None, out=None):
+    """One tree depth in one call: the head (as vt_draft_head(..., overlapped=True)) and the expansion of
+    its candidates into the node pool.  Returns (out_ids, out_logprobs, next_frontier [n_front])."""
+    _dev(h, torch.bfloat16, "h")
+    _dev(W_trim, torch.bfloat16, "W_trim")
+    _dev(temp, torch.float32, "temp")
+    B, d = h.shape
+    K = W_trim.shape[0]
+    if W_trim.shape[1] != d or temp.numel() != B:
+        raise ValueError("shape mismatch between h, W_trim and temp")
+    if map_ is not None and _dev(map_, torch.int32, "map").numel() != K:
+        raise ValueError("map must have K entries")
+    if uniforms is not None and tuple(_dev(uniforms, torch.float32, "uniforms").shape) != (B, K):
+        raise ValueError("uniforms must be [B,K]")
+    if frontier_nodes is not None and _dev(frontier_nodes, torch.int32, "frontier_nodes").numel() != B:
+        raise ValueError("frontier_nodes must have B entries")
+    tok, par, sc = pool
+    _dev(tok, torch.int32, "pool token"), _dev(par, torch.int32, "pool parent"), _dev(sc, torch.float32, "pool score")
+    if out is None:
+        out = (torch.empty((B, 1 + topk), dtype=torch.int32, device=h.device),
+               torch.empty((B, 1 + topk), dtype=torch.float32, device=h.device))
+    ids, lps = out
+    nxt = torch.empty(n_front, dtype=torch.int32, device=h.device)
+    ws = _ws(ws, workspace_bytes(VT_OP_DRAFT_HEAD, 0, 0, K, d, B, topk), h)
+    _check("vt_draft_head_expand", lib().vt_draft_head_expand(
+        _ptr(h), _ptr(W_trim), _ptr(map_), B, K, d, _ptr(temp), topk, _ptr(uniforms), _ptr(ids), _ptr(lps),
+        _ptr(frontier_nodes), _ptr(tok), _ptr(par), _ptr(sc), pool_base, min(tok.numel(), par.numel(), sc.numel()),
+        n_front, _ptr(nxt), c_void_p(ws.ptr), ws.nbytes, _stream()))
+    return ids, lps, nxt
 
 
 def vt_tree_rerank(pool, n: int, budget: int):

@@ -206,20 +206,28 @@ vt_status vt_select_minfreq(const uint32_t* counts, int32_t V, uint32_t min_coun
     return select_cut_impl(counts, V, 1, 1.0, min_count, map, inv_map, k_out, ws, ws_bytes, stream);
 }
 
-vt_status vt_tree_expand(const int32_t* cand_ids, const float* cand_logprobs, int32_t B, int32_t topk,
-                         int32_t ld, int32_t col0, const int32_t* frontier_nodes, int32_t* pool_token,
-                         int32_t* pool_parent, float* pool_score, int32_t pool_base, int32_t pool_capacity,
-                         int32_t n_front, int32_t* next_frontier, void* stream) {
-    if (!cand_ids || !cand_logprobs || !pool_token || !pool_parent || !pool_score || !next_frontier)
-        return VT_ERR_INVALID_ARG;
-    if (B < 1 || topk < 1 || col0 < 0 || ld < col0 + topk || pool_base < 0 || n_front < 1) return VT_ERR_INVALID_ARG;
+static vt_status check_tree_args(int32_t B, int32_t topk, const int32_t* frontier_nodes, const int32_t* pool_token,
+                                 const int32_t* pool_parent, const float* pool_score, int32_t pool_base,
+                                 int32_t pool_capacity, int32_t n_front, const int32_t* next_frontier) {
+    if (!pool_token || !pool_parent || !pool_score || !next_frontier) return VT_ERR_INVALID_ARG;
+    if (B < 1 || topk < 1 || pool_base < 0 || n_front < 1) return VT_ERR_INVALID_ARG;
     if (!frontier_nodes && B != 1) return VT_ERR_INVALID_ARG;
     const int64_t n_new = (int64_t)B * topk;
     if (n_new > tree_max_nodes()) return VT_ERR_UNSUPPORTED;
     if (n_front > n_new || pool_base + n_new > pool_capacity) return VT_ERR_INVALID_ARG;
-    return from_cuda(launch_tree_expand(cand_ids, cand_logprobs, B, topk, ld, col0, frontier_nodes, pool_token,
-                                        pool_parent, pool_score, pool_base, n_front, next_frontier,
-                                        as_stream(stream)));
+    return VT_OK;
+}
+
+vt_status vt_tree_expand(const int32_t* cand_ids, const float* cand_logprobs, int32_t B, int32_t topk,
+                         int32_t ld, int32_t col0, const int32_t* frontier_nodes, int32_t* pool_token,
+                         int32_t* pool_parent, float* pool_score, int32_t pool_base, int32_t pool_capacity,
+                         int32_t n_front, int32_t* next_frontier, void* stream) {
+    if (!cand_ids || !cand_logprobs || col0 < 0 || topk < 1 || ld < col0 + topk) return VT_ERR_INVALID_ARG;
+    const vt_status st = check_tree_args(B, topk, frontier_nodes, pool_token, pool_parent, pool_score, pool_base,
+                                         pool_capacity, n_front, next_frontier);
+    if (st != VT_OK) return st;
+    const TreeArgs t{frontier_nodes, pool_token, pool_parent, pool_score, pool_base, n_front, next_frontier};
+    return from_cuda(launch_tree_expand(cand_ids, cand_logprobs, B, topk, ld, col0, t, as_stream(stream)));
 }
 
 vt_status vt_tree_rerank(const int32_t* pool_token, const int32_t* pool_parent, const float* pool_score,
@@ -334,7 +342,7 @@ static vt_status draft_head_impl(const uint16_t* h, const uint16_t* W_trim, cons
                                  int32_t B, int32_t K, int32_t d, const float* temp, int32_t topk,
                                  const float* uniforms, int32_t* out_ids, float* out_logprobs,
                                  void* ws, size_t ws_bytes, void* stream, float* out_logits,
-                                 float* out_lse, int overlap) {
+                                 float* out_lse, int overlap, const TreeArgs& tree = TreeArgs{}) {
     if (!h || !W_trim || !temp || !out_ids || !out_logprobs) return VT_ERR_INVALID_ARG;
     if (B < 1 || K < 1 || d < 8 || (d & 7) || topk < 1 || topk > VT_MAX_TOPK || topk > K)
         return VT_ERR_INVALID_ARG;
@@ -343,7 +351,7 @@ static vt_status draft_head_impl(const uint16_t* h, const uint16_t* W_trim, cons
     vt_status st = check_ws(ws, ws_bytes, vt_workspace_bytes(VT_OP_DRAFT_HEAD, 0, 0, K, d, B, topk));
     if (st != VT_OK) return st;
     uint8_t* base = static_cast<uint8_t*>(ws);
-    HeadArgs a{h, W_trim, map, B, K, d, temp, topk, uniforms, out_ids, out_logprobs, out_logits, out_lse, overlap};
+    HeadArgs a{h, W_trim, map, B, K, d, temp, topk, uniforms, out_ids, out_logprobs, out_logits, out_lse, overlap, tree};
     if (head_skinny_supported(B, d))
         return from_cuda(launch_head_skinny(a, reinterpret_cast<Ctrl*>(base), base + VT_CTRL_BYTES,
                                             as_stream(stream)));
@@ -374,6 +382,20 @@ vt_status vt_draft_head_overlapped(const uint16_t* h, const uint16_t* W_trim, co
                                    size_t ws_bytes, void* stream) {
     return draft_head_impl(h, W_trim, map, B, K, d, temp, topk, uniforms, out_ids, out_logprobs, ws, ws_bytes,
                            stream, nullptr, nullptr, 1);
+}
+
+vt_status vt_draft_head_expand(const uint16_t* h, const uint16_t* W_trim, const int32_t* map, int32_t B,
+                               int32_t K, int32_t d, const float* temp, int32_t topk, const float* uniforms,
+                               int32_t* out_ids, float* out_logprobs, const int32_t* frontier_nodes,
+                               int32_t* pool_token, int32_t* pool_parent, float* pool_score, int32_t pool_base,
+                               int32_t pool_capacity, int32_t n_front, int32_t* next_frontier, void* ws,
+                               size_t ws_bytes, void* stream) {
+    const vt_status st = check_tree_args(B, topk, frontier_nodes, pool_token, pool_parent, pool_score, pool_base,
+                                         pool_capacity, n_front, next_frontier);
+    if (st != VT_OK) return st;
+    const TreeArgs t{frontier_nodes, pool_token, pool_parent, pool_score, pool_base, n_front, next_frontier};
+    return draft_head_impl(h, W_trim, map, B, K, d, temp, topk, uniforms, out_ids, out_logprobs, ws, ws_bytes,
+                           stream, nullptr, nullptr, 1, t);
 }
 
 vt_status vt_draft_head_host(const uint16_t* h_host, const uint16_t* W_trim, const int32_t* map,

@@ -47,11 +47,19 @@ cudaError_t launch_verify_greedy(const int32_t* token, const int32_t* parent, co
                                  int32_t N, int32_t* n_accept, int32_t* path, int32_t* emitted,
                                  unsigned long long* tokens_total, cudaStream_t st);
 
+// One depth of the draft-tree expansion (vt_tree_expand's arguments); pool_token == nullptr: none.
+struct TreeArgs {
+    const int32_t* frontier;      // [B] pool index of each hidden row's node, or nullptr (the prefix)
+    int32_t* pool_token;
+    int32_t* pool_parent;
+    float* pool_score;
+    int32_t pool_base, n_front;
+    int32_t* next_frontier;       // [n_front]
+};
+
 int tree_max_nodes();
 cudaError_t launch_tree_expand(const int32_t* cand_ids, const float* cand_lp, int32_t B, int32_t topk, int32_t ld,
-                               int32_t col0, const int32_t* frontier, int32_t* pool_token, int32_t* pool_parent,
-                               float* pool_score, int32_t pool_base, int32_t n_front, int32_t* next_frontier,
-                               cudaStream_t st);
+                               int32_t col0, const TreeArgs& t, cudaStream_t st);
 cudaError_t launch_tree_rerank(const int32_t* pool_token, const int32_t* pool_parent, const float* pool_score,
                                int32_t n, int32_t budget, int32_t* out_nodes, int32_t* out_token,
                                int32_t* out_parent, cudaStream_t st);
@@ -72,6 +80,7 @@ struct HeadArgs {
     float* dbg_logits;
     float* dbg_lse;
     int32_t overlap;       // launch with programmatic stream serialization (weights may be fetched early)
+    TreeArgs tree;         // expansion to run on the merged top-k (pool_token == nullptr: none)
 };
 bool head_skinny_supported(int32_t B, int32_t d);
 size_t head_skinny_scratch_bytes(int32_t B, int32_t K, int32_t topk);

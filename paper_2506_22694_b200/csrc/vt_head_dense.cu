@@ -677,7 +677,10 @@ cudaError_t launch_head_dense(const HeadArgs& a, Ctrl* ctrl, uint8_t* scratch, c
     cfg.attrs = &at;
     cfg.numAttrs = 1;
     count_launch(2);
-    return cudaLaunchKernelEx(&cfg, k_head_merge, a, ctrl, static_cast<const float*>(recs), geo.n_groups);
+    e = cudaLaunchKernelEx(&cfg, k_head_merge, a, ctrl, static_cast<const float*>(recs), geo.n_groups);
+    if (e != cudaSuccess || !a.tree.pool_token) return e;
+    // tree drafting: the expansion needs every row's merge, i.e. the whole merge grid: one more launch
+    return launch_tree_expand(a.out_ids, a.out_logprobs, a.B, a.topk, 1 + a.topk, 1, a.tree, s);
 }
 
 }  // namespace vt

@@ -28,6 +28,7 @@
 
 #include "vt_common.cuh"
 #include "vt_head_common.cuh"
+#include "vt_tree_common.cuh"
 
 namespace vt {
 
@@ -434,11 +435,19 @@ k_head_stream(const HeadArgs a, Ctrl* ctrl, float* __restrict__ recs, const Geo 
         s_last = (atomicInc(&ctrl->head_ticket, gridDim.x - 1) == gridDim.x - 1);
     }
     __syncthreads();
-    if (!s_last || b >= B) return;
+    if (!s_last) return;
     __threadfence();
 
-    merge_records(a.map, a.out_ids, a.out_logprobs, a.dbg_lse, topk, a.uniforms != nullptr, ctrl, recs, b, row_ok,
-                  (int)gridDim.x, reinterpret_cast<float*>(ring) + (size_t)b * kMergeStageWords);
+    if (b < B)
+        merge_records(a.map, a.out_ids, a.out_logprobs, a.dbg_lse, topk, a.uniforms != nullptr, ctrl, recs, b, row_ok,
+                      (int)gridDim.x, reinterpret_cast<float*>(ring) + (size_t)b * kMergeStageWords);
+    if (a.tree.pool_token) {
+        // tree drafting: the merged candidates of all rows become pool nodes and the next frontier is
+        // chosen here, by the CTA that merged them, instead of in a launch of its own
+        __syncthreads();                                   // the rows' outputs are written; the staging area is free
+        tree_expand_block(a.tree, a.out_ids, a.out_logprobs, B, topk, 1 + topk, 1,
+                          reinterpret_cast<unsigned long long*>(ring), (int)threadIdx.x, kThreads);
+    }
 }
 
 // ---- host side ---------------------------------------------------------------------------------------

@@ -138,3 +138,60 @@ def test_head_to_tree_to_verification_on_the_trimmed_vocabulary():
     r_acc, r_path, r_emit = oracle.verify_greedy(token.cpu().numpy()[None], p[None], target.numpy())
     assert np.array_equal(n_acc.cpu().numpy(), r_acc) and np.array_equal(path.cpu().numpy(), r_path)
     assert np.array_equal(emitted.cpu().numpy(), r_emit) and int(n_acc.item()) >= 1
+
+
+@pytest.mark.parametrize("K,d,topk,n_front,depth,sample", [(4096, 512, 8, 8, 3, False), (3000, 1024, 10, 10, 4, True),
+                                                            (700, 72, 4, 6, 3, True), (2048, 256, 16, 16, 2, False)])
+def test_head_with_fused_expansion_equals_head_then_expansion(K, d, topk, n_front, depth, sample):
+    """vt_draft_head_expand (one launch per tree depth on the streaming kernel) against vt_draft_head
+    followed by vt_tree_expand: same ids, log-probs, pool and frontier, bit for bit; the pool is also what
+    the oracle's expansion makes of those candidates."""
+    W = vt_inputs.gaussian_bf16((K, d), 0.05, seed=K + 1, device=DEV)
+    m = torch.randperm(K * 2, device=DEV)[:K].to(torch.int32)
+    cap = topk + (depth - 1) * n_front * topk
+    pool_a, pool_b = vt.tree_pool(cap), vt.tree_pool(cap)
+    tok = np.full(cap, -9, dtype=np.int32); par = np.full(cap, -9, dtype=np.int32)
+    sc = np.full(cap, np.nan, dtype=np.float32)
+    fa = fb = fr = None
+    base, B = 0, 1
+    for dep in range(depth):
+        h = vt_inputs.gaussian_bf16((B, d), 1.0, seed=50 + dep, device=DEV)
+        T = vt_inputs.temperatures(B, 0.7, 1.3, seed=60 + dep, device=DEV)
+        u = vt_inputs.uniforms((B, K), seed=70 + dep, device=DEV) if sample else None
+        nf = min(n_front, B * topk)
+        ids_a, lp_a = vt.vt_draft_head(h, W, m, T, topk, u)
+        fa = vt.vt_tree_expand(ids_a, lp_a, fa, pool_a, base, nf, col0=1)
+        ids_b, lp_b, fb = vt.vt_draft_head_expand(h, W, m, T, topk, u, fb, pool_b, base, nf)
+        assert torch.equal(ids_a, ids_b) and torch.equal(lp_a.view(torch.int32), lp_b.view(torch.int32))
+        assert torch.equal(fa, fb)
+        fr = oracle.tree_expand(ids_a[:, 1:].cpu().numpy(), lp_a[:, 1:].cpu().numpy(), fr, tok, par, sc, base, nf)
+        assert np.array_equal(fb.cpu().numpy(), fr)
+        base += B * topk
+        B = nf
+    for x, y in zip(pool_a, pool_b):
+        assert torch.equal(x[:base].view(torch.int32), y[:base].view(torch.int32))
+    assert np.array_equal(pool_b[0][:base].cpu().numpy(), tok[:base])
+    assert np.array_equal(pool_b[1][:base].cpu().numpy(), par[:base])
+    assert np.array_equal(_bits(pool_b[2][:base].cpu().numpy()), _bits(sc[:base]))
+
+
+def test_fused_expansion_on_the_dense_path_and_argument_checks():
+    K, d, topk, B = 1500, 128, 8, 40                         # more than 16 rows: tensor-core kernel + chained expansion
+    W = vt_inputs.gaussian_bf16((K, d), 0.05, seed=3, device=DEV)
+    h = vt_inputs.gaussian_bf16((B, d), 1.0, seed=4, device=DEV)
+    T = torch.ones(B, device=DEV)
+    cap = 64 + B * topk
+    prev = (-torch.arange(cap, dtype=torch.float32, device=DEV) / 5)
+    pool_a = (torch.zeros(cap, dtype=torch.int32, device=DEV), torch.full((cap,), -1, dtype=torch.int32, device=DEV), prev.clone())
+    pool_b = tuple(t.clone() for t in pool_a)
+    front = torch.arange(B, dtype=torch.int32, device=DEV)
+    ids_a, lp_a = vt.vt_draft_head(h, W, None, T, topk, None)
+    fa = vt.vt_tree_expand(ids_a, lp_a, front, pool_a, 64, 24, col0=1)
+    ids_b, lp_b, fb = vt.vt_draft_head_expand(h, W, None, T, topk, None, front, pool_b, 64, 24)
+    assert torch.equal(ids_a, ids_b) and torch.equal(fa, fb)
+    for x, y in zip(pool_a, pool_b):
+        assert torch.equal(x.view(torch.int32), y.view(torch.int32))
+    with pytest.raises(vt.VocabTrimError):                     # pool too small for B*topk new nodes
+        vt.vt_draft_head_expand(h, W, None, T, topk, None, front, vt.tree_pool(100), 64, 24)
+    with pytest.raises(vt.VocabTrimError):                     # several rows need their frontier nodes
+        vt.vt_draft_head_expand(h, W, None, T, topk, None, None, vt.tree_pool(cap), 0, 8)
