@@ -143,56 +143,100 @@ k_select_sort(const uint32_t* counts, int32_t V, int32_t K, int32_t* map, int32_
 // Cut of a full ranking at a data-dependent K (the Method section's Top-P and minimum-frequency
 // variants of the selection).  `map` holds all V ids in rank order.  mode 0: smallest K whose prefix
 // of counts reaches ceil(p * total); mode 1: K = number of ids with count >= min_count.  K is clamped
-// to [1, V]; inv_map entries of ranks >= K become -1.  One CTA: V is about 1e5, this is latency.
-__global__ void __launch_bounds__(kThreads, 1)
+// to [1, V]; inv_map entries of ranks >= K become -1.  Pure latency (two dependent loads per rank), so
+// the ranks are dealt to the 8 CTAs of a cluster, each thread a contiguous run; the CTAs' sums meet
+// through distributed shared memory, like the digit totals of the sort.
+__global__ void __cluster_dims__(kCluster, 1, 1) __launch_bounds__(kThreads, 1)
 k_select_cut(const uint32_t* __restrict__ counts, int32_t V, int mode, double pfrac, uint32_t min_count,
              const int32_t* __restrict__ map, int32_t* __restrict__ inv_map, int32_t* __restrict__ k_out) {
+    cg::cluster_group cluster = cg::this_cluster();
+    const unsigned rank = cluster.block_rank();
     __shared__ unsigned long long s_part[kThreads];
-    __shared__ unsigned long long s_total;
-    __shared__ int s_k;
-    const int per = (V + kThreads - 1) / kThreads;                 // consecutive ranks per thread
-    const int j0 = min(V, (int)threadIdx.x * per), j1 = min(V, j0 + per);
+    __shared__ unsigned long long s_cta_total;          // this CTA's sum (read by the peers)
+    __shared__ int s_k;                                 // CTA 0's copy is the cluster's answer
+    const int T = kCluster * kThreads;                  // threads of the cluster, in rank order
+    const int t = (int)rank * kThreads + (int)threadIdx.x;
+    const int per = (V + T - 1) / T;                    // consecutive ranks per thread
+    const int j0 = min(V, t * per), j1 = min(V, j0 + per);
     unsigned long long sum = 0;
     int ge = 0;
-    for (int j = j0; j < j1; ++j) {
-        const uint32_t c = counts[map[j]];
-        sum += c;
-        ge += c >= min_count;
+    for (int j = j0; j < j1; j += 8) {                  // eight ranks (id, then its count) in flight per thread
+        int32_t id[8];
+        uint32_t c[8];
+#pragma unroll
+        for (int q = 0; q < 8; ++q) id[q] = j + q < j1 ? map[j + q] : -1;
+#pragma unroll
+        for (int q = 0; q < 8; ++q) c[q] = id[q] >= 0 ? counts[id[q]] : 0u;
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            sum += c[q];
+            ge += (id[q] >= 0) & (c[q] >= min_count);
+        }
     }
     s_part[threadIdx.x] = mode == 0 ? sum : (unsigned long long)ge;
     if (threadIdx.x == 0) s_k = V;
     __syncthreads();
-    if (threadIdx.x == 0) {                                        // exclusive scan of 1024 partials: trivial serially
-        unsigned long long run = 0;
-        for (int t = 0; t < kThreads; ++t) {
-            const unsigned long long x = s_part[t];
-            s_part[t] = run;
-            run += x;
+    if (threadIdx.x < 32) {                             // exclusive scan of this CTA's 1024 partials by one warp
+        unsigned long long x[kThreads / 32], run = 0;
+#pragma unroll
+        for (int q = 0; q < kThreads / 32; ++q) {       // lane l owns partials 32 l .. 32 l + 31
+            x[q] = s_part[threadIdx.x * (kThreads / 32) + q];
+            run += x[q];
         }
-        s_total = run;
+        unsigned long long incl = run;
+        for (int o = 1; o < 32; o <<= 1) {
+            const unsigned long long y = __shfl_up_sync(0xffffffffu, incl, o);
+            if ((int)threadIdx.x >= o) incl += y;
+        }
+        unsigned long long pre = incl - run;
+#pragma unroll
+        for (int q = 0; q < kThreads / 32; ++q) {
+            s_part[threadIdx.x * (kThreads / 32) + q] = pre;
+            pre += x[q];
+        }
+        if (threadIdx.x == 31) s_cta_total = incl;
     }
-    __syncthreads();
+    cluster.sync();                                     // every CTA's total and s_k are in place
+    unsigned long long before = 0, total = 0;           // sums of the CTAs before this one / of all
+    for (unsigned c = 0; c < kCluster; ++c) {
+        const unsigned long long x = *cluster.map_shared_rank(&s_cta_total, c);
+        before += c < rank ? x : 0ull;
+        total += x;
+    }
+    int* k_shared = cluster.map_shared_rank(&s_k, 0);
     if (mode == 0) {
-        const double target = ceil(pfrac * (double)s_total);
-        unsigned long long cum = s_part[threadIdx.x];
-        for (int j = j0; j < j1; ++j) {
-            cum += counts[map[j]];
-            if ((double)cum >= target) { atomicMin(&s_k, j + 1); break; }
+        const double target = ceil(pfrac * (double)total);
+        unsigned long long cum = before + s_part[threadIdx.x];
+        if (t == 0 && target <= 0.0) atomicMin(k_shared, 1);           // an empty histogram: the first rank already reaches it
+        // only the thread whose run of ranks crosses the target walks it again
+        if ((double)cum < target && (double)(cum + sum) >= target) {
+            for (int j = j0; j < j1; ++j) {
+                cum += counts[map[j]];
+                if ((double)cum >= target) { atomicMin(k_shared, j + 1); break; }
+            }
         }
-    } else if (threadIdx.x == 0) {
-        s_k = (int)s_total;
+    } else if (t == 0) {
+        atomicMin(k_shared, (int)total);
     }
-    __syncthreads();
-    const int K = max(1, min(V, s_k));
-    if (threadIdx.x == 0) *k_out = K;
-    for (int j = K + (int)threadIdx.x; j < V; j += kThreads) inv_map[map[j]] = -1;
+    cluster.sync();                                     // the answer is final; CTA 0 stays until all have read it
+    const int K = max(1, min(V, *k_shared));
+    if (t == 0) *k_out = K;
+    for (int j = K + t; j < V; j += T * 8) {            // eight ids in flight per thread
+        int32_t id[8];
+#pragma unroll
+        for (int q = 0; q < 8; ++q) id[q] = j + q * T < V ? map[j + q * T] : -1;
+#pragma unroll
+        for (int q = 0; q < 8; ++q)
+            if (id[q] >= 0) inv_map[id[q]] = -1;
+    }
+    cluster.sync();                                     // nobody leaves while a peer may still read its shared memory
 }
 
 }  // namespace
 
 cudaError_t launch_select_cut(const uint32_t* counts, int32_t V, int mode, double pfrac, uint32_t min_count,
                               const int32_t* map, int32_t* inv_map, int32_t* k_out, cudaStream_t s) {
-    k_select_cut<<<1, kThreads, 0, s>>>(counts, V, mode, pfrac, min_count, map, inv_map, k_out);
+    k_select_cut<<<kCluster, kThreads, 0, s>>>(counts, V, mode, pfrac, min_count, map, inv_map, k_out);
     count_launch();
     return cudaGetLastError();
 }
