@@ -176,6 +176,9 @@ def test_config3_tree_drafting_sweep(K):
 @pytest.mark.parametrize("B,K,d,topk,sample", [
     (17, 300, 72, 5, True), (40, 1000, 256, 8, True), (64, 128, 64, 1, False), (130, 515, 200, 16, True),
     (256, 2048, 512, 8, True), (128, 4099, 1024, 4, True), (12, 700, 4104, 6, True), (200, 9, 8, 9, True),
+    (129, 300, 64, 3, True),
+    # four tiles per CTA (pair): both accumulator stages are reused, the ring wraps many times
+    (256, 60000, 64, 8, True), (100, 150001, 72, 4, False),
 ])
 def test_dense_path_small_shapes_and_ragged_tails(B, K, d, topk, sample):
     W = vt_inputs.gaussian_bf16((K, d), 0.02, seed=K + d, device=DEV)
