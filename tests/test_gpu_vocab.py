@@ -76,6 +76,27 @@ def test_histogram_degenerate_streams():
     assert np.array_equal(_u32(vt.vt_histogram(ramp, V, ws=ws)), ref)
 
 
+def test_histogram_three_ids_carry_the_whole_stream():
+    """Streams that drive single bins to 1e7 and more: neighbouring ids, ids around the middle and the
+    end of the vocabulary, with a sprinkle of a fourth id."""
+    V = 128256
+    n = 40_000_000
+    ws = vt.Workspace(vt.workspace_bytes(vt.VT_OP_HISTOGRAM, n, V))
+    for a, b, c in ((4, 5, 6), (114_687, 114_688, 0), (128_255, 128_254, 57_345)):
+        i = torch.arange(n, device=DEV, dtype=torch.int32)
+        ids = torch.where(i % 3 == 0, a, torch.where(i % 3 == 1, b, c)).to(torch.int32)
+        ids[::1_000_003] = 99_999                                   # a sprinkle of something else
+        got = _u32(vt.vt_histogram(ids, V, ws=ws))
+        ref = torch.bincount(ids.long(), minlength=V).cpu().numpy().astype(np.uint64)   # integers: torch counts as the oracle does
+        small, _ = oracle.histogram(ids[:300_000].cpu().numpy(), V)
+        assert np.array_equal(torch.bincount(ids[:300_000].long(), minlength=V).cpu().numpy().astype(np.uint64), small)
+        assert np.array_equal(got, ref)
+        _assert_clean(ws)
+    acc = vt.vt_histogram(ids, V, ws=ws)                            # accumulate on top: counts double
+    vt.vt_histogram(ids, V, counts=acc, accumulate=True, ws=ws)
+    assert np.array_equal(_u32(acc), 2 * ref)
+
+
 @pytest.mark.parametrize("V,K", [(1, 1), (6, 3), (4096, 1024), (4096, 4096), (128256, 8192), (128256, 32768),
                                  (128256, 128256), (131072, 1), (200_001, 70_000)])
 def test_select_topk_matches_oracle(V, K):
