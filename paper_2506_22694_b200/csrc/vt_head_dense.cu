@@ -11,7 +11,7 @@
 // two halves of the B operand from both shared memories.  Per SM and flop this halves the operand
 // bytes staged and read compared with two M tiles in one CTA, which is what bounded that form.
 //
-// Warp 0 feeds a shared-memory ring with TMA tensor copies (128-byte swizzle, no multicast); in a pair
+// Warp 0 feeds a shared-memory ring with TMA tensor copies (128-byte swizzle, every CTA fetches its own tiles); in a pair
 // both CTAs' copies count their bytes on the leader's barrier.  One thread of warp 1 (of the leader)
 // issues the MMAs (bf16 x bf16 -> fp32) with the operands described in place by shared-memory
 // descriptors and the accumulators in tensor memory: two accumulator stages of up to 256 columns, so
@@ -171,11 +171,13 @@ __device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap
         "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
         ::"r"(dst), "l"(tm), "r"(bar_cluster), "r"(x), "r"(y) : "memory");
 }
-// arrives on the barrier at this shared-memory offset in both CTAs once the MMAs issued so far are done
+// arrives on the barrier at this shared-memory offset in both CTAs once the MMAs issued so far are done:
+// one commit per CTA of the pair (the peer's barrier by its shared::cluster address)
 __device__ __forceinline__ void tc_commit_pair(uint64_t* bar) {
-    asm volatile(
-        "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
-        ::"r"(smem_u32(bar)), "h"((uint16_t)3) : "memory");
+    const uint32_t own = smem_u32(bar);
+    const uint32_t peer = mapa_u32(own, 1);
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(own) : "memory");
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(peer) : "memory");
 }
 // D[tmem of both CTAs] (+)= A * B^T, 256 x N x 16: each CTA supplies 128 rows of A and N/2 rows of B
 __device__ __forceinline__ void tc_mma_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t acc) {
