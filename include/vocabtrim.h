@@ -293,7 +293,9 @@ vt_status vt_draft_head_debug(const uint16_t *h, const uint16_t *W_trim, const i
 /* Same as vt_draft_head with the per-step tensors in HOST memory: h, temp, uniforms are copied
  * in and out_ids, out_logprobs copied back through staging areas in the workspace, all on
  * `stream`; the call returns after enqueueing (synchronise the stream before reading the
- * outputs).  W_trim and map are the resident model state and stay DEVICE pointers. */
+ * outputs).  W_trim and map are the resident model state and stay DEVICE pointers.  temp,
+ * out_ids and out_logprobs in page-locked (pinned) host memory are read and written in place by
+ * the kernels instead of being copied; pageable buffers work too and take the staging route. */
 vt_status vt_draft_head_host(const uint16_t *h_host, const uint16_t *W_trim, const int32_t *map,
                              int32_t B, int32_t K, int32_t d, const float *temp_host,
                              int32_t topk, const float *uniforms_host, int32_t *out_ids_host,

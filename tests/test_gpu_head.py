@@ -292,3 +292,28 @@ def test_all_candidates_in_one_slab_of_the_vocabulary():
     ref = oracle_head(h, W, None, T, topk, u)
     check_head(ref, gi, gl, T, None, lg, lse)
     assert set(gi[0, 1:].tolist()) <= set(range(3, 19))
+
+
+@pytest.mark.parametrize("pinned", [True, False])
+@pytest.mark.parametrize("B,K,d,topk,sample", [(1, 4099, 1024, 8, False), (10, 3000, 512, 10, True), (40, 700, 128, 4, True)])
+def test_host_entry_point_matches_device_entry_point(B, K, d, topk, sample, pinned):
+    """vt_draft_head_host with page-locked buffers (used in place by the kernels) and with pageable ones
+    (staged through the workspace) returns what vt_draft_head returns on device copies of the same data."""
+    W = vt_inputs.gaussian_bf16((K, d), 0.02, seed=K, device=DEV)
+    m = torch.randperm(K * 2, device=DEV)[:K].to(torch.int32)
+    h = vt_inputs.gaussian_bf16((B, d), 1.0, seed=B)
+    T = vt_inputs.temperatures(B, 0.5, 1.5, seed=d)
+    u = vt_inputs.uniforms((B, K), seed=3) if sample else None
+    out = (torch.full((B, 1 + topk), -7, dtype=torch.int32), torch.zeros((B, 1 + topk), dtype=torch.float32))
+    if pinned:
+        h, T = h.pin_memory(), T.pin_memory()
+        u = u.pin_memory() if u is not None else None
+        out = tuple(t.pin_memory() for t in out)
+    ws = vt.Workspace(vt.workspace_bytes(vt.VT_OP_DRAFT_HEAD_HOST, 0, 0, K, d, B, topk))
+    for _ in range(2):
+        ids, lps = vt.vt_draft_head_host(h, W, m, T, topk, u, ws, out)
+        torch.cuda.synchronize()
+        ref_ids, ref_lps = vt.vt_draft_head(h.to(DEV), W, m, T.to(DEV), topk, u.to(DEV) if u is not None else None)
+        assert torch.equal(ids, ref_ids.cpu())
+        assert torch.equal(lps.view(torch.int32), ref_lps.cpu().view(torch.int32))
+    assert ws.read_status() == (0, 0, 0)
