@@ -259,8 +259,8 @@ vt_status vt_draft_head(const uint16_t *h, const uint16_t *W_trim, const int32_t
  * dependent launch); it reads h, temp, uniforms, map and the workspace only after that earlier work
  * has completed.  The caller promises that W_trim was not written by work still pending on the
  * stream -- weights are static while drafting; after vt_trim_head, synchronise or make one plain
- * vt_draft_head call first.  Streaming kernel only (B <= 16 shapes); other shapes behave exactly
- * like vt_draft_head.
+ * vt_draft_head call first.  Both kernels take part: the dense kernel's first ring of W_trim tiles is
+ * requested early as well, and its merge kernel is chained the same way.
  */
 vt_status vt_draft_head_overlapped(const uint16_t *h, const uint16_t *W_trim, const int32_t *map,
                                    int32_t B, int32_t K, int32_t d, const float *temp, int32_t topk,
