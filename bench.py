@@ -37,8 +37,8 @@ if ROOT not in sys.path:
 import vt_inputs  # noqa: E402
 
 V = vt_inputs.LLAMA3_VOCAB
-HEAD = dict(d=3072, K=32768, B=1, topk=8, temp=1.0)            # BASELINE config 2 (chain drafting)
-TREE = dict(d=4096, B=10, topk=10, temp=0.7)                   # BASELINE config 3 (tree drafting)
+HEAD = dict(d=3072, K=32768, B=1, topk=8, temp=1.0)            # config 2: chain drafting
+TREE = dict(d=4096, B=10, topk=10, temp=0.7)                   # config 3: tree drafting
 TREE_KS = (8192, 16384, 32768, 65536, V)
 L2_BYTES = 126 * 1024 * 1024
 FALLBACK_HBM_GBS = 6650.0
@@ -418,7 +418,7 @@ def draft_block_case(vt, dev, timed):
     return out
 
 
-DENSE = dict(d=4096, K=32768, B=256, topk=8)                   # BASELINE config 4 (batched serving)
+DENSE = dict(d=4096, K=32768, B=256, topk=8)                   # config 4: batched serving
 
 
 def dense_case(vt, dev, steps=200, warmup=20):

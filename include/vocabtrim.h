@@ -10,8 +10,10 @@
  * Conventions (all entry points unless stated otherwise)
  *   - Every data pointer is a DEVICE pointer owned by the caller.  Entry points whose name ends
  *     in _host take HOST pointers where their comment says so.
- *   - The library allocates no device memory and keeps no global state.  Scratch comes from the
- *     caller: `ws` is a device buffer of at least vt_workspace_bytes(op, ...) bytes, 256-byte
+ *   - The library allocates no device memory.  The only process-wide state it keeps is host-side
+ *     bookkeeping (the launch counter behind vt_launch_count, the calling thread's last CUDA error,
+ *     per-device caches of the SM count and of kernel attributes) and the fixed device array of
+ *     vt_select_topk_static.  Scratch comes from the caller: `ws` is a device buffer of at least vt_workspace_bytes(op, ...) bytes, 256-byte
  *     aligned, whose first 256 bytes (the control block) must have been cleared ONCE by
  *     vt_workspace_init before its first use.  Every call leaves the control block ready for the
  *     next call.  One workspace serves one stream at a time.

@@ -258,9 +258,9 @@ def mbsu(tau: float, c: float, gamma: int) -> float:
     return float(tau) / (float(c) * float(gamma) + 1.0)
 
 
-# ---- draft-tree construction.  The paper takes "draft trees construction ... following EAGLE-2"
-# (Settings) with depth 3, top-K = 8 and at most 32 draft tokens (60 in the depth ablation); the steps
-# below restate that published procedure.  Scores are cumulative log-probabilities kept in fp32, the
+# ---- draft-tree construction.  Section 4.1 (Settings) adopts the EAGLE-2 tree procedure with depth 3,
+# top-K = 8 and at most 32 draft tokens (Table 4: 60 in the depth ablation); the steps below restate
+# that published procedure.  Scores are cumulative log-probabilities kept in fp32, the
 # precision the GPU path keeps them in, because they decide integers (which nodes are taken).
 
 def _score_order(score, index):

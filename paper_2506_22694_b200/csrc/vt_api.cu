@@ -37,10 +37,7 @@ inline vt_status from_cuda(cudaError_t e) {
 
 constexpr int64_t kHostChunkIds = 1 << 24;     // ids per staged chunk of vt_build_vocab_host
 
-bool hist_shape_ok(int32_t V) {
-    if (V < 1) return false;
-    return hist_plan(V).small || ((size_t)(V + 31) / 32 * 8 + 65536 <= (size_t)224 * 1024);
-}
+bool hist_shape_ok(int32_t V) { return hist_supported(V); }
 
 bool head_shape_ok(int32_t B, int32_t K, int32_t d, int32_t topk) {
     if (B < 1 || B > 256 || K < 1 || d < 8 || (d & 7) || topk < 1 || topk > VT_MAX_TOPK || topk > K)

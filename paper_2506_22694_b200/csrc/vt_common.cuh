@@ -33,6 +33,7 @@ struct HistPlan {
     size_t bytes;          // scratch after the control block
 };
 HistPlan hist_plan(int32_t V);
+bool hist_supported(int32_t V);   // V the counting kernels take (bins or lookup table fit shared memory)
 cudaError_t launch_histogram(const int32_t* ids, int64_t n, int32_t V, uint32_t* counts,
                              int accumulate, Ctrl* ctrl, uint8_t* scratch, cudaStream_t s);
 

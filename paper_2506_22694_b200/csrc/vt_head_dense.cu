@@ -368,7 +368,7 @@ k_head_dense(const HeadArgs a, Ctrl* ctrl, float* __restrict__ recs, const Dense
         float thr = -CUDART_INF_F;
 #pragma unroll
         for (int i = 0; i < KT; ++i) { st.tv[i] = (i < KT - topk) ? CUDART_INF_F : -CUDART_INF_F; st.tj[i] = -1; }
-        const bool vec_u = a.uniforms && ((K & 3) == 0);
+        const bool vec_u = a.uniforms && ((K & 3) == 0) && ((reinterpret_cast<uintptr_t>(a.uniforms) & 15) == 0);
         const bool use_u = row_live && a.uniforms != nullptr;
         const uint32_t acc_empty_bar = PAIR ? mapa_u32(smem_u32(&s_acc_empty[0]), 0) : 0u;
         float u[kCh];

@@ -18,6 +18,9 @@ namespace {
 
 constexpr int kThreads = 1024;
 constexpr size_t kDynSmem = 224 * 1024;        // dynamic shared memory of the counting kernels
+constexpr size_t kMaxTableBytes = 160 * 1024;  // lookup table (8 bytes per 32 ids) at most: leaves 64 KB of hot bins;
+                                               // the one limit behind hist_supported and both kernels' launches
+constexpr int kMaxDevices = 64;
 constexpr int kSampleSlots = 4096;             // aggregating cache of the sampling pre-pass
 constexpr int kSamplePerCta = 16384;           // ids sampled per CTA
 constexpr int kPickBins = 1024;                // sampled counts are clipped to kPickBins-1
@@ -281,6 +284,23 @@ k_hist_hot(const int32_t* __restrict__ ids, int64_t n, int32_t V, uint32_t* __re
 
 }  // namespace
 
+bool hist_supported(int32_t V) {
+    if (V < 1) return false;
+    if ((size_t)V * 4 <= kDynSmem) return true;
+    return ((size_t)V + 31) / 32 * 8 <= kMaxTableBytes;
+}
+
+// opt-in shared-memory sizes are per device: remember which devices have been set up
+static cudaError_t set_smem_once(const void* fn, size_t bytes, int (&done)[kMaxDevices]) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev >= 0 && dev < kMaxDevices && done[dev]) return cudaSuccess;
+    e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+    if (e == cudaSuccess && dev >= 0 && dev < kMaxDevices) done[dev] = 1;
+    return e;
+}
+
 HistPlan hist_plan(int32_t V) {
     HistPlan p{};
     p.small = (size_t)V * 4 <= kDynSmem;
@@ -307,38 +327,35 @@ cudaError_t launch_histogram(const int32_t* ids, int64_t n, int32_t V, uint32_t*
     if (grid > sms) grid = sms;
     if (grid < 1) grid = 1;
     if (p.small) {
-        static bool attr_done = false;
-        if (!attr_done) {
-            e = cudaFuncSetAttribute(k_hist_small, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     (int)kDynSmem);
-            if (e != cudaSuccess) return e;
-            attr_done = true;
-        }
+        static int done_small[kMaxDevices] = {0};
+        e = set_smem_once(reinterpret_cast<const void*>(k_hist_small), kDynSmem, done_small);
+        if (e != cudaSuccess) return e;
         k_hist_small<<<grid, kThreads, (size_t)V * 4, s>>>(ids, n, V, counts, ctrl);
         count_launch();
         return cudaGetLastError();
     }
     const size_t T32 = ((size_t)V + 31) / 32;
-    if (T32 * 8 + 4096 > kDynSmem) return cudaErrorInvalidValue;   // rejected earlier by the API
+    if (T32 * 8 > kMaxTableBytes) return cudaErrorInvalidValue;   // rejected earlier by the API
     int32_t H = (int32_t)((kDynSmem - T32 * 8) / 4);
     if (H > 65535) H = 65535;                          // slots are 16-bit in the main pass's lookup
     uint32_t* sample = reinterpret_cast<uint32_t*>(scratch + p.off_sample);
     uint2* table = reinterpret_cast<uint2*>(scratch + p.off_table);
     e = cudaMemsetAsync(sample, 0, (size_t)V * 4, s);
     if (e != cudaSuccess) return e;
-    static bool attr_done_hot = false;
-    if (!attr_done_hot) {
-        e = cudaFuncSetAttribute(k_hist_pick, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(kDynSmem / 2));
-        if (e != cudaSuccess) return e;
-        e = cudaFuncSetAttribute(k_hist_hot, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)kDynSmem);
-        if (e != cudaSuccess) return e;
-        attr_done_hot = true;
-    }
+    static int done_pick[kMaxDevices] = {0}, done_hot[kMaxDevices] = {0};
+    e = set_smem_once(reinterpret_cast<const void*>(k_hist_pick), kMaxTableBytes, done_pick);
+    if (e != cudaSuccess) return e;
+    e = set_smem_once(reinterpret_cast<const void*>(k_hist_hot), kDynSmem, done_hot);
+    if (e != cudaSuccess) return e;
+    // a refused launch must stop the chain: the main pass would count through an unwritten table
     k_hist_sample<<<grid, kThreads, 0, s>>>(ids, n, V, sample);
+    count_launch();
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
     k_hist_pick<<<1, kThreads, T32 * 8, s>>>(sample, V, H, table);
+    count_launch();
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
     k_hist_hot<<<grid, kThreads, kDynSmem, s>>>(ids, n, V, counts, table, H, ctrl);
-    count_launch(3);
+    count_launch();
     return cudaGetLastError();
 }
 

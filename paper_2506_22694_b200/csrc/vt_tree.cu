@@ -1,5 +1,5 @@
-// Draft-tree construction around the head (Settings: "draft trees construction ... following EAGLE-2",
-// depth 3 / top-K 8 / 32 draft tokens, 60 in the depth ablation).  Two on-chip selections over at most
+// Draft-tree construction around the head (Section 4.1, Settings: the EAGLE-2 tree procedure with
+// depth 3 / top-K 8 / 32 draft tokens; Table 4: 60 draft tokens in the depth ablation).  Two on-chip selections over at most
 // a few thousand values: the frontier of the next depth, and the final rerank of the node pool.
 // Scores are cumulative log-probabilities in fp32; ties go to the lower node index; NaN ranks last.
 #include "vt_common.cuh"

@@ -4,6 +4,9 @@ Tolerances (stated by the benchmark spec, written out here):
   * histograms, map, inv_map, gathered rows: bit-exact;
   * logits: |err| <= 1e-3 + 1e-3 * |ref|;
   * probabilities exp(logprob): within 1e-5 absolute of the oracle's value for the same index;
+  * log-probabilities themselves: |logp - ref| <= 2e-3, which is what the logit tolerance (1e-3 in z at
+    T = 1, the lse being an average of the same errors) already implies; the probability test alone
+    is blind at p ~ 1e-5, where a sampled id of a 32768-row head lives;
   * greedy / top-k / Gumbel ids: equal to the oracle's, except where the oracle's own margin
     between the two competing candidates is below 1e-3 in logit units, i.e.
     T_b * |score_ref[oracle choice] - score_ref[gpu choice]| < 1e-3 with score = z for candidates
@@ -18,6 +21,7 @@ import oracle
 LOGIT_ATOL = 1e-3
 LOGIT_RTOL = 1e-3
 PROB_ATOL = 1e-5
+LOGP_ATOL = 2e-3
 MARGIN = 1e-3
 
 
@@ -57,8 +61,10 @@ def check_head(ref, gpu_ids, gpu_lps, temp, map_, gpu_logits=None, gpu_lse=None,
                 gap = T[b] * abs(score[jo] - score[jg])
                 assert gap < MARGIN, "row %d col %d: gpu %d vs oracle %d, logit margin %.3e" % (b, c, jg, jo, gap)
                 slack += 1
-            p_ref = np.exp(ref.z[b, jg] - ref.lse[b])
-            assert abs(np.exp(lps[b, c]) - p_ref) <= PROB_ATOL, "row %d col %d: probability off" % (b, c)
+            lp_ref = ref.z[b, jg] - ref.lse[b]
+            assert abs(np.exp(lps[b, c]) - np.exp(lp_ref)) <= PROB_ATOL, "row %d col %d: probability off" % (b, c)
+            assert abs(lps[b, c] - lp_ref) <= LOGP_ATOL, \
+                "row %d col %d: log-prob %.6f vs %.6f" % (b, c, lps[b, c], lp_ref)
     if gpu_logits is not None:
         lg = gpu_logits.cpu().numpy().astype(np.float64)
         err = np.abs(lg - ref.logits)

@@ -54,6 +54,10 @@ def test_workspace_bytes(lib):
     host = vt.workspace_bytes(vt.VT_OP_DRAFT_HEAD_HOST, 0, 0, 32768, 4096, 10, 10)
     assert host >= vt.workspace_bytes(vt.VT_OP_DRAFT_HEAD, 0, 0, 32768, 4096, 10, 10) + 10 * 32768 * 4
     assert vt.workspace_bytes(12345) == 0
+    # largest vocabulary the histogram takes: its lookup table (8 bytes per 32 ids) may use 160 KB
+    assert vt.workspace_bytes(vt.VT_OP_HISTOGRAM, 100, 655_360) > 256
+    assert vt.workspace_bytes(vt.VT_OP_HISTOGRAM, 100, 655_361) == 0
+    assert vt.workspace_bytes(vt.VT_OP_BUILD_VOCAB, 100, 655_361, 10) == 0
 
 
 def test_argument_errors_return_before_any_cuda_call(lib):

@@ -123,6 +123,16 @@ def test_bad_temperature_is_flagged_not_fatal():
     assert ws.read_status()[0] == 0 and int(gi2.min()) >= 0
 
 
+SLACK = {}            # workload -> [positions accepted through the margin rule, positions compared]
+
+
+def _tally(name, slack, positions):
+    acc = SLACK.setdefault(name, [0, 0])
+    acc[0] += slack
+    acc[1] += positions
+    print("parity_slack %s: %d of %d positions accepted through the 1e-3 logit margin" % (name, slack, positions))
+
+
 def test_config2_chain_drafting_trimmed_vs_full_head():
     """V=128256, d=3072, K=32768, B=1, 7 sequential steps, greedy + top-8, against the full head."""
     d, K, topk, steps = 3072, 32768, 8, 7
@@ -133,34 +143,38 @@ def test_config2_chain_drafting_trimmed_vs_full_head():
     ws = vt.Workspace(vt.workspace_bytes(vt.VT_OP_DRAFT_HEAD, 0, 0, V3, d, 1, topk))
     Wb = vt_inputs.bf16_bits(W).cpu().numpy().view(np.uint16)
     mh = m.cpu().numpy()
+    slack = 0
     for step in range(steps):
         h = vt_inputs.gaussian_bf16((1, d), 1.0, seed=2000 + step, device=DEV)
         gi, gl, lg, lse = _run(h, Wt, m, T, topk, None, ws=ws)
         ref = oracle_head(h, Wt, m, T, topk, None)
-        check_head(ref, gi, gl, T, m, lg, lse, sampled=False)
+        slack += check_head(ref, gi, gl, T, m, lg, lse, sampled=False)
         fi, fl, flg, flse = _run(h, W, None, T, topk, None, ws=ws)            # full K = V head, identity map
         if step < 2:
             full = oracle_head(h, W, None, T, topk, None)
-            check_head(full, fi, fl, T, None, flg, flse, sampled=False)
+            slack += check_head(full, fi, fl, T, None, flg, flse, sampled=False)
             # trimmed logits are the full head's logits at the mapped rows (oracle: exactly)
             assert np.array_equal(ref.logits[0], full.logits[0, mh])
         assert torch.allclose(lg[0], flg[0, m.long()], rtol=0, atol=2e-5)
+    _tally("config2 K=32768 and K=V", slack, (steps + 2) * (1 + topk))
+    assert slack <= 1
     assert ws.read_status() == (0, 0, 0)
 
 
-@pytest.mark.parametrize("K", [8192, 32768, V3])
+@pytest.mark.parametrize("K", [8192, 16384, 32768, 65536, V3])
 def test_config3_tree_drafting_sweep(K):
-    """V=128256, d=4096, B=10 nodes, top-10, T=0.7, Gumbel sampling; K = V uses the identity map."""
-    d, B, topk = 4096, 10, 10
+    """V=128256, d=4096, B=10 nodes, top-10, T=0.7, Gumbel sampling, 6 tree depths at every K of the
+    sweep; K = V uses the identity map.  Every logit, log-probability and id meets the oracle."""
+    d, B, topk, depths = 4096, 10, 10, 6
     W = vt_inputs.gaussian_bf16((V3, d), 0.02, seed=1003, device=DEV)
     if K == V3:
         m, Wt = None, W
     else:
         m, _ = _vocab_map(V3, K, seed=1103)
         Wt = vt.vt_trim_head(W, m)
+        del W
     T = vt_inputs.temperatures(B, 0.7, 0.7, 0, device=DEV)
     ws = vt.Workspace(vt.workspace_bytes(vt.VT_OP_DRAFT_HEAD, 0, 0, K, d, B, topk))
-    depths = 6 if K == 8192 else 2
     slack = 0
     for depth in range(depths):
         h = vt_inputs.gaussian_bf16((B, d), 1.0, seed=3000 + depth, device=DEV)
@@ -168,7 +182,12 @@ def test_config3_tree_drafting_sweep(K):
         gi, gl, lg, lse = _run(h, Wt, m, T, topk, u, ws=ws)
         ref = oracle_head(h, Wt, m, T, topk, u)
         slack += check_head(ref, gi, gl, T, m, lg, lse)
-    assert slack <= 0.02 * depths * B * (1 + topk)
+        # the timed entry point (no logits written) returns the same bits
+        gi2, gl2 = _run(h, Wt, m, T, topk, u, debug=False, ws=ws)
+        assert torch.equal(gi, gi2) and torch.equal(gl, gl2)
+    positions = depths * B * (1 + topk)
+    _tally("config3 K=%d" % K, slack, positions)
+    assert slack <= 0.005 * positions + 1
     assert ws.read_status() == (0, 0, 0)
 
 
@@ -197,6 +216,23 @@ def test_dense_path_small_shapes_and_ragged_tails(B, K, d, topk, sample):
     assert torch.equal(a[0], gi) and torch.equal(b[0], gi) and torch.equal(a[1], b[1])
 
 
+def test_dense_path_uniforms_need_no_16_byte_alignment():
+    """The header asks 16-byte alignment of the bf16 tensors only: a [B,K] fp32 view that starts 4 bytes
+    into an allocation must give the result of an aligned copy."""
+    B, K, d, topk = 40, 1000, 256, 8
+    W = vt_inputs.gaussian_bf16((K, d), 0.02, seed=11, device=DEV)
+    h = vt_inputs.gaussian_bf16((B, d), 1.0, seed=12, device=DEV)
+    T = vt_inputs.temperatures(B, 0.5, 1.5, seed=13, device=DEV)
+    u = vt_inputs.uniforms((B, K), seed=14, device=DEV)
+    flat = torch.empty(B * K + 1, dtype=torch.float32, device=DEV)
+    shifted = flat[1:].view(B, K)
+    shifted.copy_(u)
+    assert shifted.data_ptr() % 16 == 4
+    a = _run(h, W, None, T, topk, u, debug=False)
+    b = _run(h, W, None, T, topk, shifted, debug=False)
+    assert torch.equal(a[0], b[0]) and torch.equal(a[1], b[1])
+
+
 def test_dense_path_rejects_long_candidate_lists():
     W = vt_inputs.gaussian_bf16((256, 64), 0.02, seed=1, device=DEV)
     h = vt_inputs.gaussian_bf16((32, 64), 1.0, seed=2, device=DEV)
@@ -207,8 +243,9 @@ def test_dense_path_rejects_long_candidate_lists():
 
 def test_config4_batched_serving_dense_head():
     """64 sequences x 4 tree nodes = 256 rows, d=4096, V=128256, K=32768, per-row T in [0.5,1.5],
-    top-8, Gumbel sampling.  The oracle checks every row on a 4096-row slice of the trimmed head
-    (all logits) and a sample of rows on the full K (ids, log-probs)."""
+    top-8, Gumbel sampling.  All 256 rows meet the oracle at the full K in the launch configuration the
+    benchmark times (ids, log-probabilities); the logits themselves are compared on a 4096-row slice
+    of the trimmed head (a full dump would be 33 MB of fp32 per call for no extra coverage)."""
     d, K, B, topk = 4096, 32768, 256, 8
     m, _ = _vocab_map(V3, K, seed=1104)
     W = vt_inputs.gaussian_bf16((V3, d), 0.02, seed=1004, device=DEV)
@@ -224,19 +261,16 @@ def test_config4_batched_serving_dense_head():
     gi, gl, lg, lse = _run(h, Wt[:Ks], m[:Ks], T, topk, us, ws=ws)
     ref = oracle_head(h, Wt[:Ks], m[:Ks], T, topk, us)
     slack = check_head(ref, gi, gl, T, m[:Ks], lg, lse)
-    assert slack <= 0.02 * B * (1 + topk)
-    # full size, launch configuration of the benchmark: sampled rows against the oracle
+    _tally("config4 slice K=4096", slack, B * (1 + topk))
+    assert slack <= 0.005 * B * (1 + topk) + 1
+    # full size, launch configuration of the benchmark: every row against the oracle
     gi, gl = _run(h, Wt, m, T, topk, u, debug=False, ws=ws)
-    rows = [0, 1, 31, 32, 127, 128, 200, 255]
-    ref = oracle_head(h[rows], Wt, m, T[rows], topk, u[rows])
-    check_head(ref, gi[rows], gl[rows], T[rows], m)
-    # every row: ids are members of the map, candidates distinct and ordered by log-prob
-    mm = set(m.cpu().numpy().tolist())
-    ids, lps = gi.cpu().numpy(), gl.cpu().numpy()
-    for b in range(B):
-        assert all(int(x) in mm for x in ids[b])
-        assert len(set(ids[b, 1:].tolist())) == topk
-        assert np.all(np.diff(lps[b, 1:]) <= 1e-6)
+    ref = oracle_head(h, Wt, m, T, topk, u)
+    slack = check_head(ref, gi, gl, T, m)
+    _tally("config4 K=32768", slack, B * (1 + topk))
+    assert slack <= 0.005 * B * (1 + topk) + 1
+    gi2, gl2 = _run(h, Wt, m, T, topk, u, debug=False, ws=ws)
+    assert torch.equal(gi, gi2) and torch.equal(gl, gl2)                  # bitwise run-to-run
     assert ws.read_status() == (0, 0, 0)
 
 
@@ -317,3 +351,14 @@ def test_host_entry_point_matches_device_entry_point(B, K, d, topk, sample, pinn
         assert torch.equal(ids, ref_ids.cpu())
         assert torch.equal(lps.view(torch.int32), ref_lps.cpu().view(torch.int32))
     assert ws.read_status() == (0, 0, 0)
+
+
+def test_zz_parity_slack_report():
+    """Totals of the margin-rule acceptances over the full-size configurations run above (printed with
+    -s or -rP); the expectation is a handful at most, since a GPU id differs from the oracle's only
+    where fp32 rounding flips two candidates whose fp64 scores are within ~1e-5."""
+    for name in sorted(SLACK):
+        print("parity_slack total %s: %d of %d" % (name, SLACK[name][0], SLACK[name][1]))
+    tot = sum(v[0] for v in SLACK.values())
+    pos = sum(v[1] for v in SLACK.values())
+    assert tot <= 0.005 * pos + 1

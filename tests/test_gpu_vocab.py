@@ -22,7 +22,8 @@ def _assert_clean(ws):
 
 
 @pytest.mark.parametrize("n,V", [(0, 4096), (1, 4096), (7, 100), (100_000, 4096), (250_003, 50_000),
-                                 (1_000_003, 128256), (3_000_000, 57_345), (777, 128256)])
+                                 (1_000_003, 128256), (3_000_000, 57_345), (777, 128256),
+                                 (2_000_000, 655_360), (500_000, 300_001)])
 def test_histogram_matches_oracle(n, V):
     ids = vt_inputs.zipf_ids(n, V, 1.1, seed=100 + n % 97, noise_frac=0.05, device=DEV) if n else \
         torch.empty(0, dtype=torch.int32, device=DEV)
