@@ -303,6 +303,18 @@ vt_status vt_draft_head_host(const uint16_t *h_host, const uint16_t *W_trim, con
                              int32_t topk, const float *uniforms_host, int32_t *out_ids_host,
                              float *out_logprobs_host, void *ws, size_t ws_bytes, void *stream);
 
+#ifdef VT_STAMPS
+/*
+ * Instrumented builds only (compiled with -DVT_STAMPS; the regular library does not export it).  The
+ * streaming head kernel then writes a nanosecond clock stamp per CTA at fixed phases of Algorithm 2's
+ * head step (entry, ring requested, released by the launch dependency, first stage landed, last stage
+ * consumed, record written, fence, ticket, merge loads / selection / outputs) into the workspace:
+ * 8-byte words [max_ctas][slots] at byte `offset` of `ws`.  Returns 0 for shapes the streaming kernel
+ * does not take.  Pure host arithmetic.
+ */
+int32_t vt_stamps_region(int32_t B, int32_t d, int32_t topk, size_t *offset, int32_t *slots, int32_t *max_ctas);
+#endif
+
 #ifdef __cplusplus
 }
 #endif

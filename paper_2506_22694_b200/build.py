@@ -14,6 +14,8 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libvocabtrim.so")
 OBJ_DIR = os.path.join(HERE, "_build")
+LIB_STAMPS = os.path.join(HERE, "libvocabtrim_stamps.so")     # -DVT_STAMPS: phase stamps in the head kernel
+OBJ_DIR_STAMPS = os.path.join(HERE, "_build_stamps")
 
 NVCC_FLAGS = [
     "-O3", "-std=c++17", "-lineinfo",
@@ -31,20 +33,22 @@ def _deps():
     return _sources() + glob.glob(os.path.join(CSRC, "*.cuh")) + glob.glob(os.path.join(ROOT, "include", "*.h"))
 
 
-def needs_build() -> bool:
-    if not os.path.exists(LIB):
+def needs_build(lib: str = LIB) -> bool:
+    if not os.path.exists(lib):
         return True
-    t = os.path.getmtime(LIB)
+    t = os.path.getmtime(lib)
     return any(os.path.getmtime(p) > t for p in _deps())
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    """Compile every .cu under csrc/ (one object each, in parallel) and link the shared library."""
-    if not force and not needs_build():
+def build(force: bool = False, verbose: bool = False, stamps: bool = False) -> str:
+    """Compile every .cu under csrc/ (one object each, in parallel) and link the shared library.
+    stamps=True builds the instrumented twin (libvocabtrim_stamps.so, -DVT_STAMPS) instead."""
+    LIB, OBJ_DIR = (LIB_STAMPS, OBJ_DIR_STAMPS) if stamps else (globals()["LIB"], globals()["OBJ_DIR"])
+    if not force and not needs_build(LIB):
         return LIB
     nvcc = os.environ.get("NVCC", "nvcc")
     os.makedirs(OBJ_DIR, exist_ok=True)
-    extra = ["-Xptxas", "-v"] if verbose else []
+    extra = (["-Xptxas", "-v"] if verbose else []) + (["-DVT_STAMPS"] if stamps else [])
     procs, objs = [], []
     hdr_time = max(os.path.getmtime(p) for p in _deps() if not p.endswith(".cu"))
     for src in _sources():
@@ -70,4 +74,4 @@ def build(force: bool = False, verbose: bool = False) -> str:
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="--verbose" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="--verbose" in sys.argv, stamps="--stamps" in sys.argv))

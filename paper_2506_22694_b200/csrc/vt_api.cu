@@ -154,6 +154,16 @@ const char* vt_status_str(vt_status s) {
     }
 }
 
+#ifdef VT_STAMPS
+int32_t vt_stamps_region(int32_t B, int32_t d, int32_t topk, size_t* offset, int32_t* slots, int32_t* max_ctas) {
+    if (!head_skinny_supported(B, d) || !offset || !slots || !max_ctas) return 0;
+    *offset = VT_CTRL_BYTES + head_skinny_stamps_offset(B, topk);
+    *slots = 16;
+    *max_ctas = 160;
+    return 1;
+}
+#endif
+
 uint64_t vt_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
 const char* vt_last_cuda_error(void) { return cudaGetErrorString(t_last_cuda); }

@@ -24,6 +24,9 @@ int num_sms();                    // SM count of the current device (cached per 
 void count_launch(int n = 1);     // host-side launch counter behind vt_launch_count
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+#ifdef __CUDACC__
+__device__ __forceinline__ size_t align_up_dev(size_t x, size_t a) { return (x + a - 1) / a * a; }
+#endif
 
 // ---- launchers implemented in the .cu files (host functions) --------------------------------
 struct HistPlan {
@@ -86,6 +89,9 @@ struct HeadArgs {
 bool head_skinny_supported(int32_t B, int32_t d);
 size_t head_skinny_scratch_bytes(int32_t B, int32_t K, int32_t topk);
 cudaError_t launch_head_skinny(const HeadArgs& a, Ctrl* ctrl, uint8_t* scratch, cudaStream_t s);
+#ifdef VT_STAMPS
+size_t head_skinny_stamps_offset(int32_t B, int32_t topk);   // offset of the phase stamps in the head scratch
+#endif
 
 bool head_dense_supported(int32_t B, int32_t K, int32_t d);
 bool head_dense_topk_ok(int32_t topk);

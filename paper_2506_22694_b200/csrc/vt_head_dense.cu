@@ -447,6 +447,10 @@ k_head_dense(const HeadArgs a, Ctrl* ctrl, float* __restrict__ recs, const Dense
                     // last entry.  The loop is warp-uniform (it runs while any row of the warp still has
                     // a candidate) and everything inside is select-based: one row's insertions never
                     // make the other 31 rows branch.
+                    // a NaN logit poisons the row's lse (reported through VT_FLAG_NAN_ROW) but must not hide the
+                    // chunk's other candidates: it competes as -inf
+#pragma unroll
+                    for (int i = 0; i < kCh; ++i) z[i] = (z[i] == z[i]) ? z[i] : -CUDART_INF_F;
                     float mx = z[0];
                     int mi = 0;
 #pragma unroll
@@ -517,19 +521,17 @@ k_head_dense(const HeadArgs a, Ctrl* ctrl, float* __restrict__ recs, const Dense
                 }
             }
             // ---- this CTA's record of hidden row b ---------------------------------------------------------
-            int* irecs = reinterpret_cast<int*>(recs);
+            unsigned long long* kp = rec_keys(recs, b, topk);
+            float* fp = rec_f32(recs, b, topk);
             const int c = group;
-            recs[rec_at(b, 0, topk) + c] = st.m;
-            recs[rec_at(b, 1, topk) + c] = st.s;
-            recs[rec_at(b, 2, topk) + c] = st.gb_s;
-            irecs[rec_at(b, 3, topk) + c] = st.gb_j;
-            recs[rec_at(b, 4, topk) + c] = st.gb_z;
+            fp[c] = st.m;
+            fp[kMaxGrid + c] = st.s;
+            fp[2 * kMaxGrid + c] = st.gb_z;
+            kp[c] = st.gb_j >= 0 ? key64(st.gb_s, st.gb_j) : 0ull;
 #pragma unroll
             for (int p = 0; p < KT; ++p)
-                if (p >= KT - topk) {
-                    recs[rec_at(b, 5 + p - (KT - topk), topk) + c] = st.tv[p];
-                    irecs[rec_at(b, 5 + topk + p - (KT - topk), topk) + c] = st.tj[p];
-                }
+                if (p >= KT - topk)
+                    kp[(size_t)(1 + p - (KT - topk)) * kMaxGrid + c] = st.tj[p] >= 0 ? key64(st.tv[p], st.tj[p]) : 0ull;
         }
     }
     tc_fence_before();
@@ -543,17 +545,18 @@ k_head_dense(const HeadArgs a, Ctrl* ctrl, float* __restrict__ recs, const Dense
     if (threadIdx.x == 0 && s_abort) atomicOr(&ctrl->flags, (uint32_t)VT_FLAG_TIMEOUT);
 }
 
-// One warp per hidden row: merge the CTA records, remap, write the outputs.
-__global__ void __launch_bounds__(32)
-k_head_merge(const HeadArgs a, Ctrl* ctrl, const float* __restrict__ recs, int G) {
-    __shared__ float s_stage[kMergeStageWords];
+// Two warps per hidden row (candidates / statistics): merge the CTA records, remap, write the outputs.
+__global__ void __launch_bounds__(64)
+k_head_merge(const HeadArgs a, Ctrl* ctrl, float* __restrict__ recs, int G) {
+    __shared__ __align__(8) float s_stage[kMergeStageWords];
+    __shared__ float s_xch;
     const int b = blockIdx.x;
     griddep_launch_dependents();                                  // the next step may start fetching its weights
     griddep_wait();                                               // the records are complete
     const float T = a.temp[b];
     const bool row_ok = (T > 0.f) && (T < CUDART_INF_F);
-    merge_records(a.map, a.out_ids, a.out_logprobs, a.dbg_lse, a.topk, a.uniforms != nullptr, ctrl, recs, b, row_ok, G,
-                  s_stage);
+    const MergeOut mo{a.map, a.out_ids, a.out_logprobs, a.dbg_lse, a.topk, a.uniforms != nullptr};
+    merge_records(mo, ctrl, recs, b, row_ok, G, s_stage, threadIdx.x < 32 ? kRoleCand : kRoleStats, &s_xch, 1);
 }
 
 // ---- host side ----------------------------------------------------------------------------------------
@@ -671,7 +674,7 @@ cudaError_t launch_head_dense(const HeadArgs& a, Ctrl* ctrl, uint8_t* scratch, c
     // the merge always follows its own producer closely: it takes its seats early and waits on the device
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3((unsigned)a.B);
-    cfg.blockDim = dim3(32);
+    cfg.blockDim = dim3(64);
     cfg.stream = s;
     cudaLaunchAttribute at{};
     at.id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -679,7 +682,7 @@ cudaError_t launch_head_dense(const HeadArgs& a, Ctrl* ctrl, uint8_t* scratch, c
     cfg.attrs = &at;
     cfg.numAttrs = 1;
     count_launch(2);
-    e = cudaLaunchKernelEx(&cfg, k_head_merge, a, ctrl, static_cast<const float*>(recs), geo.n_groups);
+    e = cudaLaunchKernelEx(&cfg, k_head_merge, a, ctrl, recs, geo.n_groups);
     if (e != cudaSuccess || !a.tree.pool_token) return e;
     // tree drafting: the expansion needs every row's merge, i.e. the whole merge grid: one more launch
     return launch_tree_expand(a.out_ids, a.out_logprobs, a.B, a.topk, 1 + a.topk, 1, a.tree, s);

@@ -46,6 +46,16 @@ constexpr int kSelPerLane = (VT_MAX_TOPK + kCand) / 32;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 
 
+// Phase stamps (-DVT_STAMPS builds only): thread 0 of every CTA writes %globaltimer at fixed points into
+// a region behind the records; bench.py --case stamps reads them back.  Slots: 0 entry, 1 ring fill
+// requested, 2 released by the launch dependency, 3 first stage landed, 4 last stage consumed,
+// 5 record written, 6 after the fence, 7 after the ticket, 8-10 merge (loads, selection, outputs), 11 SM id.
+#ifdef VT_STAMPS
+#define VT_STAMP(slot) do { if (threadIdx.x == 0) stamps[(size_t)blockIdx.x * kStampSlots + (slot)] = global_ns(); } while (0)
+#else
+#define VT_STAMP(slot) do {} while (0)
+#endif
+
 struct Geo {
     int RB;            // row blocks of 8 vocabulary rows
     int S;             // ring stages
@@ -93,9 +103,10 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* b, uint32_t parity, volatile
     }
     return __all_sync(0xffffffffu, ok);
 }
-__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint64_t* bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(dst), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
+// bulk copy global -> shared with an L2 eviction-priority hint for the lines it brings in
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint64_t* bar, uint64_t pol) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(smem_u32(bar)), "l"(pol) : "memory");
 }
 __device__ __forceinline__ uint4 lds_u4(uint32_t addr) {
     uint4 v;
@@ -176,6 +187,8 @@ k_head_stream(const HeadArgs a, Ctrl* ctrl, float* __restrict__ recs, const Geo 
     extern __shared__ __align__(128) uint8_t s_raw[];
     __shared__ uint64_t s_full[kMaxStages], s_empty[kMaxStages], s_pfull[2], s_pempty[2];
     __shared__ int s_last, s_abort;
+    __shared__ int s_rowok[kMaxB];                       // per hidden row: its temperature is usable
+    __shared__ float s_xch[kMaxB];                       // merge: a row's lse, from its statistics warp to its candidate warp
     constexpr int KC = kNW * KBC * 32;                   // columns per chunk
     const int B = a.B, K = a.K, d = a.d, topk = a.topk;
     const int S = geo.S, pitch = geo.pitch, PT = geo.part_stride;
@@ -189,6 +202,15 @@ k_head_stream(const HeadArgs a, Ctrl* ctrl, float* __restrict__ recs, const Geo 
 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int g = lane >> 2, t = lane & 3;
+#ifdef VT_STAMPS
+    unsigned long long* stamps = reinterpret_cast<unsigned long long*>(
+        reinterpret_cast<uint8_t*>(recs) + align_up_dev((size_t)kMaxGrid * B * rec_fields(topk) * 4, 256));
+    if (threadIdx.x == 0) {
+        unsigned smid;
+        asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
+        stamps[(size_t)blockIdx.x * kStampSlots + 11] = smid;
+    }
+#endif
     const int rb0 = (int)((long long)geo.RB * blockIdx.x / gridDim.x);
     const int rb1 = (int)((long long)geo.RB * (blockIdx.x + 1) / gridDim.x);
 
@@ -200,6 +222,7 @@ k_head_stream(const HeadArgs a, Ctrl* ctrl, float* __restrict__ recs, const Geo 
     }
     for (int i = threadIdx.x; i < B * topk; i += kThreads) { topv[i] = -CUDART_INF_F; topj[i] = -1; }
     __syncthreads();
+    VT_STAMP(0);
     volatile int* abort_flag = &s_abort;
 
     // per-row state of warp b (identical in its four 8-lane groups); declared here so that the
@@ -214,6 +237,10 @@ k_head_stream(const HeadArgs a, Ctrl* ctrl, float* __restrict__ recs, const Geo 
     // ---- producer duty: one bulk copy per vocabulary row of a stage (lanes 0..7 of the duty warp) ----
     // Every warp tracks the fetch sequence; fetch f is issued by one warp of the duty group (the
     // warps that own no hidden row, so the epilogue warps are spared), in rotation.
+    // W_trim is read once per step: its lines are the first to go when L2 needs room, so that the
+    // records, the index mapper and h stay resident from step to step
+    uint64_t w_policy;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(w_policy));
     const int n_items = (rb1 - rb0) * NCH;
     const int n_duty = (B < kNW) ? kNW - B : 1;
     int f_item = 0, f_rb = rb0, f_c = 0, f_s = 0, f_duty = kNW - 1;   // next item to fetch, its duty warp
@@ -230,7 +257,7 @@ k_head_stream(const HeadArgs a, Ctrl* ctrl, float* __restrict__ recs, const Geo 
                 __syncwarp();
                 if (lane < nrows)
                     bulk_g2s(smem_u32(ring + (size_t)f_s * stage_bytes + lane * pitch),
-                             a.W + (size_t)(f_rb * kRows + lane) * d + col0, cbytes, &s_full[f_s]);
+                             a.W + (size_t)(f_rb * kRows + lane) * d + col0, cbytes, &s_full[f_s], w_policy);
             }
         }
         ++f_item;
@@ -240,12 +267,14 @@ k_head_stream(const HeadArgs a, Ctrl* ctrl, float* __restrict__ recs, const Geo 
         return ok;
     };
     for (int i = 0; i < S && f_item < n_items; ++i) fetch_next();          // fill the ring (no waits)
+    VT_STAMP(1);
 
     // Programmatic dependent launch (a no-op unless the launch asked for it): the next kernel on the
     // stream may become resident as soon as SMs free up, and this kernel goes no further than
     // fetching weights until everything enqueued before it has completed and is visible.
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     asm volatile("griddepcontrol.wait;" ::: "memory");
+    VT_STAMP(2);
 
     // ---- h fragments of this warp's columns, straight from global memory into registers ----------
     uint4 hl[NCH][KBC], hh[NCH][KBC];
@@ -266,6 +295,7 @@ k_head_stream(const HeadArgs a, Ctrl* ctrl, float* __restrict__ recs, const Geo 
         const float T = a.temp[b];
         row_ok = (T > 0.f) && (T < CUDART_INF_F);
         invT = row_ok ? 1.f / T : CUDART_NAN_F;
+        if (lane == 0) s_rowok[b] = row_ok ? 1 : 0;
     }
     float thr = -CUDART_INF_F;                              // k-th best so far (warp uniform)
     int tk_cnt = 0, n_cand = 0;
@@ -296,6 +326,9 @@ k_head_stream(const HeadArgs a, Ctrl* ctrl, float* __restrict__ recs, const Geo 
 #pragma unroll
                 for (int c = 0; c < NCH; ++c) {
                     if (!alive || !mbar_wait(&s_full[s], ph, abort_flag)) { alive = false; continue; }
+#ifdef VT_STAMPS
+                    if (item == 0) VT_STAMP(3);
+#endif
                     const uint32_t base = ring_u32 + (uint32_t)s * (uint32_t)stage_bytes + lane_off;
                     uint4 w[KBC];
 #pragma unroll
@@ -386,6 +419,7 @@ k_head_stream(const HeadArgs a, Ctrl* ctrl, float* __restrict__ recs, const Geo 
             }
         }
     }
+    VT_STAMP(4);
     if (warp == kNW - 1 && *abort_flag) {
         // drain: every stage that was filled must have landed before the CTA may leave
         const int back = min(f_item, S);
@@ -403,44 +437,63 @@ k_head_stream(const HeadArgs a, Ctrl* ctrl, float* __restrict__ recs, const Geo 
                                             candj + b * kCand, n_cand, topk);
             tk_cnt = ts.cnt;
         }
-        // lanes sharing a logit hold identical state: fold the 8R distinct lanes only
+        // Fold the lanes (those sharing a logit hold identical state: only the 8R distinct ones add to the
+        // sum): the maximum by one warp reduction, every lane's sum rescaled to it once, a butterfly of
+        // additions; the Gumbel candidate by two reductions over its 64-bit key.
+        const float Mall = ord2f(__reduce_max_sync(0xffffffffu, f2ord(st_m)));
+        float sc = (lane < 8 * (TWO ? 2 : 4) && st_m != -CUDART_INF_F) ? st_s * __expf(st_m - Mall) : 0.f;
 #pragma unroll
-        for (int o = 1; o < 8 * (TWO ? 2 : 4); o <<= 1) {
-            const float m2 = __shfl_xor_sync(0xffffffffu, st_m, o);
-            const float s2 = __shfl_xor_sync(0xffffffffu, st_s, o);
-            lse_merge(st_m, st_s, m2, s2);
-            const float gs2 = __shfl_xor_sync(0xffffffffu, gb_s, o);
-            const float gz2 = __shfl_xor_sync(0xffffffffu, gb_z, o);
-            const int gj2 = __shfl_xor_sync(0xffffffffu, gb_j, o);
-            if (gj2 >= 0 && (gb_j < 0 || better(gs2, gj2, gb_s, gb_j))) { gb_s = gs2; gb_j = gj2; gb_z = gz2; }
-        }
-        int* irecs = reinterpret_cast<int*>(recs);
+        for (int o = 16; o; o >>= 1) sc += __shfl_xor_sync(0xffffffffu, sc, o);
+        const unsigned long long gk = gb_j >= 0 ? key64(gb_s, gb_j) : 0ull;
+        const unsigned ghi = (unsigned)(gk >> 32);
+        const unsigned gmax = __reduce_max_sync(0xffffffffu, ghi);
+        const unsigned glo = __reduce_max_sync(0xffffffffu, ghi == gmax ? (unsigned)gk : 0u);
+        const unsigned who = __ballot_sync(0xffffffffu, ghi == gmax && (unsigned)gk == glo);
+        const float gzw = __shfl_sync(0xffffffffu, gb_z, __ffs(who) - 1);
+        unsigned long long* kp = rec_keys(recs, b, topk);
+        float* fp = rec_f32(recs, b, topk);
         const int c = blockIdx.x;
         if (lane == 0) {
-            recs[rec_at(b, 0, topk) + c] = st_m;
-            recs[rec_at(b, 1, topk) + c] = st_s;
-            recs[rec_at(b, 2, topk) + c] = gb_s;
-            irecs[rec_at(b, 3, topk) + c] = gb_j;
-            recs[rec_at(b, 4, topk) + c] = gb_z;
+            fp[c] = Mall;
+            fp[kMaxGrid + c] = sc;
+            fp[2 * kMaxGrid + c] = gzw;
+            kp[c] = ((unsigned long long)gmax << 32) | glo;
         }
         for (int r = lane; r < topk; r += 32) {
-            recs[rec_at(b, 5 + r, topk) + c] = topv[b * topk + r];
-            irecs[rec_at(b, 5 + topk + r, topk) + c] = topj[b * topk + r];
+            const int j = topj[b * topk + r];
+            kp[(size_t)(1 + r) * kMaxGrid + c] = j >= 0 ? key64(topv[b * topk + r], j) : 0ull;
         }
+        __threadfence();                                    // the record is visible before the ticket is taken
     }
-    __threadfence();
+    VT_STAMP(5);
     __syncthreads();
+    VT_STAMP(6);
     if (threadIdx.x == 0) {
         if (s_abort) atomicOr(&ctrl->flags, (uint32_t)VT_FLAG_TIMEOUT);
-        s_last = (atomicInc(&ctrl->head_ticket, gridDim.x - 1) == gridDim.x - 1);
+        // acquire + release in one: the last CTA's loads below see every other CTA's record
+        unsigned old;
+        asm volatile("atom.acq_rel.gpu.global.inc.u32 %0, [%1], %2;"
+                     : "=r"(old) : "l"(&ctrl->head_ticket), "r"(gridDim.x - 1) : "memory");
+        s_last = (old == gridDim.x - 1);
     }
     __syncthreads();
+    VT_STAMP(7);
     if (!s_last) return;
-    __threadfence();
 
-    if (b < B)
-        merge_records(a.map, a.out_ids, a.out_logprobs, a.dbg_lse, topk, a.uniforms != nullptr, ctrl, recs, b, row_ok,
-                      (int)gridDim.x, reinterpret_cast<float*>(ring) + (size_t)b * kMergeStageWords);
+    {
+        // B <= 8: two warps per hidden row (candidates / statistics) side by side; more rows: one warp each
+        const MergeOut mo{a.map, a.out_ids, a.out_logprobs, a.dbg_lse, topk, a.uniforms != nullptr};
+        const bool split = B <= kNW / 2;
+        const int row = split ? (warp & (kNW / 2 - 1)) : warp;
+        const int roles = split ? (warp < kNW / 2 ? kRoleCand : kRoleStats) : (kRoleCand | kRoleStats);
+        if (row < B)
+            merge_records(mo, ctrl, recs, row, s_rowok[row] != 0, (int)gridDim.x,
+                          reinterpret_cast<float*>(ring) + (size_t)row * kMergeStageWords, roles, &s_xch[row], 1 + row
+#ifdef VT_STAMPS
+                          , stamps + (size_t)blockIdx.x * kStampSlots
+#endif
+                          );
+    }
     if (a.tree.pool_token) {
         // tree drafting: the merged candidates of all rows become pool nodes and the next frontier is
         // chosen here, by the CTA that merged them, instead of in a launch of its own
@@ -530,8 +583,14 @@ bool head_skinny_supported(int32_t B, int32_t d) { return shape_ok(B, d); }
 
 size_t head_skinny_scratch_bytes(int32_t B, int32_t K, int32_t topk) {
     (void)K;
+    return align_up((size_t)kMaxGrid * B * rec_fields(topk) * 4, 256) + kStampBytes;
+}
+
+#ifdef VT_STAMPS
+size_t head_skinny_stamps_offset(int32_t B, int32_t topk) {
     return align_up((size_t)kMaxGrid * B * rec_fields(topk) * 4, 256);
 }
+#endif
 
 cudaError_t launch_head_skinny(const HeadArgs& a, Ctrl* ctrl, uint8_t* scratch, cudaStream_t s) {
     if (!shape_ok(a.B, a.d)) return cudaErrorInvalidValue;
