@@ -80,6 +80,14 @@ size_t vt_workspace_bytes(int op, int64_t n, int32_t V, int32_t K, int32_t d, in
  * allocating `ws`, before any other call that takes it. */
 vt_status vt_workspace_init(void *ws, size_t ws_bytes, void *stream);
 
+/* Every wait inside the kernels (for a bulk copy to land, for another warp's hand-over) is bounded;
+ * when a bound expires the kernel stops waiting, lets its own copies land, raises VT_FLAG_TIMEOUT and,
+ * for vt_draft_head, reports every row as id -1 / logprob NaN.  This call sets the bound used by the
+ * streaming head kernel of calls that take `ws`: `nanoseconds` of device time per wait, 0 = the
+ * built-in default (2 s).  The value stays until changed (vt_workspace_init resets it to 0).
+ * Synchronises `stream`.  (No counterpart in the paper: failure handling of this library.) */
+vt_status vt_workspace_set_wait_limit(void *ws, uint64_t nanoseconds, void *stream);
+
 /* Synchronises `stream`, copies the sticky flags (VT_FLAG_*) and the count of skipped token
  * ids to the HOST locations `flags` / `n_bad` (either may be NULL), clears them on the device
  * and returns VT_OK, VT_ERR_RANGE (bad ids / map entries), VT_ERR_NUMERIC or VT_ERR_TIMEOUT. */

@@ -28,7 +28,7 @@ VT_MAX_TOPK = 64
 VT_CTRL_BYTES = 256
 
 EXPORTS = (
-    "vt_workspace_bytes", "vt_workspace_init", "vt_read_status", "vt_status_str", "vt_launch_count",
+    "vt_workspace_bytes", "vt_workspace_init", "vt_workspace_set_wait_limit", "vt_read_status", "vt_status_str", "vt_launch_count",
     "vt_last_cuda_error",
     "vt_histogram", "vt_select_topk", "vt_build_vocab", "vt_build_vocab_host", "vt_trim_head",
     "vt_draft_head", "vt_draft_head_debug", "vt_draft_head_host", "vt_select_topk_static",
@@ -58,6 +58,7 @@ def lib() -> ctypes.CDLL:
         L.vt_workspace_bytes.argtypes = [c_int, c_int64, c_int32, c_int32, c_int32, c_int32, c_int32]
         L.vt_workspace_init.argtypes = [c_void_p, c_size_t, c_void_p]
         L.vt_read_status.argtypes = [c_void_p, c_void_p, ctypes.POINTER(c_uint32), ctypes.POINTER(c_uint64)]
+        L.vt_workspace_set_wait_limit.argtypes = [c_void_p, c_uint64, c_void_p]
         L.vt_status_str.restype = c_char_p
         L.vt_status_str.argtypes = [c_int]
         L.vt_launch_count.restype = c_uint64
@@ -130,6 +131,11 @@ class Workspace:
         off = (-self.buf.data_ptr()) % 256
         self.ptr = self.buf.data_ptr() + off
         _check("vt_workspace_init", lib().vt_workspace_init(c_void_p(self.ptr), self.nbytes, _stream()))
+
+    def set_wait_limit(self, nanoseconds: int) -> None:
+        """Bound of every device-side wait of the streaming head kernel (0 = the default of 2 s)."""
+        _check("vt_workspace_set_wait_limit",
+               lib().vt_workspace_set_wait_limit(c_void_p(self.ptr), int(nanoseconds), _stream()))
 
     def read_status(self):
         """Synchronises the current stream; returns (status, flags, n_bad) and clears the flags."""

@@ -117,6 +117,15 @@ vt_status vt_workspace_init(void* ws, size_t ws_bytes, void* stream) {
     return from_cuda(cudaMemsetAsync(ws, 0, VT_CTRL_BYTES, as_stream(stream)));
 }
 
+vt_status vt_workspace_set_wait_limit(void* ws, uint64_t nanoseconds, void* stream) {
+    if (!ws || !aligned(ws, 256)) return VT_ERR_WORKSPACE;
+    Ctrl* dev = static_cast<Ctrl*>(ws);
+    const unsigned long long v = nanoseconds;
+    cudaStream_t s = as_stream(stream);
+    if (cudaMemcpyAsync(&dev->wait_ns, &v, sizeof(v), cudaMemcpyHostToDevice, s) != cudaSuccess) return VT_ERR_CUDA;
+    return from_cuda(cudaStreamSynchronize(s));            // `v` lives on this stack frame
+}
+
 vt_status vt_read_status(void* ws, void* stream, uint32_t* flags, uint64_t* n_bad) {
     if (!ws) return VT_ERR_WORKSPACE;
     Ctrl host{};

@@ -14,7 +14,8 @@ struct Ctrl {
     uint32_t flags;               // sticky VT_FLAG_* bits
     uint32_t head_ticket;         // "last CTA merges" ticket of the head kernels (wraps to 0)
     unsigned long long n_bad;     // ids skipped by the histogram
-    uint32_t pad[60];
+    unsigned long long wait_ns;   // bound of a device-side wait in nanoseconds (0 = the built-in default)
+    uint32_t pad[58];
 };
 static_assert(sizeof(Ctrl) == VT_CTRL_BYTES, "control block size");
 

@@ -43,7 +43,7 @@ constexpr int kMaxB = 16;
 constexpr size_t kSmemLimit = 227 * 1024 - 1024; // opt-in limit minus static shared memory
 constexpr int kCand = 64;                        // candidate buffer entries per hidden row
 constexpr int kSelPerLane = (VT_MAX_TOPK + kCand) / 32;
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // default bound of a device-side wait (Ctrl::wait_ns overrides)
 
 
 // Phase stamps (-DVT_STAMPS builds only): thread 0 of every CTA writes %globaltimer at fixed points into
@@ -82,6 +82,14 @@ __device__ __forceinline__ bool mbar_try(uint64_t* b, uint32_t parity) {
         : "=r"(ok) : "r"(smem_u32(b)), "r"(parity) : "memory");
     return ok != 0;
 }
+// non-blocking probe of a phase (try_wait may suspend the thread for a system-chosen time before it answers)
+__device__ __forceinline__ bool mbar_test(uint64_t* b, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{ .reg .pred p; mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
+        : "=r"(ok) : "r"(smem_u32(b)), "r"(parity) : "memory");
+    return ok != 0;
+}
 __device__ __forceinline__ unsigned long long global_ns() {
     unsigned long long t;
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
@@ -90,17 +98,23 @@ __device__ __forceinline__ unsigned long long global_ns() {
 // Bounded wait, called by all 32 lanes of a warp; false when the CTA is aborting or the time limit
 // expired (which starts an abort).  The outcome is voted on, so the lanes of a warp never part ways
 // before a warp-collective instruction (mma, shuffle, ballot).
-__device__ __forceinline__ bool mbar_wait(uint64_t* b, uint32_t parity, volatile int* abort_flag) {
-    bool ok = mbar_try(b, parity);
-    if (!ok) {
-        const unsigned long long t0 = global_ns();
-        for (;;) {
+__device__ __noinline__ bool mbar_wait_slow(uint64_t* b, uint32_t parity, volatile int* abort_flag,
+                                            unsigned long long limit_ns) {
+    bool ok = false;
+    const unsigned long long t0 = global_ns();
+    for (;;) {
+        if (*abort_flag) break;
+        if (global_ns() - t0 > limit_ns) { *abort_flag = 1; break; }
 #pragma unroll 1
-            for (int i = 0; i < 128 && !ok; ++i) ok = mbar_try(b, parity);
-            if (ok || *abort_flag) break;
-            if (global_ns() - t0 > kWaitLimitNs) { *abort_flag = 1; break; }
-        }
+        for (int i = 0; i < 32 && !ok; ++i) ok = mbar_try(b, parity);
+        if (ok) break;
     }
+    return ok;
+}
+__device__ __forceinline__ bool mbar_wait(uint64_t* b, uint32_t parity, volatile int* abort_flag,
+                                          unsigned long long limit_ns) {
+    bool ok = mbar_test(b, parity);
+    if (!ok) ok = mbar_wait_slow(b, parity, abort_flag, limit_ns);     // kept out of line: the hot loop stays small
     return __all_sync(0xffffffffu, ok);
 }
 // bulk copy global -> shared with an L2 eviction-priority hint for the lines it brings in
@@ -186,7 +200,8 @@ __global__ void __launch_bounds__(kThreads, 1)
 k_head_stream(const HeadArgs a, Ctrl* ctrl, float* __restrict__ recs, const Geo geo) {
     extern __shared__ __align__(128) uint8_t s_raw[];
     __shared__ uint64_t s_full[kMaxStages], s_empty[kMaxStages], s_pfull[2], s_pempty[2];
-    __shared__ int s_last, s_abort;
+    __shared__ int s_last, s_abort, s_any_abort;
+    __shared__ int s_issued[kMaxStages];                 // fills requested per stage (for the drain after an abort)
     __shared__ int s_rowok[kMaxB];                       // per hidden row: its temperature is usable
     __shared__ float s_xch[kMaxB];                       // merge: a row's lse, from its statistics warp to its candidate warp
     constexpr int KC = kNW * KBC * 32;                   // columns per chunk
@@ -215,7 +230,7 @@ k_head_stream(const HeadArgs a, Ctrl* ctrl, float* __restrict__ recs, const Geo 
     const int rb1 = (int)((long long)geo.RB * (blockIdx.x + 1) / gridDim.x);
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < S; ++s) { mbar_init(&s_full[s], 1); mbar_init(&s_empty[s], kNW); }
+        for (int s = 0; s < S; ++s) { mbar_init(&s_full[s], 1); mbar_init(&s_empty[s], kNW); s_issued[s] = 0; }
         for (int p = 0; p < 2; ++p) { mbar_init(&s_pfull[p], kNW); mbar_init(&s_pempty[p], B); }
         s_abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -224,6 +239,7 @@ k_head_stream(const HeadArgs a, Ctrl* ctrl, float* __restrict__ recs, const Geo 
     __syncthreads();
     VT_STAMP(0);
     volatile int* abort_flag = &s_abort;
+    unsigned long long wait_ns = kWaitLimitNs;
 
     // per-row state of warp b (identical in its four 8-lane groups); declared here so that the
     // record code after the loop sees it
@@ -248,12 +264,15 @@ k_head_stream(const HeadArgs a, Ctrl* ctrl, float* __restrict__ recs, const Geo 
     auto fetch_next = [&]() -> bool {                         // false = abort
         bool ok = true;
         if (warp == f_duty) {
-            if (f_item >= S && !mbar_wait(&s_empty[f_s], f_ph ^ 1, abort_flag)) ok = false;
+            if (f_item >= S && !mbar_wait(&s_empty[f_s], f_ph ^ 1, abort_flag, wait_ns)) ok = false;
             if (ok) {
                 const int nrows = min(kRows, K - f_rb * kRows);
                 const int col0 = f_c * KC;
                 const uint32_t cbytes = (uint32_t)(min(d, col0 + KC) - col0) * 2u;
-                if (lane == 0) mbar_expect_tx(&s_full[f_s], cbytes * (uint32_t)nrows);
+                if (lane == 0) {
+                    s_issued[f_s] += 1;
+                    mbar_expect_tx(&s_full[f_s], cbytes * (uint32_t)nrows);
+                }
                 __syncwarp();
                 if (lane < nrows)
                     bulk_g2s(smem_u32(ring + (size_t)f_s * stage_bytes + lane * pitch),
@@ -291,6 +310,10 @@ k_head_stream(const HeadArgs a, Ctrl* ctrl, float* __restrict__ recs, const Geo 
                     hh[c][i] = __ldg(reinterpret_cast<const uint4*>(a.h + (size_t)(g + 8) * d + col));
             }
         }
+    {
+        const unsigned long long lim = ctrl->wait_ns;        // 0 = the default
+        if (lim) wait_ns = lim;
+    }
     if (b < B) {
         const float T = a.temp[b];
         row_ok = (T > 0.f) && (T < CUDART_INF_F);
@@ -325,7 +348,7 @@ k_head_stream(const HeadArgs a, Ctrl* ctrl, float* __restrict__ recs, const Geo 
                 float acc0[4] = {0.f, 0.f, 0.f, 0.f}, acc1[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
                 for (int c = 0; c < NCH; ++c) {
-                    if (!alive || !mbar_wait(&s_full[s], ph, abort_flag)) { alive = false; continue; }
+                    if (!alive || !mbar_wait(&s_full[s], ph, abort_flag, wait_ns)) { alive = false; continue; }
 #ifdef VT_STAMPS
                     if (item == 0) VT_STAMP(3);
 #endif
@@ -357,7 +380,7 @@ k_head_stream(const HeadArgs a, Ctrl* ctrl, float* __restrict__ recs, const Geo 
         // ---- hand the partial tiles over ------------------------------------------------------------
         const int pb = n & 1;
         const uint32_t use = (uint32_t)(n >> 1);
-        if (n >= 2 && !mbar_wait(&s_pempty[pb], (use - 1) & 1, abort_flag)) break;
+        if (n >= 2 && !mbar_wait(&s_pempty[pb], (use - 1) & 1, abort_flag, wait_ns)) break;
 #pragma unroll
         for (int r = 0; r < R; ++r) {
             if (r < rc) {
@@ -371,7 +394,7 @@ k_head_stream(const HeadArgs a, Ctrl* ctrl, float* __restrict__ recs, const Geo 
         if (lane == 0) mbar_arrive(&s_pfull[pb]);
         if (b >= B) continue;
         // ---- warp b: reduce the tiles, update hidden row b --------------------------------------------
-        if (!mbar_wait(&s_pfull[pb], use & 1, abort_flag)) break;
+        if (!mbar_wait(&s_pfull[pb], use & 1, abort_flag, wait_ns)) break;
         const bool in_group = e_r < rc;
         float x = 0.f;
         if (in_group) {
@@ -420,16 +443,6 @@ k_head_stream(const HeadArgs a, Ctrl* ctrl, float* __restrict__ recs, const Geo 
         }
     }
     VT_STAMP(4);
-    if (warp == kNW - 1 && *abort_flag) {
-        // drain: every stage that was filled must have landed before the CTA may leave
-        const int back = min(f_item, S);
-        for (int i = 1; i <= back; ++i) {
-            const int it = f_item - i;
-            const unsigned long long t0 = global_ns();
-            while (!mbar_try(&s_full[it % S], (uint32_t)((it / S) & 1)) && global_ns() - t0 < kWaitLimitNs) {}
-        }
-    }
-
     // ---- this CTA's record per hidden row ----------------------------------------------------------
     if (b < B && !*abort_flag) {
         if (n_cand > 0) {
@@ -466,19 +479,43 @@ k_head_stream(const HeadArgs a, Ctrl* ctrl, float* __restrict__ recs, const Geo 
         __threadfence();                                    // the record is visible before the ticket is taken
     }
     VT_STAMP(5);
-    __syncthreads();
+    __syncthreads();                                        // every warp has left the loop: no copy is requested from here on
     VT_STAMP(6);
+    if (warp == 0 && *abort_flag) {
+        // drain: every stage that was requested must have landed before the CTA may leave
+        for (int st = lane; st < S; st += 32) {
+            const int fills = s_issued[st];
+            if (fills > 0) {
+                const unsigned long long t0 = global_ns();
+                while (!mbar_try(&s_full[st], (uint32_t)((fills - 1) & 1)) && global_ns() - t0 < kWaitLimitNs) {}
+            }
+        }
+        __syncwarp();
+    }
     if (threadIdx.x == 0) {
-        if (s_abort) atomicOr(&ctrl->flags, (uint32_t)VT_FLAG_TIMEOUT);
-        // acquire + release in one: the last CTA's loads below see every other CTA's record
+        const bool aborted = s_abort != 0;
+        if (aborted) atomicOr(&ctrl->flags, (uint32_t)VT_FLAG_TIMEOUT);
+        // Ticket: arrivals in the low half, aborted CTAs in the high half.  Acquire + release in one, so
+        // that the last CTA's loads below see every other CTA's record.
         unsigned old;
-        asm volatile("atom.acq_rel.gpu.global.inc.u32 %0, [%1], %2;"
-                     : "=r"(old) : "l"(&ctrl->head_ticket), "r"(gridDim.x - 1) : "memory");
-        s_last = (old == gridDim.x - 1);
+        asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], %2;"
+                     : "=r"(old) : "l"(&ctrl->head_ticket), "r"(aborted ? 0x10001u : 1u) : "memory");
+        s_last = ((old & 0xffffu) == gridDim.x - 1);
+        s_any_abort = aborted || (old >> 16) != 0;
+        if (s_last) ctrl->head_ticket = 0;                  // ready for the next launch
     }
     __syncthreads();
     VT_STAMP(7);
     if (!s_last) return;
+
+    if (s_any_abort) {
+        // a bounded wait expired somewhere: the records are incomplete; report every row as missing
+        for (int i = threadIdx.x; i < B * (1 + topk); i += kThreads) {
+            a.out_ids[i] = -1;
+            a.out_logprobs[i] = CUDART_NAN_F;
+        }
+        return;
+    }
 
     {
         // B <= 8: two warps per hidden row (candidates / statistics) side by side; more rows: one warp each

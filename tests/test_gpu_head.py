@@ -123,6 +123,31 @@ def test_bad_temperature_is_flagged_not_fatal():
     assert ws.read_status()[0] == 0 and int(gi2.min()) >= 0
 
 
+def test_an_expired_wait_is_reported_and_the_workspace_stays_usable():
+    """Every device-side wait is bounded.  With the bound set to 1 ns the first wait that is not
+    satisfied at once (the first stage of weights is still on its way) gives up: the kernel lets its
+    copies land, reports VT_ERR_TIMEOUT and marks every row missing; nothing hangs, nothing is broken
+    on purpose.  With the default bound back, the same workspace serves a clean call."""
+    B, K, d, topk = 2, 20_000, 3072, 8
+    W = vt_inputs.gaussian_bf16((K, d), 0.02, seed=21, device=DEV)
+    h = vt_inputs.gaussian_bf16((B, d), 1.0, seed=22, device=DEV)
+    T = vt_inputs.temperatures(B, 1.0, 1.0, 0, device=DEV)
+    u = vt_inputs.uniforms((B, K), seed=23, device=DEV)
+    ws = vt.Workspace(vt.workspace_bytes(vt.VT_OP_DRAFT_HEAD, 0, 0, K, d, B, topk))
+    good = tuple(t.clone() for t in _run(h, W, None, T, topk, u, debug=False, ws=ws))
+    assert ws.read_status() == (0, 0, 0)
+    ws.set_wait_limit(1)
+    gi, gl = _run(h, W, None, T, topk, u, debug=False, ws=ws)
+    st, flags, _ = ws.read_status()
+    assert st == 5 and flags & vt.VT_FLAG_TIMEOUT                    # VT_ERR_TIMEOUT
+    assert bool((gi == -1).all()) and bool(torch.isnan(gl).all())
+    ws.set_wait_limit(0)
+    for _ in range(2):
+        gi, gl = _run(h, W, None, T, topk, u, debug=False, ws=ws)
+        assert torch.equal(gi, good[0]) and torch.equal(gl, good[1])
+    assert ws.read_status() == (0, 0, 0)
+
+
 SLACK = {}            # workload -> [positions accepted through the margin rule, positions compared]
 
 
