@@ -43,9 +43,36 @@ TREE_KS = (8192, 16384, 32768, 65536, V)
 L2_BYTES = 126 * 1024 * 1024
 FALLBACK_HBM_GBS = 6650.0
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the head kernel on the headline
-# workload, from the ncu capture summarised under profiles/ (None until a capture exists).
-NCU_TRAFFIC_BYTES = {"k_head_stream": 206_000_000, "k_hist_hot": None}
+PROFILE_KERNEL_SOURCES = {           # kernel -> the sources whose change invalidates its captured counters
+    "k_head_stream": ("vt_head_skinny.cu", "vt_head_common.cuh"),
+    "k_head_dense": ("vt_head_dense.cu", "vt_head_common.cuh"),
+    "k_hist_hot": ("vt_hist.cu",),
+}
+
+
+def source_digest(kernel: str) -> str:
+    """Short hash of the source files a kernel is built from (what a profile summary records)."""
+    import hashlib
+
+    h = hashlib.sha256()
+    for name in PROFILE_KERNEL_SOURCES[kernel]:
+        h.update(open(os.path.join(ROOT, "paper_2506_22694_b200", "csrc", name), "rb").read())
+    return h.hexdigest()[:16]
+
+
+def profile_traffic(kernel: str, workload: str):
+    """dram__bytes_read.sum + dram__bytes_write.sum per launch of `kernel` on `workload`, read from the
+    ncu summary under profiles/ (a line `traffic_bytes_per_launch[<kernel>|<workload>] = <bytes> @ <digest>`).
+    None when no capture exists or the kernel's sources changed since it was taken."""
+    import glob
+    import re
+
+    pat = re.compile(r"traffic_bytes_per_launch\[%s\|%s\]\s*=\s*(\d+)\s*@\s*([0-9a-f]+)" % (re.escape(kernel), re.escape(workload)))
+    for path in sorted(glob.glob(os.path.join(ROOT, "profiles", "*.md"))):
+        m = pat.search(open(path).read())
+        if m:
+            return int(m.group(1)) if m.group(2) == source_digest(kernel) else None
+    return None
 
 
 def measured_peaks():
@@ -65,7 +92,7 @@ class ClockSampler:
     SLOW_BITS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown",
                  0x4: "sw_power_cap", 0x80: "hw_power_brake"}
 
-    def __init__(self, device_index: int, period_s: float = 0.02):
+    def __init__(self, device_index: int, period_s: float = 0.005):
         self.samples, self.reasons, self.max_mhz = [], set(), None
         self.period, self._stop, self._thr, self._h = period_s, threading.Event(), None, None
         try:
@@ -116,6 +143,36 @@ def _events():
     return torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
 
 
+def roofline(kernel, workload, bound, algo, seconds, peak, unit, peak_kind, extra=None):
+    """The roofline object of one kernel: achieved = algorithmic bytes (or flops) per launch / measured
+    launch time, against the measured peak; traffic from the committed ncu summary when it is current."""
+    scale = 1e9 if unit == "GB/s" else 1e12
+    ach = algo / seconds / scale
+    r = {"kernel": kernel, "bound": bound, "achieved": ach, "peak": peak, "unit": unit, "frac": ach / peak,
+         "peak_source": peak_kind, "algorithmic_%s_per_launch" % ("bytes" if unit == "GB/s" else "flops"): algo,
+         "traffic": profile_traffic(kernel, workload)}
+    if unit == "GB/s":
+        r["frac_of_8000"] = ach / 8000.0
+    if extra:
+        r.update(extra)
+    return r
+
+
+def clocks_under(fn, device_index, min_ms=60.0):
+    """SM clock / throttle record while `fn(i)` (one step) is repeated for at least `min_ms`: the timed
+    regions themselves can be shorter than one sampling period, so the record is taken over a repeat
+    of the same steps long enough to hold a dozen samples."""
+    with ClockSampler(device_index) as clk:
+        t0 = time.perf_counter()
+        i = 0
+        while (time.perf_counter() - t0) * 1e3 < min_ms:
+            for _ in range(64):
+                fn(i)
+                i += 1
+            torch.cuda.synchronize()
+    return clk.summary()
+
+
 def _copies_for_cold_l2(nbytes: int) -> int:
     """Number of distinct copies of a weight matrix to rotate through so that at least 8x the L2
     capacity is streamed between two uses of the same copy."""
@@ -158,8 +215,34 @@ def run_head_steps(vt, wl, steps, start=0, overlapped=True):
                          us[i % len(us)] if us else None, ws=wl["ws"], out=wl["out"], overlapped=overlapped)
 
 
-def time_head(vt, wl, steps, warmup):
+def first_touch(vt, wl):
+    """Set-up, not warm-up: one plain step on every weight copy and every h of the pool, so that no
+    buffer (nor its page-table entries) is touched for the first time inside a timed region."""
     torch.cuda.synchronize()                    # the weights were written earlier: they are final from here on
+    n = max(len(wl["copies"]), len(wl["hs"]), len(wl["us"]) if wl["us"] else 0)
+    run_head_steps(vt, wl, n, overlapped=False)
+    torch.cuda.synchronize()
+
+
+def time_head_latency(vt, wl, n=200):
+    """Dependent-step latency: plain vt_draft_head calls (no overlap with the previous step), one event
+    pair per call, everything enqueued ahead so that the host is not in the measured path.  Returns
+    (median, p10, p90) in microseconds over n calls."""
+    copies, hs, us = wl["copies"], wl["hs"], wl["us"]
+    first_touch(vt, wl)
+    ev = [_events() for _ in range(n)]
+    for i, (e0, e1) in enumerate(ev):
+        e0.record()
+        vt.vt_draft_head(hs[i % len(hs)], copies[i % len(copies)], wl["map"], wl["T"], wl["topk"],
+                         us[i % len(us)] if us else None, ws=wl["ws"], out=wl["out"], overlapped=False)
+        e1.record()
+    torch.cuda.synchronize()
+    t = sorted(e0.elapsed_time(e1) * 1e3 for e0, e1 in ev[n // 10:])
+    return t[len(t) // 2], t[len(t) // 10], t[(9 * len(t)) // 10]
+
+
+def time_head(vt, wl, steps, warmup):
+    first_touch(vt, wl)
     run_head_steps(vt, wl, warmup)
     torch.cuda.synchronize()
     e0, e1 = _events()
@@ -203,30 +286,50 @@ def time_head_e2e(vt, wl, steps, warmup):
 
 
 # --------------------------------------------------------------------------------------------------
-def oracle_head_rate(wl, seconds=12.0, rows=None):
-    """Times the CPU oracle on a bounded sample (the first `rows` vocabulary rows) of one head step;
-    returns (us per FULL step scaled by K/rows, rows used, threads, repetitions)."""
+def oracle_head_rate(vt, wl, seconds=12.0):
+    """The CPU baseline leg: times the fp64 oracle, as it stands, on full head steps of the same workload
+    for about `seconds`, and -- since its results are at hand -- compares the GPU's ids and
+    log-probabilities of the same steps with them under the parity rules of the tests (ids equal unless
+    the oracle's own logit margin is below 1e-3; |logp - ref| <= 2e-3).
+    Returns (us per step, threads, repetitions, parity record)."""
     import numpy as np
 
     import oracle
 
     K, B, topk = wl["K"], wl["B"], wl["topk"]
     Wb = vt_inputs.bf16_bits(wl["copies"][0]).cpu().numpy().view(np.uint16)
-    hb = vt_inputs.bf16_bits(wl["hs"][0]).cpu().numpy().view(np.uint16)
+    mh = wl["map"].cpu().numpy() if wl["map"] is not None else None
+    inv = {int(v): j for j, v in enumerate(mh)} if mh is not None else None
     T = wl["T"].cpu().numpy()
-    u = wl["us"][0].cpu().numpy() if wl["us"] else None
-    rows = K if rows is None else max(topk, min(K, rows))
-    Ws = Wb[:rows]
-    us = None if u is None else np.ascontiguousarray(u[:, :rows])
-    t0 = time.perf_counter()
-    reps = 0
+    t_cpu, reps = 0.0, 0
+    par = {"positions": 0, "margin_rule_accepts": 0, "mismatches": 0, "max_abs_logprob_err": 0.0}
     while True:
-        oracle.draft_head(hb, Ws, None, T, topk, us, want_full=False)
+        i = reps % len(wl["hs"])
+        hb = vt_inputs.bf16_bits(wl["hs"][i]).cpu().numpy().view(np.uint16)
+        u = wl["us"][i % len(wl["us"])].cpu().numpy() if wl["us"] else None
+        t0 = time.perf_counter()
+        ref = oracle.draft_head(hb, Wb, mh, T, topk, u, want_full=True)
+        t_cpu += time.perf_counter() - t0
         reps += 1
-        el = time.perf_counter() - t0
-        if el >= seconds or (reps >= 3 and el >= seconds / 2):
+        gi, gl = vt.vt_draft_head(wl["hs"][i], wl["copies"][0], wl["map"], wl["T"], topk,
+                                  wl["us"][i % len(wl["us"])] if wl["us"] else None, ws=wl["ws"])
+        gi, gl = gi.cpu().numpy(), gl.cpu().numpy().astype(np.float64)
+        for b in range(B):
+            for c in range(1 + topk):
+                jg = inv[int(gi[b, c])] if inv is not None else int(gi[b, c])
+                jo = int(ref.trim[b, c])
+                score = ref.score[b] if (c == 0 and u is not None) else ref.z[b]
+                par["positions"] += 1
+                if jg != jo:
+                    if float(T[b]) * abs(score[jo] - score[jg]) < 1e-3:
+                        par["margin_rule_accepts"] += 1
+                    else:
+                        par["mismatches"] += 1
+                err = abs(gl[b, c] - (ref.z[b, jg] - ref.lse[b]))
+                par["max_abs_logprob_err"] = max(par["max_abs_logprob_err"], float(err))
+        if t_cpu >= seconds or (reps >= 3 and t_cpu >= seconds / 2):
             break
-    return el / reps * 1e6 * (K / rows), rows, oracle.max_threads(), reps
+    return t_cpu / reps * 1e6, oracle.max_threads(), reps, par
 
 
 def run_reference(args, rank):
@@ -280,8 +383,9 @@ def head_config():
 
 
 # --------------------------------------------------------------------------------------------------
-def extras(vt, dev, peak_gbs):
-    """K sweep of the tree-drafting head, the full-vocabulary chain head, and the vocabulary build."""
+def extras(vt, dev, peak_gbs, peak_kind):
+    """K sweep of the tree-drafting head, the full-vocabulary chain head, and the vocabulary build; every
+    kernel-level figure comes as a roofline object with the clocks sampled while its steps repeat."""
     out = {}
     sweep = []
     for K in TREE_KS:
@@ -289,9 +393,12 @@ def extras(vt, dev, peak_gbs):
                                  seed=1003)
         n = max(50, min(2000, int(0.25 / (K * TREE["d"] * 2 / 5e12))))
         ms = time_head(vt, wl, n, 20)
-        gbs = wl["algo_bytes"] / (ms * 1e-3) / 1e9
-        sweep.append({"K": K, "us_per_step": ms * 1e3, "gbs": gbs, "frac_of_measured": gbs / peak_gbs,
-                      "frac_of_8000": gbs / 8000.0})
+        lat = time_head_latency(vt, wl)
+        clk = clocks_under(lambda i: run_head_steps(vt, wl, 1, start=i), dev.index)
+        sweep.append({"K": K, "us_per_step": ms * 1e3, "us_dependent_step": {"median": lat[0], "p10": lat[1], "p90": lat[2]},
+                      "roofline": roofline("k_head_stream", "config3 K=%d" % K, "hbm", wl["algo_bytes"], ms * 1e-3, peak_gbs,
+                                           "GB/s", peak_kind),
+                      "clocks": clk})
         del wl
         torch.cuda.empty_cache()
     out["tree_head_k_sweep"] = {"workload": "config3: d=4096 B=10 topk=10 T=0.7 Gumbel sampling, cold L2",
@@ -305,18 +412,22 @@ def extras(vt, dev, peak_gbs):
         wl = build_head_workload(vt, dev, d_, K_, 1, 8, 1.0, False, seed=1007)
         ms = time_head(vt, wl, 2000, 50)
         gbs = wl["algo_bytes"] / (ms * 1e-3) / 1e9
+        lat = time_head_latency(vt, wl)
         warm = dict(wl, copies=wl["copies"][:1])                      # one copy: the head stays in L2
         ms_w = time_head(vt, warm, 2000, 50)
         small.append({"workload": name + ", B=1, top-8", "mbytes": wl["algo_bytes"] / 1e6, "us_per_step_cold": ms * 1e3,
-                      "gbs_cold": gbs, "frac_of_measured_cold": gbs / peak_gbs, "us_per_step_l2_resident": ms_w * 1e3})
+                      "gbs_cold": gbs, "frac_of_measured_cold": gbs / peak_gbs, "us_per_step_l2_resident": ms_w * 1e3,
+                      "us_dependent_step_cold": {"median": lat[0], "p10": lat[1], "p90": lat[2]}})
         del wl, warm
         torch.cuda.empty_cache()
     out["small_heads"] = small
     wl = build_head_workload(vt, dev, HEAD["d"], V, HEAD["B"], HEAD["topk"], HEAD["temp"], False, seed=1002)
     ms = time_head(vt, wl, 300, 20)
-    gbs = wl["algo_bytes"] / (ms * 1e-3) / 1e9
+    clk = clocks_under(lambda i: run_head_steps(vt, wl, 1, start=i), dev.index)
     out["full_head"] = {"workload": "config2 with the untrimmed head K=V=128256", "us_per_step": ms * 1e3,
-                        "gbs": gbs, "frac_of_measured": gbs / peak_gbs}
+                        "roofline": roofline("k_head_stream", "config2 K=V", "hbm", wl["algo_bytes"], ms * 1e-3, peak_gbs,
+                                             "GB/s", peak_kind),
+                        "clocks": clk}
     del wl
     torch.cuda.empty_cache()
     # vocabulary build at corpus scale
@@ -337,12 +448,14 @@ def extras(vt, dev, peak_gbs):
         torch.cuda.synchronize()
         return e0.elapsed_time(e1) / reps
 
-    ms_h = timed(lambda: vt.vt_histogram(ids, V, counts=counts, ws=ws))
+    ms_h = timed(lambda: vt.vt_histogram(ids, V, counts=counts, ws=ws), reps=20, warm=3)
+    clk = clocks_under(lambda i: vt.vt_histogram(ids, V, counts=counts, ws=ws), dev.index)
     vb = {"workload": "config5: 1e9 int32 ids, V=128256, 95% Zipf(1.07) + 5% uniform",
           "histogram_ms": ms_h, "histogram_gtok_s": n / (ms_h * 1e-3) / 1e9,
-          "histogram_gbs": 4.0 * n / (ms_h * 1e-3) / 1e9}
-    vb["histogram_frac_of_measured"] = vb["histogram_gbs"] / peak_gbs
-    vb["histogram_frac_of_8000"] = vb["histogram_gbs"] / 8000.0
+          "roofline": roofline("k_hist_hot", "config5 1e9 ids", "hbm", 4.0 * n, ms_h * 1e-3, peak_gbs, "GB/s", peak_kind,
+                               {"note": "whole vt_histogram call (all its kernels) per 4 bytes of every id"}),
+          "clocks": clk}
+    vb["histogram_frac_of_measured"] = vb["roofline"]["frac"]
     for K in (8192, 32768):
         ms_b = timed(lambda: vt.vt_build_vocab(ids, V, K, ws=ws))
         vb["build_vocab_K%d_ms" % K] = ms_b
@@ -360,8 +473,8 @@ def extras(vt, dev, peak_gbs):
     W_trim = torch.empty((32768, 4096), dtype=torch.bfloat16, device=dev)
     ms_g = timed(lambda: vt.vt_trim_head(W_full, map_, W_trim), reps=20)
     vb["trim_head_K32768_d4096_us"] = ms_g * 1e3
-    vb["trim_head_gbs"] = 2 * 32768 * 4096 * 2 / (ms_g * 1e-3) / 1e9
-    vb["trim_head_frac_of_measured"] = vb["trim_head_gbs"] / peak_gbs
+    vb["trim_head_roofline"] = roofline("k_gather_rows", "config5 K=32768 d=4096", "hbm", 2.0 * 32768 * 4096 * 2, ms_g * 1e-3,
+                                        peak_gbs, "GB/s", peak_kind)
     out["vocab_build"] = vb
     out["draft_block"] = draft_block_case(vt, dev, timed)
     return out
@@ -422,25 +535,90 @@ DENSE = dict(d=4096, K=32768, B=256, topk=8)                   # config 4: batch
 
 
 def dense_case(vt, dev, steps=200, warmup=20):
-    """Config 4: 256 rows x K=32768 x d=4096 on the tensor-core path, per-row temperatures, Gumbel sampling."""
-    peaks, _ = measured_peaks()
+    """Config 4: 256 rows x K=32768 x d=4096 on the tensor-core path, per-row temperatures, Gumbel sampling.
+    Reported against the slower of its two bounds (tensor pipe at the measured bf16 burst rate, HBM at the
+    measured copy rate)."""
+    peaks, peak_kind = measured_peaks()
     d, K, B, topk = DENSE["d"], DENSE["K"], DENSE["B"], DENSE["topk"]
     wl = build_head_workload(vt, dev, d, K, B, topk, 1.0, True, seed=1004, pool=4)
     wl["T"] = vt_inputs.temperatures(B, 0.5, 1.5, seed=5001, device=dev)
     ms = time_head(vt, wl, steps, warmup)
+    clk = clocks_under(lambda i: run_head_steps(vt, wl, 1, start=i), dev.index)
     st, flags, _ = wl["ws"].read_status()
     flops = 2.0 * B * K * d
-    tf = flops / (ms * 1e-3) / 1e12
-    gbs = wl["algo_bytes"] / (ms * 1e-3) / 1e9
     t_tensor = flops / (float(peaks["bf16_tflops"]) * 1e12) * 1e6
     t_hbm = wl["algo_bytes"] / (float(peaks["hbm_gbs"]) * 1e9) * 1e6
+    if t_hbm >= t_tensor:
+        roof = roofline("k_head_dense", "config4", "hbm", wl["algo_bytes"], ms * 1e-3, float(peaks["hbm_gbs"]), "GB/s", peak_kind)
+    else:
+        roof = roofline("k_head_dense", "config4", "tensor", flops, ms * 1e-3, float(peaks["bf16_tflops"]), "TFLOP/s", peak_kind)
+    tf = flops / (ms * 1e-3) / 1e12
     return {"workload": "config4: 64 seq x 4 nodes = 256 rows, d=4096, K=32768, T_b~U[0.5,1.5], top-8, Gumbel, cold L2",
-            "us_per_step": ms * 1e3, "tflops": tf, "gbs": gbs, "status": st,
+            "us_per_step": ms * 1e3, "tflops": tf, "status": st, "roofline": roof, "clocks": clk,
             "frac_of_bf16_burst": tf / float(peaks["bf16_tflops"]),
             "frac_of_bf16_sustained": tf / float(peaks["bf16_tflops_sustained"]),
-            "frac_of_hbm": gbs / float(peaks["hbm_gbs"]),
             "bound_us": {"tensor_burst": t_tensor, "hbm": t_hbm},
             "frac_of_lower_bound": max(t_tensor, t_hbm) / (ms * 1e3)}
+
+
+STAMP_NAMES = ("entry", "ring_requested", "released", "first_stage_landed", "last_stage_consumed", "record_written",
+               "after_fence_barrier", "after_ticket", "merge_loads_done", "merge_selection_done", "merge_outputs_written")
+
+
+def stamps_case(vt, vt_build, dev, args):
+    """Where a head step's time goes: runs the headline step with the instrumented twin of the library
+    (-DVT_STAMPS, built on demand) whose streaming kernel writes a nanosecond stamp per CTA and phase into
+    the workspace, and prints, per launch mode, the median over launches of each phase's time after the
+    first CTA was released by the launch dependency (maximum over CTAs unless said otherwise)."""
+    import ctypes
+
+    import numpy as np
+
+    vt.LIB_PATH = vt_build.build(stamps=True)
+    vt._lib = None
+    L = vt.lib()
+    L.vt_stamps_region.argtypes = [ctypes.c_int32] * 3 + [ctypes.c_void_p] * 3
+    L.vt_stamps_region.restype = ctypes.c_int32
+    shapes = {"config2": (HEAD["d"], HEAD["K"], HEAD["B"], HEAD["topk"], HEAD["temp"], False),
+              "config3 K=8192": (TREE["d"], 8192, TREE["B"], TREE["topk"], TREE["temp"], True),
+              "small d=1024 K=5000": (1024, 5000, 1, 8, 1.0, False)}
+    for name, (d, K, B, topk, temp, sample) in shapes.items():
+        wl = build_head_workload(vt, dev, d, K, B, topk, temp, sample, seed=1002)
+        off, slots, ctas = ctypes.c_size_t(0), ctypes.c_int32(0), ctypes.c_int32(0)
+        if not L.vt_stamps_region(B, d, topk, ctypes.byref(off), ctypes.byref(slots), ctypes.byref(ctas)):
+            continue
+        ws = wl["ws"]
+        view = ws.buf[(ws.ptr - ws.buf.data_ptr()) + off.value:][: ctas.value * slots.value * 8].view(torch.int64)
+        first_touch(vt, wl)
+        rec = {"case": "stamps", "workload": name, "unit": "us after the first CTA's release, median over launches"}
+        for mode, ov in (("overlapped", True), ("plain", False)):
+            rows = []
+            for rep_ in range(max(8, args.steps)):
+                view.zero_()
+                run_head_steps(vt, wl, 5, start=rep_ * 5, overlapped=ov)
+                torch.cuda.synchronize()
+                x = view.cpu().numpy().reshape(ctas.value, slots.value)
+                x = x[x[:, 0] > 0]
+                t_rel = x[:, 2].min()
+                last = int(np.argmax(x[:, 8]))
+                row = {"ctas": int(x.shape[0]), "entry_first": (x[:, 0].min() - t_rel) / 1e3}
+                for k in range(2, 8):
+                    row[STAMP_NAMES[k] + "_last"] = (x[:, k].max() - t_rel) / 1e3
+                row["last_stage_consumed_median"] = float(np.median(x[:, 4] - t_rel)) / 1e3
+                row["last_stage_consumed_first"] = (x[:, 4].min() - t_rel) / 1e3
+                for k in range(8, 11):
+                    row[STAMP_NAMES[k]] = (x[last, k] - t_rel) / 1e3
+                rows.append(row)
+            rec[mode] = {k: round(float(np.median([r[k] for r in rows])), 2) for k in rows[0]}
+            e0, e1 = _events()
+            e0.record()
+            run_head_steps(vt, wl, 200, overlapped=ov)
+            e1.record()
+            torch.cuda.synchronize()
+            rec[mode]["us_per_step_with_stamps"] = round(e0.elapsed_time(e1) * 5, 2)
+        print(json.dumps(rec), flush=True)
+        del wl
+        torch.cuda.empty_cache()
 
 
 def small_case(vt, dev, args, peak_gbs):
@@ -498,9 +676,10 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-extras", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--case", default="head", choices=["head", "hist", "tree", "dense"],
-                    help="head: the full bench line (default); hist / tree: a short run of the vocabulary "
-                         "histogram (--hist-n ids) or of the tree-drafting head, for profiler captures")
+    ap.add_argument("--case", default="head", choices=["head", "hist", "tree", "dense", "stamps"],
+                    help="head: the full bench line (default); hist / tree / dense: a short run of the vocabulary "
+                         "histogram (--hist-n ids), of the tree-drafting head or of the batched head, for profiler "
+                         "captures; stamps: per-phase timeline of a head step from the instrumented build")
     ap.add_argument("--hist-n", type=int, default=200_000_000)
     args = ap.parse_args()
     args.warmup = max(3, args.warmup)
@@ -527,57 +706,65 @@ def main():
 
     peaks, peak_kind = measured_peaks()
     peak_gbs = float(peaks["hbm_gbs"])
+    if args.case == "stamps":
+        stamps_case(vt, vt_build, dev, args)
+        return
     if args.case != "head":
         small_case(vt, dev, args, peak_gbs)
         return
     wl = build_head_workload(vt, dev, HEAD["d"], HEAD["K"], HEAD["B"], HEAD["topk"], HEAD["temp"], False,
                              seed=1002)
-    torch.cuda.synchronize()
+    first_touch(vt, wl)                          # set-up: every weight copy and every h has been used once
     run_head_steps(vt, wl, args.warmup)
     torch.cuda.synchronize()
     if dist:
         dist.barrier()
     launches0 = vt.launch_count()
-    with ClockSampler(local) as clk:
-        torch.cuda.synchronize()
-        e0, e1 = _events()
-        e0.record()
-        run_head_steps(vt, wl, args.steps, start=args.warmup)
-        e1.record()
-        torch.cuda.synchronize()
+    torch.cuda.synchronize()
+    e0, e1 = _events()
+    e0.record()
+    run_head_steps(vt, wl, args.steps, start=args.warmup)
+    e1.record()
+    torch.cuda.synchronize()
     launches = vt.launch_count() - launches0
     if dist:
         dist.barrier()
     ms_step = max_over_ranks(e0.elapsed_time(e1), dist, dev) / args.steps
+    # clocks: sampled while the same steps repeat for a few dozen milliseconds (the timed region above can
+    # be shorter than one sampling period)
+    clocks = clocks_under(lambda i: run_head_steps(vt, wl, 1, start=i), local)
+    lat = time_head_latency(vt, wl)
+    lat_ms = max_over_ranks(lat[0], dist, dev)
     e2e_ms, h2d, d2h = time_head_e2e(vt, wl, max(200, min(args.steps, 5000)), 50)
     e2e_ms = max_over_ranks(e2e_ms, dist, dev)
     st, flags, _ = wl["ws"].read_status()
     if st != 0:
         raise SystemExit("device-side status after the timed region: %s (flags %d)" % (vt.status_str(st), flags))
 
-    gbs = wl["algo_bytes"] / (ms_step * 1e-3) / 1e9
+    roof = roofline("k_head_stream", "config2", "hbm", wl["algo_bytes"], ms_step * 1e-3, peak_gbs, "GB/s", peak_kind)
     line = {
         "metric": "drafter_lm_head_us_per_step", "value": ms_step * 1e3, "unit": "us", "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": False,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": head_config(),
         "e2e": {"value": e2e_ms * 1e3, "unit": "us", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
-        "gpu_launches": int(launches), "clocks": clk.summary(),
-        "hbm_gbs": gbs,
-        "roofline": {"kernel": "k_head_stream", "bound": "hbm", "achieved": gbs, "peak": peak_gbs, "unit": "GB/s",
-                     "frac": gbs / peak_gbs, "frac_of_8000": gbs / 8000.0, "peak_source": peak_kind,
-                     "algorithmic_bytes_per_launch": wl["algo_bytes"],
-                     "traffic": NCU_TRAFFIC_BYTES["k_head_stream"]},
+        "gpu_launches": int(launches), "clocks": clocks,
+        "hbm_gbs": roof["achieved"],
+        "roofline": roof,
+        "dependent_step": {"what": "plain vt_draft_head, one event pair per call, nothing overlapped with the previous step",
+                           "us_median": lat_ms, "us_p10": lat[1], "us_p90": lat[2],
+                           "frac_of_measured_hbm": wl["algo_bytes"] / (lat_ms * 1e-6) / 1e9 / peak_gbs},
     }
     line = aggregate_line(line, world)
     if rank == 0 and world == 1:
         if not args.no_cpu_baseline:
-            us, rows, threads, reps = oracle_head_rate(wl, seconds=12.0)
+            us, threads, reps, par = oracle_head_rate(vt, wl, seconds=12.0)
             line["cpu_baseline"] = {"value": us, "unit": "us", "cores": threads, "kind": "oracle",
-                                    "sample": "%d full head steps (all %d rows) of the same workload" % (reps, rows)}
+                                    "sample": "%d full head steps (all %d rows) of the same workload" % (reps, wl["K"])}
+            line["parity_slack"] = par
         del wl
         torch.cuda.empty_cache()
         if not args.no_extras:
-            line.update(extras(vt, dev, peak_gbs))
+            line.update(extras(vt, dev, peak_gbs, peak_kind))
     if rank == 0:
         print(json.dumps(line), flush=True)
     if dist:

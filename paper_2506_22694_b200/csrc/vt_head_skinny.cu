@@ -95,26 +95,37 @@ __device__ __forceinline__ unsigned long long global_ns() {
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
     return t;
 }
-// Bounded wait, called by all 32 lanes of a warp; false when the CTA is aborting or the time limit
-// expired (which starts an abort).  The outcome is voted on, so the lanes of a warp never part ways
-// before a warp-collective instruction (mma, shuffle, ballot).
-__device__ __noinline__ bool mbar_wait_slow(uint64_t* b, uint32_t parity, volatile int* abort_flag,
-                                            unsigned long long limit_ns) {
-    bool ok = false;
-    const unsigned long long t0 = global_ns();
-    for (;;) {
-        if (*abort_flag) break;
-        if (global_ns() - t0 > limit_ns) { *abort_flag = 1; break; }
-#pragma unroll 1
-        for (int i = 0; i < 32 && !ok; ++i) ok = mbar_try(b, parity);
-        if (ok) break;
-    }
-    return ok;
+// The bound of a wait is kept with the SM's cycle counter (reading the nanosecond timer costs far more
+// than a probe): two cycles per nanosecond, i.e. at least the time asked for at any SM clock up to
+// 2 GHz.  It lives in shared memory and is looked at only once a wait has to spin, so it costs the hot
+// loop no register.  Bounds under a millisecond spin on non-blocking probes only: try_wait may park the
+// warp for a system-chosen time before it answers, which is what a long wait wants and a short bound
+// cannot afford.
+__device__ __forceinline__ long long bound_cycles(unsigned long long ns) {
+    return (long long)(ns < (1ull << 61) ? 2 * ns : (1ull << 62));
 }
+constexpr long long kShortBoundCycles = 2000000;      // 1 ms
+// Bounded wait, called by all 32 lanes of a warp; false when the CTA is aborting or the bound
+// expired (which starts an abort).  The outcome is voted on, so the lanes of a warp never part ways
+// before a warp-collective instruction (mma, shuffle, ballot).  Inline on purpose: a call here would
+// spill the caller's registers at every wait that is not satisfied at once, i.e. at most of them.
 __device__ __forceinline__ bool mbar_wait(uint64_t* b, uint32_t parity, volatile int* abort_flag,
-                                          unsigned long long limit_ns) {
+                                          const volatile long long* bound) {
     bool ok = mbar_test(b, parity);
-    if (!ok) ok = mbar_wait_slow(b, parity, abort_flag, limit_ns);     // kept out of line: the hot loop stays small
+    if (!ok) {
+        const long long t0 = clock64();
+        const long long lim = *bound;
+        const bool nb = lim < kShortBoundCycles;
+        for (;;) {
+#pragma unroll 1
+            for (int i = 0; i < 64 && !ok; ++i) {
+                ok = nb ? mbar_test(b, parity) : mbar_try(b, parity);
+                if (nb && clock64() - t0 > lim) break;
+            }
+            if (ok || *abort_flag) break;
+            if (clock64() - t0 > lim) { *abort_flag = 1; break; }
+        }
+    }
     return __all_sync(0xffffffffu, ok);
 }
 // bulk copy global -> shared with an L2 eviction-priority hint for the lines it brings in
@@ -201,7 +212,8 @@ k_head_stream(const HeadArgs a, Ctrl* ctrl, float* __restrict__ recs, const Geo 
     extern __shared__ __align__(128) uint8_t s_raw[];
     __shared__ uint64_t s_full[kMaxStages], s_empty[kMaxStages], s_pfull[2], s_pempty[2];
     __shared__ int s_last, s_abort, s_any_abort;
-    __shared__ int s_issued[kMaxStages];                 // fills requested per stage (for the drain after an abort)
+    __shared__ long long s_bound;                        // bound of a wait in SM cycles
+    __shared__ int s_issued[kMaxStages];                 // per stage: 0 = never requested, else 2 | parity of the latest fill
     __shared__ int s_rowok[kMaxB];                       // per hidden row: its temperature is usable
     __shared__ float s_xch[kMaxB];                       // merge: a row's lse, from its statistics warp to its candidate warp
     constexpr int KC = kNW * KBC * 32;                   // columns per chunk
@@ -233,13 +245,14 @@ k_head_stream(const HeadArgs a, Ctrl* ctrl, float* __restrict__ recs, const Geo 
         for (int s = 0; s < S; ++s) { mbar_init(&s_full[s], 1); mbar_init(&s_empty[s], kNW); s_issued[s] = 0; }
         for (int p = 0; p < 2; ++p) { mbar_init(&s_pfull[p], kNW); mbar_init(&s_pempty[p], B); }
         s_abort = 0;
+        s_bound = bound_cycles(kWaitLimitNs);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     for (int i = threadIdx.x; i < B * topk; i += kThreads) { topv[i] = -CUDART_INF_F; topj[i] = -1; }
     __syncthreads();
     VT_STAMP(0);
     volatile int* abort_flag = &s_abort;
-    unsigned long long wait_ns = kWaitLimitNs;
+    const volatile long long* wait_ns = &s_bound;
 
     // per-row state of warp b (identical in its four 8-lane groups); declared here so that the
     // record code after the loop sees it
@@ -255,8 +268,8 @@ k_head_stream(const HeadArgs a, Ctrl* ctrl, float* __restrict__ recs, const Geo 
     // warps that own no hidden row, so the epilogue warps are spared), in rotation.
     // W_trim is read once per step: its lines are the first to go when L2 needs room, so that the
     // records, the index mapper and h stay resident from step to step
-    uint64_t w_policy;
-    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(w_policy));
+    uint64_t w_policy;                                       // (not volatile: may be re-made where it is used)
+    asm("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(w_policy));
     const int n_items = (rb1 - rb0) * NCH;
     const int n_duty = (B < kNW) ? kNW - B : 1;
     int f_item = 0, f_rb = rb0, f_c = 0, f_s = 0, f_duty = kNW - 1;   // next item to fetch, its duty warp
@@ -270,7 +283,7 @@ k_head_stream(const HeadArgs a, Ctrl* ctrl, float* __restrict__ recs, const Geo 
                 const int col0 = f_c * KC;
                 const uint32_t cbytes = (uint32_t)(min(d, col0 + KC) - col0) * 2u;
                 if (lane == 0) {
-                    s_issued[f_s] += 1;
+                    s_issued[f_s] = 2 | (int)f_ph;           // requested at least once; parity of the latest fill
                     mbar_expect_tx(&s_full[f_s], cbytes * (uint32_t)nrows);
                 }
                 __syncwarp();
@@ -312,7 +325,7 @@ k_head_stream(const HeadArgs a, Ctrl* ctrl, float* __restrict__ recs, const Geo 
         }
     {
         const unsigned long long lim = ctrl->wait_ns;        // 0 = the default
-        if (lim) wait_ns = lim;
+        if (lim && threadIdx.x == 0) s_bound = bound_cycles(lim);   // (a race with early waiters only shortens or keeps their bound)
     }
     if (b < B) {
         const float T = a.temp[b];
@@ -418,8 +431,13 @@ k_head_stream(const HeadArgs a, Ctrl* ctrl, float* __restrict__ recs, const Geo 
             st_m = m_new;
         }
         if (a.uniforms) {
+            // g = -log(-log u): -log u from a short series in 1-u near 1 (where a fast logarithm's absolute
+            // error would dominate the tiny result), fast logarithms elsewhere
             const float uc = fminf(fmaxf(u_next, 0x1p-24f), 1.f - 0x1p-24f);
-            const float sc = z - logf(-logf(uc));
+            const float t1 = 1.f - uc;
+            const float lp = t1 * (1.f + t1 * (0.5f + t1 * (0.33333334f + t1 * (0.25f + t1 * 0.2f))));
+            const float L = uc > 0.95f ? lp : -__logf(uc);
+            const float sc = z - __logf(L);
             if (valid && sc > gb_s) { gb_s = sc; gb_j = j; gb_z = z; }
             const int jn = (rb + R + e_r) * kRows + e_v8;
             if (rb + R + e_r < rb1 && jn < K) u_next = __ldg(a.uniforms + (size_t)b * K + jn);
@@ -484,10 +502,10 @@ k_head_stream(const HeadArgs a, Ctrl* ctrl, float* __restrict__ recs, const Geo 
     if (warp == 0 && *abort_flag) {
         // drain: every stage that was requested must have landed before the CTA may leave
         for (int st = lane; st < S; st += 32) {
-            const int fills = s_issued[st];
-            if (fills > 0) {
+            const int last_fill = s_issued[st];
+            if (last_fill) {
                 const unsigned long long t0 = global_ns();
-                while (!mbar_try(&s_full[st], (uint32_t)((fills - 1) & 1)) && global_ns() - t0 < kWaitLimitNs) {}
+                while (!mbar_try(&s_full[st], (uint32_t)(last_fill & 1)) && global_ns() - t0 < kWaitLimitNs) {}
             }
         }
         __syncwarp();
