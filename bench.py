@@ -640,6 +640,31 @@ def small_case(vt, dev, args, peak_gbs):
         ms = e0.elapsed_time(e1) / args.steps
         print(json.dumps({"case": "hist", "n": n, "ms": ms, "gtok_s": n / ms / 1e6, "gbs": 4.0 * n / ms / 1e6,
                           "frac_of_measured": 4.0 * n / ms / 1e6 / peak_gbs}), flush=True)
+    elif args.case == "hist-ceiling":
+        # what shared-memory atomics can take on this stream: the same walk with all ids folded into
+        # directly indexed bins (one reduction per token, no lookup, no path for cold ids), next to the
+        # histogram proper on the same ids
+        n = args.hist_n
+        ids = vt_inputs.zipf_ids(n, V, 1.07, seed=1005, noise_frac=0.05, device=dev)
+        ws = vt.Workspace(vt.workspace_bytes(vt.VT_OP_BUILD_VOCAB, n, V, 32768), dev)
+        counts = torch.empty(V, dtype=torch.int32, device=dev)
+        folded = torch.empty(57344, dtype=torch.int32, device=dev)
+        rec = {"case": "hist-ceiling", "n": n, "bins": 57344}
+        for name, fn in (("folded", lambda: vt.vt_histogram_folded(ids, V, 57344, folded)),
+                         ("histogram", lambda: vt.vt_histogram(ids, V, counts=counts, ws=ws))):
+            for _ in range(args.warmup):
+                fn()
+            torch.cuda.synchronize()
+            e0, e1 = _events()
+            e0.record()
+            for _ in range(args.steps):
+                fn()
+            e1.record()
+            torch.cuda.synchronize()
+            ms = e0.elapsed_time(e1) / args.steps
+            rec[name] = {"ms": ms, "gtok_s": n / ms / 1e6, "gbs": 4.0 * n / ms / 1e6, "frac_of_measured": 4.0 * n / ms / 1e6 / peak_gbs}
+        rec["histogram_over_ceiling"] = rec["folded"]["ms"] / rec["histogram"]["ms"]
+        print(json.dumps(rec), flush=True)
     elif args.case == "dense":
         print(json.dumps(dict(case="dense", **dense_case(vt, dev, args.steps, args.warmup))), flush=True)
     else:
@@ -676,7 +701,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-extras", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--case", default="head", choices=["head", "hist", "tree", "dense", "stamps"],
+    ap.add_argument("--case", default="head", choices=["head", "hist", "hist-ceiling", "tree", "dense", "stamps"],
                     help="head: the full bench line (default); hist / tree / dense: a short run of the vocabulary "
                          "histogram (--hist-n ids), of the tree-drafting head or of the batched head, for profiler "
                          "captures; stamps: per-phase timeline of a head step from the instrumented build")

@@ -30,7 +30,7 @@ VT_CTRL_BYTES = 256
 EXPORTS = (
     "vt_workspace_bytes", "vt_workspace_init", "vt_workspace_set_wait_limit", "vt_read_status", "vt_status_str", "vt_launch_count",
     "vt_last_cuda_error",
-    "vt_histogram", "vt_select_topk", "vt_build_vocab", "vt_build_vocab_host", "vt_trim_head",
+    "vt_histogram", "vt_histogram_folded", "vt_select_topk", "vt_build_vocab", "vt_build_vocab_host", "vt_trim_head",
     "vt_draft_head", "vt_draft_head_debug", "vt_draft_head_host", "vt_select_topk_static",
     "vt_draft_head_overlapped", "vt_select_topp", "vt_select_minfreq", "vt_verify_greedy", "vt_mbsu", "vt_tree_expand", "vt_tree_rerank", "vt_draft_head_expand",
 )
@@ -64,6 +64,7 @@ def lib() -> ctypes.CDLL:
         L.vt_launch_count.restype = c_uint64
         L.vt_last_cuda_error.restype = c_char_p
         L.vt_histogram.argtypes = [c_void_p, c_int64, c_int32, c_void_p, c_int, c_void_p, c_size_t, c_void_p]
+        L.vt_histogram_folded.argtypes = [c_void_p, c_int64, c_int32, c_int32, c_void_p, c_void_p]
         L.vt_select_topk.argtypes = [c_void_p, c_int32, c_int32, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
         L.vt_select_topk_static.argtypes = [c_void_p, c_int32, c_int32, c_void_p, c_void_p, c_void_p]
         L.vt_select_topp.argtypes = [c_void_p, c_int32, c_double, c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
@@ -163,6 +164,17 @@ def vt_histogram(ids: torch.Tensor, V: int, counts: torch.Tensor | None = None, 
     ws = _ws(ws, workspace_bytes(VT_OP_HISTOGRAM, ids.numel(), V), ids)
     _check("vt_histogram", lib().vt_histogram(_ptr(ids), ids.numel(), V, _ptr(counts), int(bool(accumulate)),
                                               c_void_p(ws.ptr), ws.nbytes, _stream()))
+    return counts
+
+
+def vt_histogram_folded(ids: torch.Tensor, V: int, bins: int, counts: torch.Tensor | None = None) -> torch.Tensor:
+    """Measurement aid: counts[id mod bins] over the ids inside [0,V), all bins directly indexed in
+    shared memory (bins <= 57344)."""
+    _dev(ids, torch.int32, "ids")
+    if counts is None:
+        counts = torch.empty(bins, dtype=torch.int32, device=ids.device)
+    _dev(counts, torch.int32, "counts")
+    _check("vt_histogram_folded", lib().vt_histogram_folded(_ptr(ids), ids.numel(), V, bins, _ptr(counts), _stream()))
     return counts
 
 

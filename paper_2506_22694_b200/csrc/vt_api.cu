@@ -189,6 +189,13 @@ vt_status vt_histogram(const int32_t* ids, int64_t n, int32_t V, uint32_t* count
                                       base + VT_CTRL_BYTES, as_stream(stream)));
 }
 
+vt_status vt_histogram_folded(const int32_t* ids, int64_t n, int32_t V, int32_t bins, uint32_t* counts, void* stream) {
+    if (n < 0 || n >= ((int64_t)1 << 32) || V < 1 || bins < 1 || !counts || (n > 0 && !ids)) return VT_ERR_INVALID_ARG;
+    if (!aligned(ids, 4) || !aligned(counts, 4)) return VT_ERR_INVALID_ARG;
+    if (bins > VT_FOLDED_MAX_BINS) return VT_ERR_UNSUPPORTED;
+    return from_cuda(launch_hist_fold(ids, n, V, bins, counts, as_stream(stream)));
+}
+
 vt_status vt_select_topk(const uint32_t* counts, int32_t V, int32_t K, int32_t* map,
                          int32_t* inv_map, void* ws, size_t ws_bytes, void* stream) {
     if (!counts || !map || !inv_map || V < 1 || K < 1 || K > V) return VT_ERR_INVALID_ARG;

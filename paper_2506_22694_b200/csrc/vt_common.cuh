@@ -41,6 +41,8 @@ bool hist_supported(int32_t V);   // V the counting kernels take (bins or lookup
 cudaError_t launch_histogram(const int32_t* ids, int64_t n, int32_t V, uint32_t* counts,
                              int accumulate, Ctrl* ctrl, uint8_t* scratch, cudaStream_t s);
 
+cudaError_t launch_hist_fold(const int32_t* ids, int64_t n, int32_t V, int32_t bins, uint32_t* counts, cudaStream_t s);
+
 size_t select_scratch_bytes(int32_t V);
 cudaError_t launch_select_topk(const uint32_t* counts, int32_t V, int32_t K, int32_t* map,
                                int32_t* inv_map, uint8_t* scratch, cudaStream_t s);

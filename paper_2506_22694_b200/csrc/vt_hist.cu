@@ -58,6 +58,35 @@ __device__ __forceinline__ void stream_ids(const int32_t* __restrict__ ids, int6
     }
 }
 
+// Same walk, handing whole 128-bit loads (4 ids) to `tally4` and the ragged ends to `tally1`.
+template <class F4, class F1>
+__device__ __forceinline__ void stream_ids4(const int32_t* __restrict__ ids, int64_t n, F4&& tally4, F1&& tally1) {
+    const uintptr_t addr = reinterpret_cast<uintptr_t>(ids);
+    int64_t head = ((16 - (addr & 15)) & 15) >> 2;
+    if (head > n) head = n;
+    const int64_t nvec = (n - head) >> 2;
+    const int64_t tail0 = head + nvec * 4;
+    if (blockIdx.x == 0) {
+        if ((int64_t)threadIdx.x < head) tally1((uint32_t)ids[threadIdx.x]);
+        const int64_t t = tail0 + threadIdx.x;
+        if (t < n) tally1((uint32_t)ids[t]);
+    }
+    const uint4* vec = reinterpret_cast<const uint4*>(ids + head);
+    const int64_t v0 = nvec * blockIdx.x / gridDim.x;
+    const int64_t v1 = nvec * (blockIdx.x + 1) / gridDim.x;
+    for (int64_t v = v0 + threadIdx.x; v < v1; v += 4 * kThreads) {
+        uint4 a = ld_stream_u4(vec + v), b, c, d;
+        const bool pb = v + kThreads < v1, pc = v + 2 * kThreads < v1, pd = v + 3 * kThreads < v1;
+        if (pb) b = ld_stream_u4(vec + v + kThreads);
+        if (pc) c = ld_stream_u4(vec + v + 2 * kThreads);
+        if (pd) d = ld_stream_u4(vec + v + 3 * kThreads);
+        tally4(a.x, a.y, a.z, a.w);
+        if (pb) tally4(b.x, b.y, b.z, b.w);
+        if (pc) tally4(c.x, c.y, c.z, c.w);
+        if (pd) tally4(d.x, d.y, d.z, d.w);
+    }
+}
+
 __device__ __forceinline__ void report_bad(unsigned long long bad, Ctrl* ctrl) {
     for (int o = 16; o; o >>= 1) bad += __shfl_xor_sync(0xffffffffu, bad, o);
     if ((threadIdx.x & 31) == 0 && bad) {
@@ -257,15 +286,47 @@ k_hist_hot(const int32_t* __restrict__ ids, int64_t n, int32_t V, uint32_t* __re
     for (int i = threadIdx.x; i < H; i += kThreads) s_cnt[i] = 0;
     __syncthreads();
     unsigned long long bad = 0;
-    stream_ids(ids, n, [&](uint32_t id) {
-        if (id < (uint32_t)V) {
-            const uint32_t e = s_t16[id >> 4];
-            const uint32_t bit = 1u << (id & 15);
-            if (e & bit) atomicAdd(&s_cnt[(e >> 16) + __popc(e & (bit - 1))], 1u);
-            else atomicAdd(&counts[id], 1u);
+    const uint32_t tbl_addr = (uint32_t)__cvta_generic_to_shared(s_t16);
+    const uint32_t cnt_addr = (uint32_t)__cvta_generic_to_shared(s_cnt);
+    // One token, id < V known: a handful of integer instructions, one shared-memory load and one
+    // reduction -- into the token's shared-memory counter when its id is hot, into global memory
+    // when it is not -- chosen by a predicate: no branch, the warp never splits.
+    auto tally_in_range = [&](uint32_t id) {
+        asm volatile(
+            "{\n\t"
+            ".reg .pred ph;\n\t"
+            ".reg .b32 w, e, sh, bit, m, r, sl;\n\t"
+            ".reg .b64 ga;\n\t"
+            "shr.u32 w, %0, 4;\n\t"
+            "mad.lo.u32 w, w, 4, %1;\n\t"
+            "ld.shared.u32 e, [w];\n\t"
+            "and.b32 sh, %0, 15;\n\t"
+            "shl.b32 bit, 1, sh;\n\t"
+            "and.b32 r, e, bit;\n\t"
+            "setp.ne.u32 ph, r, 0;\n\t"
+            "add.u32 m, bit, -1;\n\t"
+            "and.b32 r, e, m;\n\t"
+            "popc.b32 r, r;\n\t"
+            "shr.u32 sl, e, 16;\n\t"
+            "add.u32 sl, sl, r;\n\t"
+            "mad.lo.u32 sl, sl, 4, %2;\n\t"
+            "@ph red.shared.add.u32 [sl], 1;\n\t"
+            "mad.wide.u32 ga, %0, 4, %3;\n\t"
+            "@!ph red.global.add.u32 [ga], 1;\n\t"
+            "}" ::"r"(id), "r"(tbl_addr), "r"(cnt_addr), "l"(counts) : "memory");
+    };
+    stream_ids4(ids, n, [&](uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+        // one range test per 128-bit load; ids outside [0, V) are rare and take the careful path
+        if (max(max(a, b), max(c, d)) < (uint32_t)V) {
+            tally_in_range(a); tally_in_range(b); tally_in_range(c); tally_in_range(d);
         } else {
-            ++bad;
+            if (a < (uint32_t)V) tally_in_range(a); else ++bad;
+            if (b < (uint32_t)V) tally_in_range(b); else ++bad;
+            if (c < (uint32_t)V) tally_in_range(c); else ++bad;
+            if (d < (uint32_t)V) tally_in_range(d); else ++bad;
         }
+    }, [&](uint32_t id) {
+        if (id < (uint32_t)V) tally_in_range(id); else ++bad;
     });
     __syncthreads();
     for (int i = threadIdx.x; i < 2 * T32; i += kThreads) {
@@ -282,13 +343,33 @@ k_hist_hot(const int32_t* __restrict__ ids, int64_t n, int32_t V, uint32_t* __re
     report_bad(bad, ctrl);
 }
 
-}  // namespace
-
-bool hist_supported(int32_t V) {
-    if (V < 1) return false;
-    if ((size_t)V * 4 <= kDynSmem) return true;
-    return ((size_t)V + 31) / 32 * 8 <= kMaxTableBytes;
+// ---- measurement aid: directly indexed bins, one shared-memory reduction per token, nothing else -------
+// counts[id mod bins] over the ids inside [0, V): what the shared-memory atomics of one SM can take on this
+// stream when no lookup and no cold path stand beside them.
+__global__ void __launch_bounds__(kThreads, 1)
+k_hist_fold(const int32_t* __restrict__ ids, int64_t n, int32_t V, int32_t bins, uint32_t* __restrict__ counts) {
+    extern __shared__ __align__(16) uint32_t s_bins[];
+    for (int i = threadIdx.x; i < bins; i += kThreads) s_bins[i] = 0;
+    __syncthreads();
+    const uint32_t nb = (uint32_t)bins;
+    const bool two_steps = (uint32_t)V <= 3u * nb;           // id mod bins by at most two subtractions
+    stream_ids(ids, n, [&](uint32_t id) {
+        if (id < (uint32_t)V) {
+            uint32_t b = id;
+            if (two_steps) { b = b >= nb ? b - nb : b; b = b >= nb ? b - nb : b; }
+            else b = b % nb;
+            atomicAdd(&s_bins[b], 1u);
+        }
+    });
+    __syncthreads();
+    for (int i = threadIdx.x; i < bins; i += kThreads) {
+        const int v = (i + blockIdx.x * 61) % bins;
+        const uint32_t c = s_bins[v];
+        if (c) atomicAdd(&counts[v], c);
+    }
 }
+
+}  // namespace
 
 // opt-in shared-memory sizes are per device: remember which devices have been set up
 static cudaError_t set_smem_once(const void* fn, size_t bytes, int (&done)[kMaxDevices]) {
@@ -299,6 +380,26 @@ static cudaError_t set_smem_once(const void* fn, size_t bytes, int (&done)[kMaxD
     e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
     if (e == cudaSuccess && dev >= 0 && dev < kMaxDevices) done[dev] = 1;
     return e;
+}
+
+cudaError_t launch_hist_fold(const int32_t* ids, int64_t n, int32_t V, int32_t bins, uint32_t* counts, cudaStream_t s) {
+    if (bins < 1 || (size_t)bins * 4 > kDynSmem) return cudaErrorInvalidValue;
+    cudaError_t e = cudaMemsetAsync(counts, 0, (size_t)bins * 4, s);
+    if (e != cudaSuccess || n == 0) return e;
+    static int done_fold[kMaxDevices] = {0};
+    e = set_smem_once(reinterpret_cast<const void*>(k_hist_fold), kDynSmem, done_fold);
+    if (e != cudaSuccess) return e;
+    int grid = (int)((n + 4095) / 4096);
+    if (grid > num_sms()) grid = num_sms();
+    k_hist_fold<<<grid, kThreads, (size_t)bins * 4, s>>>(ids, n, V, bins, counts);
+    count_launch();
+    return cudaGetLastError();
+}
+
+bool hist_supported(int32_t V) {
+    if (V < 1) return false;
+    if ((size_t)V * 4 <= kDynSmem) return true;
+    return ((size_t)V + 31) / 32 * 8 <= kMaxTableBytes;
 }
 
 HistPlan hist_plan(int32_t V) {

@@ -66,6 +66,17 @@ def test_histogram_skips_and_reports_out_of_range_ids(V):
     assert ws.read_status() == (0, 0, 0)                   # flags are cleared by the read
 
 
+@pytest.mark.parametrize("V,bins,n", [(128256, 57344, 1_000_003), (128256, 1000, 50_000), (300_000, 7, 100_001), (64, 64, 1000)])
+def test_folded_histogram_counts_ids_modulo_the_bins(V, bins, n):
+    ids = vt_inputs.zipf_ids(n, V, 1.07, seed=5, noise_frac=0.05, device=DEV)
+    ids[::997] = V + 3                                            # skipped
+    got = _u32(vt.vt_histogram_folded(ids, V, bins))
+    full, _ = oracle.histogram(ids.cpu().numpy(), V)              # the oracle's histogram, folded on the host
+    ref = np.zeros(bins, dtype=np.uint64)
+    np.add.at(ref, np.arange(V) % bins, full)
+    assert np.array_equal(got, ref)
+
+
 def test_histogram_degenerate_streams():
     V = 128256
     ws = vt.Workspace(vt.workspace_bytes(vt.VT_OP_HISTOGRAM, 1 << 20, V))
