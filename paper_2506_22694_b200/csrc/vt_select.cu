@@ -25,13 +25,19 @@ constexpr int kCluster = 8;
 constexpr int kThreads = 1024;
 constexpr int kWarps = kThreads / 32;
 constexpr int kDigits = 256;
+constexpr int kFine = 4096;                      // buckets of the selection pass (3328 in use)
+constexpr int kSortCap = 16384;                  // 64-bit keys one CTA ranks in shared memory
+constexpr int kCountCap = 2048;                  // largest bucket ranked by counting its greater keys
+constexpr uint32_t kWorkCap = 6u << 10;          // key comparisons one CTA spends on that at most, in units of 1024 (~6 K per thread)
+constexpr size_t kSelectSmem = sizeof(uint32_t) * 4 * kFine + sizeof(unsigned long long) * kSortCap;
+static_assert(sizeof(uint32_t) * 4 * kFine >= sizeof(uint32_t) * kWarps * kDigits, "the full ranking reuses the bucket arrays");
 
-__global__ void __cluster_dims__(kCluster, 1, 1) __launch_bounds__(kThreads, 1)
-k_select_sort(const uint32_t* counts, int32_t V, int32_t K, int32_t* map, int32_t* inv_map, uint32_t* keyA, uint32_t* valA, uint32_t* keyB,
-              uint32_t* valB) {
-    cg::cluster_group cluster = cg::this_cluster();
+// ---- full ranking: least-significant-digit radix sort over the whole cluster -------------------------
+// s_wcnt: [kWarps][kDigits] words of shared memory.
+__device__ void lsd_rank_all(cg::cluster_group& cluster, const uint32_t* counts, int32_t V, int32_t K, int32_t* map,
+                             int32_t* inv_map, uint32_t* keyA, uint32_t* valA, uint32_t* keyB, uint32_t* valB,
+                             uint32_t (*s_wcnt)[kDigits]) {
     const unsigned rank = cluster.block_rank();
-    __shared__ uint32_t s_wcnt[kWarps][kDigits];   // per-warp digit counts, then running offsets
     __shared__ uint32_t s_tot[kDigits];            // this CTA's digit totals (read by the peers)
     __shared__ uint32_t s_base[kDigits];           // global start of (digit, this CTA)
     __shared__ uint32_t s_scan[kDigits / 32 + 1];
@@ -138,6 +144,173 @@ k_select_sort(const uint32_t* counts, int32_t V, int32_t K, int32_t* map, int32_
         if (j < K) map[j] = v;
         inv_map[v] = j < K ? j : -1;
     }
+}
+
+// Order-preserving bucket of a count: its leading one and the seven bits behind it (counts below 128 map to
+// themselves).  3328 buckets whose widths grow with the count, so a heavy-tailed histogram spreads over
+// many of them and a bucket near the cut holds a few hundred ids at most.
+__device__ __forceinline__ uint32_t fine_bucket(uint32_t c) {
+    if (c < 128u) return c;
+    const int e = 31 - __clz(c);                                       // 7 .. 31
+    return 128u + (uint32_t)(e - 7) * 128u + ((c >> (e - 7)) & 127u);  // 128 .. 3327
+}
+
+// Radix select (Eq. 1, Top-K(c,k)): one pass of bucket counts finds the bucket that holds the K-th key;
+// only the keys of that bucket and of the buckets above it -- K of them plus part of one bucket -- are
+// moved, bucket by bucket, into a scratch array, which is thereby already in bucket order.  Each CTA of
+// the cluster then takes a contiguous run of whole buckets into shared memory and gives every key its
+// place inside its bucket by counting the bucket's greater keys (64-bit keys (count, ~id): unique, so
+// the result is the one right answer; buckets are small, so the counting is cheap).  Everything below
+// the cut is never touched again.  When a run does not fit a CTA's shared memory (K close to V) or a
+// bucket is too large to rank by counting (counts that all fall into one bucket), the full ranking
+// above takes over.
+__global__ void __cluster_dims__(kCluster, 1, 1) __launch_bounds__(kThreads, 1)
+k_select_sort(const uint32_t* counts, int32_t V, int32_t K, int32_t* map, int32_t* inv_map, uint32_t* keyA, uint32_t* valA, uint32_t* keyB,
+              uint32_t* valB) {
+    cg::cluster_group cluster = cg::this_cluster();
+    const unsigned rank = cluster.block_rank();
+    extern __shared__ __align__(16) uint8_t s_dyn[];
+    uint32_t* s_hist = reinterpret_cast<uint32_t*>(s_dyn);             // [kFine] this CTA's bucket counts (read by the peers)
+    uint32_t* s_gstart = s_hist + kFine;                               // [kFine] start of the bucket in the ranking
+    uint32_t* s_gsize = s_gstart + kFine;                              // [kFine] its size over all CTAs
+    uint32_t* s_next = s_gsize + kFine;                                // [kFine] scratch position of this CTA's next key
+    unsigned long long* s_run = reinterpret_cast<unsigned long long*>(s_next + kFine);     // [kSortCap]
+    __shared__ uint32_t s_warp[kWarps + 1];
+    __shared__ uint32_t s_load[kCluster];          // keys each CTA would have to rank
+    __shared__ uint32_t s_work[kCluster];          // key comparisons that would take: sum of squared bucket sizes, in units of 1024
+    __shared__ uint32_t s_T;
+    __shared__ int s_cut, s_lo, s_hi, s_big;
+
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    // ids of this CTA: a contiguous slice walked with coalesced loads, eight in flight per thread
+    const int slice = (V + kCluster - 1) / kCluster;
+    const int i0 = min(V, (int)rank * slice), i1 = min(V, i0 + slice);
+    constexpr int kInFlight = 8;
+    unsigned long long* pairs = reinterpret_cast<unsigned long long*>(keyA);       // [V] 64-bit keys (keyA and valA are adjacent)
+
+    for (int i = threadIdx.x; i < kFine; i += kThreads) s_hist[i] = 0;
+    if (threadIdx.x < kCluster) { s_load[threadIdx.x] = 0; s_work[threadIdx.x] = 0u; }
+    if (threadIdx.x == 0) { s_cut = 0; s_lo = 0x7fffffff; s_hi = 0; s_big = 0; }
+    __syncthreads();
+    // phase 1: bucket counts (descending order: inverted bucket index)
+    for (int i = i0 + (int)threadIdx.x; i < i1; i += kThreads * kInFlight) {
+        uint32_t c[kInFlight];
+#pragma unroll
+        for (int q = 0; q < kInFlight; ++q) c[q] = i + q * kThreads < i1 ? __ldg(counts + i + q * kThreads) : 0u;
+#pragma unroll
+        for (int q = 0; q < kInFlight; ++q)
+            if (i + q * kThreads < i1) atomicAdd(&s_hist[kFine - 1 - fine_bucket(c[q])], 1u);
+    }
+    cluster.sync();
+    // phase 2: start of every bucket in descending order (each thread owns kFine / kThreads neighbouring
+    // buckets), the bucket of the K-th key, who ranks what
+    constexpr int BPT = kFine / kThreads;
+    static_assert(BPT == 4, "one 128-bit load per peer and thread");
+    uint32_t tot[BPT], mine_before[BPT], sum = 0;
+#pragma unroll
+    for (int q = 0; q < BPT; ++q) { tot[q] = 0; mine_before[q] = 0; }
+    uint4 pv[kCluster];
+#pragma unroll
+    for (unsigned c = 0; c < kCluster; ++c)                         // all eight remote loads in flight
+        pv[c] = reinterpret_cast<const uint4*>(cluster.map_shared_rank(s_hist, c))[threadIdx.x];
+#pragma unroll
+    for (unsigned c = 0; c < kCluster; ++c) {
+        const uint32_t t4[BPT] = {pv[c].x, pv[c].y, pv[c].z, pv[c].w};
+#pragma unroll
+        for (int q = 0; q < BPT; ++q) {
+            if (c < rank) mine_before[q] += t4[q];
+            tot[q] += t4[q];
+        }
+    }
+#pragma unroll
+    for (int q = 0; q < BPT; ++q) sum += tot[q];
+    uint32_t incl = sum;
+    for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t y = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += y;
+    }
+    if (lane == 31) s_warp[warp] = incl;
+    __syncthreads();
+    uint32_t start = incl - sum;
+    for (int w = 0; w < warp; ++w) start += s_warp[w];
+#pragma unroll
+    for (int q = 0; q < BPT; ++q) {
+        const int b = threadIdx.x * BPT + q;
+        s_gstart[b] = start;
+        s_gsize[b] = tot[q];
+        s_next[b] = start + mine_before[q];
+        if (start < (uint32_t)K && start + tot[q] >= (uint32_t)K) { s_cut = b; s_T = start + tot[q]; }   // exactly one bucket
+        start += tot[q];
+    }
+    __syncthreads();
+    const int cut = s_cut;
+    const uint32_t T = s_T;                             // keys to be ranked = end of the cut bucket
+#pragma unroll
+    for (int q = 0; q < BPT; ++q) {
+        const int b = threadIdx.x * BPT + q;
+        if (b <= cut && tot[q] > 0) {
+            const uint32_t st = s_gstart[b];
+            const unsigned owner = min((unsigned)kCluster - 1u, (unsigned)(((unsigned long long)st * kCluster) / T));
+            atomicAdd(&s_load[owner], tot[q]);
+            if (tot[q] > (uint32_t)kCountCap) s_big = 1;
+            else atomicAdd(&s_work[owner], (tot[q] * tot[q] + 1023u) >> 10);
+            if (owner == rank) {
+                atomicMin(&s_lo, (int)st);
+                atomicMax(&s_hi, (int)(st + tot[q]));
+            }
+        }
+    }
+    __syncthreads();
+    bool fits = s_big == 0;
+    for (int c = 0; c < kCluster; ++c) fits = fits && s_load[c] <= (uint32_t)kSortCap && s_work[c] <= kWorkCap;
+    if (!fits) {                                        // the same decision in every CTA (same inputs)
+        cluster.sync();                                 // peers are done reading this CTA's counts
+        lsd_rank_all(cluster, counts, V, K, map, inv_map, keyA, valA, keyB, valB,
+                     reinterpret_cast<uint32_t (*)[kDigits]>(s_dyn));
+        return;
+    }
+    // phase 3: move the keys of the buckets down to the cut into bucket order; order inside a bucket is
+    // whatever the atomics make of it; ids below the cut are pruned here
+    for (int i = i0 + (int)threadIdx.x; i < i1; i += kThreads * kInFlight) {
+        uint32_t c[kInFlight];
+#pragma unroll
+        for (int q = 0; q < kInFlight; ++q) c[q] = i + q * kThreads < i1 ? __ldg(counts + i + q * kThreads) : 0u;
+#pragma unroll
+        for (int q = 0; q < kInFlight; ++q) {
+            const int id = i + q * kThreads;
+            if (id >= i1) continue;
+            const int b = (int)(kFine - 1 - fine_bucket(c[q]));
+            if (b <= cut) pairs[atomicAdd(&s_next[b], 1u)] = ((unsigned long long)c[q] << 32) | (0xffffffffu - (uint32_t)id);
+            else inv_map[id] = -1;
+        }
+    }
+    __threadfence();
+    cluster.sync();
+    // phase 4: this CTA's run of buckets into shared memory; place of a key = start of its bucket + number
+    // of greater keys in the bucket (neighbouring lanes mostly share a bucket: the reads are broadcasts)
+    const int r0 = s_lo, n = s_hi > s_lo ? s_hi - s_lo : 0;
+    for (int j = threadIdx.x; j < n; j += kThreads) s_run[j] = __ldcg(pairs + r0 + j);
+    __syncthreads();
+    for (int j = threadIdx.x; j < n; j += kThreads) {
+        const unsigned long long key = s_run[j];
+        const int b = (int)(kFine - 1 - fine_bucket((uint32_t)(key >> 32)));
+        const int bs = (int)s_gstart[b] - r0, be = bs + (int)s_gsize[b];
+        int r = 0;
+        for (int i = bs; i < be; ++i) r += s_run[i] > key ? 1 : 0;
+        const int rk = r0 + bs + r;
+        const int32_t v = (int32_t)(0xffffffffu - (uint32_t)key);
+        if (rk < K) map[rk] = v;
+        inv_map[v] = rk < K ? rk : -1;
+    }
+}
+
+// The full ranking alone, for calls that want (nearly) all of it anyway.
+__global__ void __cluster_dims__(kCluster, 1, 1) __launch_bounds__(kThreads, 1)
+k_select_full(const uint32_t* counts, int32_t V, int32_t K, int32_t* map, int32_t* inv_map, uint32_t* keyA, uint32_t* valA,
+              uint32_t* keyB, uint32_t* valB) {
+    cg::cluster_group cluster = cg::this_cluster();
+    extern __shared__ __align__(16) uint8_t s_dyn[];
+    lsd_rank_all(cluster, counts, V, K, map, inv_map, keyA, valA, keyB, valB, reinterpret_cast<uint32_t (*)[kDigits]>(s_dyn));
 }
 
 // Cut of a full ranking at a data-dependent K (the Method section's Top-P and minimum-frequency
@@ -250,7 +423,19 @@ cudaError_t launch_select_topk(const uint32_t* counts, int32_t V, int32_t K, int
     uint32_t* valA = reinterpret_cast<uint32_t*>(scratch + seg);
     uint32_t* keyB = reinterpret_cast<uint32_t*>(scratch + 2 * seg);
     uint32_t* valB = reinterpret_cast<uint32_t*>(scratch + 3 * seg);
-    k_select_sort<<<kCluster, kThreads, 0, s>>>(counts, V, K, map, inv_map, keyA, valA, keyB, valB);
+    static int attr_done[64] = {0};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64 || !attr_done[dev]) {
+        e = cudaFuncSetAttribute(k_select_sort, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSelectSmem);
+        if (e != cudaSuccess) return e;
+        if (dev >= 0 && dev < 64) attr_done[dev] = 1;
+    }
+    if ((long long)K * 2 > V)          // more than half the ranking is wanted: rank everything, select nothing
+        k_select_full<<<kCluster, kThreads, sizeof(uint32_t) * kWarps * kDigits, s>>>(counts, V, K, map, inv_map, keyA, valA, keyB, valB);
+    else
+        k_select_sort<<<kCluster, kThreads, kSelectSmem, s>>>(counts, V, K, map, inv_map, keyA, valA, keyB, valB);
     count_launch();
     return cudaGetLastError();
 }
