@@ -315,10 +315,38 @@ k_hist_hot(const int32_t* __restrict__ ids, int64_t n, int32_t V, uint32_t* __re
             "@!ph red.global.add.u32 [ga], 1;\n\t"
             "}" ::"r"(id), "r"(tbl_addr), "r"(cnt_addr), "l"(counts) : "memory");
     };
+    // Four tokens at once, all in range: the four lookups are requested back to back before anything waits
+    // for one of them, so a warp has four shared-memory loads in flight instead of one.
+    auto tally4_in_range = [&](uint32_t i0, uint32_t i1, uint32_t i2, uint32_t i3) {
+        asm volatile(
+            "{\n\t"
+            ".reg .pred p0, p1, p2, p3;\n\t"
+            ".reg .b32 w0, w1, w2, w3, e0, e1, e2, e3, b0, b1, b2, b3, r0, r1, r2, r3, s0, s1, s2, s3;\n\t"
+            ".reg .b64 g0, g1, g2, g3;\n\t"
+            "shr.u32 w0, %0, 4;\n\t shr.u32 w1, %1, 4;\n\t shr.u32 w2, %2, 4;\n\t shr.u32 w3, %3, 4;\n\t"
+            "mad.lo.u32 w0, w0, 4, %4;\n\t mad.lo.u32 w1, w1, 4, %4;\n\t mad.lo.u32 w2, w2, 4, %4;\n\t mad.lo.u32 w3, w3, 4, %4;\n\t"
+            "ld.shared.u32 e0, [w0];\n\t ld.shared.u32 e1, [w1];\n\t ld.shared.u32 e2, [w2];\n\t ld.shared.u32 e3, [w3];\n\t"
+            "and.b32 b0, %0, 15;\n\t and.b32 b1, %1, 15;\n\t and.b32 b2, %2, 15;\n\t and.b32 b3, %3, 15;\n\t"
+            "shl.b32 b0, 1, b0;\n\t shl.b32 b1, 1, b1;\n\t shl.b32 b2, 1, b2;\n\t shl.b32 b3, 1, b3;\n\t"
+            "mad.wide.u32 g0, %0, 4, %6;\n\t mad.wide.u32 g1, %1, 4, %6;\n\t mad.wide.u32 g2, %2, 4, %6;\n\t mad.wide.u32 g3, %3, 4, %6;\n\t"
+            "and.b32 r0, e0, b0;\n\t and.b32 r1, e1, b1;\n\t and.b32 r2, e2, b2;\n\t and.b32 r3, e3, b3;\n\t"
+            "setp.ne.u32 p0, r0, 0;\n\t setp.ne.u32 p1, r1, 0;\n\t setp.ne.u32 p2, r2, 0;\n\t setp.ne.u32 p3, r3, 0;\n\t"
+            "add.u32 b0, b0, -1;\n\t add.u32 b1, b1, -1;\n\t add.u32 b2, b2, -1;\n\t add.u32 b3, b3, -1;\n\t"
+            "and.b32 r0, e0, b0;\n\t and.b32 r1, e1, b1;\n\t and.b32 r2, e2, b2;\n\t and.b32 r3, e3, b3;\n\t"
+            "popc.b32 r0, r0;\n\t popc.b32 r1, r1;\n\t popc.b32 r2, r2;\n\t popc.b32 r3, r3;\n\t"
+            "shr.u32 s0, e0, 16;\n\t shr.u32 s1, e1, 16;\n\t shr.u32 s2, e2, 16;\n\t shr.u32 s3, e3, 16;\n\t"
+            "add.u32 s0, s0, r0;\n\t add.u32 s1, s1, r1;\n\t add.u32 s2, s2, r2;\n\t add.u32 s3, s3, r3;\n\t"
+            "mad.lo.u32 s0, s0, 4, %5;\n\t mad.lo.u32 s1, s1, 4, %5;\n\t mad.lo.u32 s2, s2, 4, %5;\n\t mad.lo.u32 s3, s3, 4, %5;\n\t"
+            "@p0 red.shared.add.u32 [s0], 1;\n\t @p1 red.shared.add.u32 [s1], 1;\n\t"
+            "@p2 red.shared.add.u32 [s2], 1;\n\t @p3 red.shared.add.u32 [s3], 1;\n\t"
+            "@!p0 red.global.add.u32 [g0], 1;\n\t @!p1 red.global.add.u32 [g1], 1;\n\t"
+            "@!p2 red.global.add.u32 [g2], 1;\n\t @!p3 red.global.add.u32 [g3], 1;\n\t"
+            "}" ::"r"(i0), "r"(i1), "r"(i2), "r"(i3), "r"(tbl_addr), "r"(cnt_addr), "l"(counts) : "memory");
+    };
     stream_ids4(ids, n, [&](uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
         // one range test per 128-bit load; ids outside [0, V) are rare and take the careful path
         if (max(max(a, b), max(c, d)) < (uint32_t)V) {
-            tally_in_range(a); tally_in_range(b); tally_in_range(c); tally_in_range(d);
+            tally4_in_range(a, b, c, d);
         } else {
             if (a < (uint32_t)V) tally_in_range(a); else ++bad;
             if (b < (uint32_t)V) tally_in_range(b); else ++bad;
