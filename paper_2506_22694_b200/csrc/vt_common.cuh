@@ -33,6 +33,9 @@ __device__ __forceinline__ size_t align_up_dev(size_t x, size_t a) { return (x +
 struct HistPlan {
     bool small;            // all bins fit in one CTA's shared memory
     size_t off_sample;     // uint32 [V]   sampled counts
+    size_t off_packed;     // uint32 [V]   what the packed kernel counted (only when three bins per word fit)
+    size_t off_gate;       // uint32 [4]   {recount, -, skipped ids (64 bits)} of the packed kernel
+    size_t clear_bytes;    // the scratch prefix every call zeroes
     size_t off_table;      // uint2  [ceil(V/32)] hot-bin table {bitmap word, slot base}
     size_t bytes;          // scratch after the control block
 };

@@ -4,10 +4,14 @@
 // per-token work stays in shared memory:
 //   * V * 4 bytes fit in one CTA's shared memory  -> every CTA keeps a private copy of all bins
 //     (k_hist_small) and flushes the non-zero ones at the end.
-//   * otherwise (Llama-3: 128256 bins = 513 KB) a short pre-pass samples the stream, picks the
-//     hottest bins that fit (about 49.8 K of them), and the main pass keeps those in shared
-//     memory; the rare cold tokens go to L2 with one red.global each.  The hot set only steers
-//     traffic: counts are exact whichever bins were picked.
+//   * ceil(V / 3) * 4 bytes fit (Llama-3: 128256 bins = 171 KB)  -> every CTA still keeps all bins,
+//     three 10-bit fields to a word (k_hist_packed): one shared-memory add per token and nothing else.
+//     A field hands 512 counts on to global memory whenever it gets there; the add that would wrap a
+//     field notices, and the stream is then counted again by the kernels of the next case.
+//   * otherwise a short pre-pass samples the stream, picks the hottest bins that fit (about 49.8 K of
+//     them for 128256 bins), and the main pass keeps those in shared memory; the rare cold tokens go
+//     to L2 with one red.global each.  The hot set only steers traffic: counts are exact whichever
+//     bins were picked.
 //       hot lookup: entry[id >> 4] = {16 membership bits, 16-bit slot of the group's first member};
 //       slot = base + popc(bits & below(id)), one 4-byte shared load per token.
 #include "vt_common.cuh"
@@ -117,10 +121,8 @@ k_hist_small(const int32_t* __restrict__ ids, int64_t n, int32_t V, uint32_t* __
 }
 
 // ---- pre-pass 1: sample the stream into sample[V] through a per-CTA aggregating cache -----------
-__global__ void __launch_bounds__(kThreads, 1)
-k_hist_sample(const int32_t* __restrict__ ids, int64_t n, int32_t V, uint32_t* __restrict__ sample) {
-    __shared__ int s_tag[kSampleSlots];
-    __shared__ uint32_t s_cnt[kSampleSlots];
+__device__ __forceinline__ void sample_stream(const int32_t* __restrict__ ids, int64_t n, int32_t V,
+                                              uint32_t* __restrict__ sample, int* s_tag, uint32_t* s_cnt) {
     for (int i = threadIdx.x; i < kSampleSlots; i += kThreads) { s_tag[i] = -1; s_cnt[i] = 0; }
     __syncthreads();
     const int64_t lo = n * blockIdx.x / gridDim.x;
@@ -137,6 +139,13 @@ k_hist_sample(const int32_t* __restrict__ ids, int64_t n, int32_t V, uint32_t* _
     __syncthreads();
     for (int i = threadIdx.x; i < kSampleSlots; i += kThreads)
         if (s_tag[i] >= 0) atomicAdd(&sample[s_tag[i]], s_cnt[i]);
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+k_hist_sample(const int32_t* __restrict__ ids, int64_t n, int32_t V, uint32_t* __restrict__ sample) {
+    __shared__ int s_tag[kSampleSlots];
+    __shared__ uint32_t s_cnt[kSampleSlots];
+    sample_stream(ids, n, V, sample, s_tag, s_cnt);
 }
 
 // Exclusive scan over one value per thread (kThreads threads); returns the prefix, *total the sum.
@@ -167,8 +176,10 @@ __device__ uint32_t block_excl_scan(uint32_t x, uint32_t* s_warp /*[33]*/, uint3
 // ---- pre-pass 2: choose at most H hot bins from the sampled counts, build the lookup table ------
 // hot = sampled count >= tau, plus (in id order) as many bins with count == tau-1 as still fit.
 __global__ void __launch_bounds__(kThreads, 1)
-k_hist_pick(const uint32_t* __restrict__ sample, int32_t V, int32_t H, uint2* __restrict__ table) {
+k_hist_pick(const uint32_t* __restrict__ sample, int32_t V, int32_t H, uint2* __restrict__ table,
+            const uint32_t* __restrict__ gate) {
     extern __shared__ __align__(16) uint8_t s_dyn[];
+    if (gate && *gate == 0) return;                        // the packed count stood: nothing to recount
     __shared__ uint32_t s_hist[kPickBins];
     __shared__ uint32_t s_warp[33];
     __shared__ uint32_t s_definite;
@@ -270,8 +281,9 @@ k_hist_pick(const uint32_t* __restrict__ sample, int32_t V, int32_t H, uint2* __
 // ---- main pass: hot bins in shared memory, cold bins through L2 ----------------------------------
 __global__ void __launch_bounds__(kThreads, 1)
 k_hist_hot(const int32_t* __restrict__ ids, int64_t n, int32_t V, uint32_t* __restrict__ counts,
-           const uint2* __restrict__ table, int32_t H, Ctrl* ctrl) {
+           const uint2* __restrict__ table, int32_t H, Ctrl* ctrl, const uint32_t* __restrict__ gate) {
     extern __shared__ __align__(16) uint8_t s_raw[];
+    if (gate && *gate == 0) return;
     const int T32 = (V + 31) >> 5;
     // The lookup is repacked for the main pass: one 4-byte word per 16 ids = {16 membership bits,
     // 16-bit slot of the first member} -- a 4-byte gather costs half the shared-memory wavefronts of
@@ -371,6 +383,92 @@ k_hist_hot(const int32_t* __restrict__ ids, int64_t n, int32_t V, uint32_t* __re
     report_bad(bad, ctrl);
 }
 
+// ---- every bin in shared memory, three 10-bit fields to a word -----------------------------------------
+// Word w holds the counters of ids w, W + w and 2W + w (W = ceil(V / 3)).  Each token is one returning
+// shared-memory add of 1 << (10 * field); the thread looks at the field's old value before it touches the
+// next token.  The add that takes a field from kSpill-1 to kSpill subtracts kSpill again and credits them
+// to out[id] in global memory, so a field holds fewer than kSpill counts plus whatever other threads add
+// between those two operations: at most one add per other thread of the CTA is in flight at any time,
+// which keeps a field under 2 * kSpill as long as no single token makes up half of the stream.  An add that
+// finds kFieldMax in its field has carried into the neighbour: it raises the gate, and the launcher's
+// next kernels throw this count away and count the stream again with the hot / cold kernels.
+constexpr uint32_t kFieldBits = 10, kFieldMax = (1u << kFieldBits) - 1, kSpill = 512;
+constexpr int kGateWords = 4;                  // {recount, unused, skipped ids (64 bits)}
+
+__global__ void __launch_bounds__(kThreads, 1)
+k_hist_packed(const int32_t* __restrict__ ids, int64_t n, int32_t V, uint32_t W, uint32_t* __restrict__ out,
+              uint32_t* __restrict__ gate) {
+    extern __shared__ __align__(16) uint32_t s_fields[];
+    for (uint32_t i = threadIdx.x; i < W; i += kThreads) s_fields[i] = 0;
+    __syncthreads();
+    unsigned long long bad = 0;
+    uint32_t wrapped = 0;
+    const uint32_t W2 = 2 * W;
+    auto tally_in_range = [&](uint32_t id) {
+        const uint32_t f = (id >= W) + (id >= W2);
+        const uint32_t w = id - f * W, sh = f * kFieldBits;
+        const uint32_t fld = (atomicAdd(&s_fields[w], 1u << sh) >> sh) & kFieldMax;
+        if ((fld & (kSpill - 1)) == kSpill - 1) {           // kSpill-1 or kFieldMax: one add in kSpill gets here
+            if (fld == kFieldMax) {
+                wrapped = 1;
+            } else {
+                atomicSub(&s_fields[w], kSpill << sh);
+                atomicAdd(&out[id], kSpill);
+            }
+        }
+    };
+    auto tally1 = [&](uint32_t id) {
+        if (id < (uint32_t)V) tally_in_range(id); else ++bad;
+    };
+    stream_ids4(ids, n, [&](uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+        if (max(max(a, b), max(c, d)) < (uint32_t)V) {       // one range test per 128-bit load
+            tally_in_range(a); tally_in_range(b); tally_in_range(c); tally_in_range(d);
+        } else {
+            tally1(a); tally1(b); tally1(c); tally1(d);
+        }
+    }, tally1);
+    __syncthreads();
+    for (uint32_t i = threadIdx.x; i < W; i += kThreads) {
+        const uint32_t w = (i + blockIdx.x * 61u) % W;       // de-phase the CTAs' flushes
+        const uint32_t x = s_fields[w];
+#pragma unroll
+        for (uint32_t f = 0; f < 3; ++f) {
+            const uint32_t c = (x >> (f * kFieldBits)) & kFieldMax, id = f * W + w;
+            if (c && id < (uint32_t)V) atomicAdd(&out[id], c);
+        }
+    }
+    if (wrapped) atomicOr(&gate[0], 1u);
+    for (int o = 16; o; o >>= 1) bad += __shfl_xor_sync(0xffffffffu, bad, o);
+    if ((threadIdx.x & 31) == 0 && bad) atomicAdd(reinterpret_cast<unsigned long long*>(gate + 2), bad);
+}
+
+// After the packed count: if it stood, counts (+)= packed and the skipped ids are reported; if a field
+// wrapped, counts is left as the recount needs it (zero unless accumulating) and the recount's sampling
+// pre-pass runs here.
+__global__ void __launch_bounds__(kThreads, 1)
+k_hist_settle(const int32_t* __restrict__ ids, int64_t n, int32_t V, const uint32_t* __restrict__ packed,
+              uint32_t* __restrict__ counts, int accumulate, uint32_t* __restrict__ sample,
+              const uint32_t* __restrict__ gate, Ctrl* ctrl) {
+    __shared__ int s_tag[kSampleSlots];
+    __shared__ uint32_t s_cnt[kSampleSlots];
+    const bool recount = gate[0] != 0;
+    for (int v = blockIdx.x * kThreads + threadIdx.x; v < V; v += gridDim.x * kThreads) {
+        const uint32_t c = recount ? 0u : packed[v];
+        counts[v] = accumulate ? counts[v] + c : c;
+    }
+    if (!recount) {
+        if (blockIdx.x == 0 && threadIdx.x == 0) {
+            const unsigned long long bad = *reinterpret_cast<const unsigned long long*>(gate + 2);
+            if (bad) {
+                atomicAdd(&ctrl->n_bad, bad);
+                atomicOr(&ctrl->flags, (uint32_t)VT_FLAG_BAD_ID);
+            }
+        }
+        return;
+    }
+    sample_stream(ids, n, V, sample, s_tag, s_cnt);
+}
+
 // ---- measurement aid: directly indexed bins, one shared-memory reduction per token, nothing else -------
 // counts[id mod bins] over the ids inside [0, V): what the shared-memory atomics of one SM can take on this
 // stream when no lookup and no cold path stand beside them.
@@ -430,13 +528,19 @@ bool hist_supported(int32_t V) {
     return ((size_t)V + 31) / 32 * 8 <= kMaxTableBytes;
 }
 
+static bool packed_fits(int32_t V) { return ((size_t)V + 2) / 3 * 4 <= kDynSmem; }
+
 HistPlan hist_plan(int32_t V) {
     HistPlan p{};
     p.small = (size_t)V * 4 <= kDynSmem;
-    if (p.small) { p.off_sample = p.off_table = 0; p.bytes = 0; return p; }
+    if (p.small) { p.off_sample = p.off_packed = p.off_gate = p.off_table = 0; p.bytes = 0; return p; }
     const size_t T32 = ((size_t)V + 31) / 32;
+    // sample, packed counts and gate lie together: one memset clears all three
     p.off_sample = 0;
-    p.off_table = align_up((size_t)V * 4, 256);
+    p.off_packed = (size_t)V * 4;
+    p.off_gate = packed_fits(V) ? 2 * (size_t)V * 4 : p.off_packed;
+    p.clear_bytes = packed_fits(V) ? p.off_gate + kGateWords * 4 : (size_t)V * 4;
+    p.off_table = align_up(p.clear_bytes, 256);
     p.bytes = p.off_table + align_up(T32 * 8, 256);
     return p;
 }
@@ -444,12 +548,13 @@ HistPlan hist_plan(int32_t V) {
 cudaError_t launch_histogram(const int32_t* ids, int64_t n, int32_t V, uint32_t* counts,
                              int accumulate, Ctrl* ctrl, uint8_t* scratch, cudaStream_t s) {
     cudaError_t e;
-    if (!accumulate) {
+    const HistPlan p = hist_plan(V);
+    const bool packed_path = !p.small && packed_fits(V) && n != 0;
+    if (!accumulate && !packed_path) {                     // (the packed path's second kernel writes every count)
         e = cudaMemsetAsync(counts, 0, (size_t)V * 4, s);
         if (e != cudaSuccess) return e;
     }
     if (n == 0) return cudaSuccess;
-    const HistPlan p = hist_plan(V);
     const int sms = num_sms();
     // enough CTAs to fill the chip, never more than one per 4096 ids
     int grid = (int)((n + 4095) / 4096);
@@ -469,21 +574,36 @@ cudaError_t launch_histogram(const int32_t* ids, int64_t n, int32_t V, uint32_t*
     if (H > 65535) H = 65535;                          // slots are 16-bit in the main pass's lookup
     uint32_t* sample = reinterpret_cast<uint32_t*>(scratch + p.off_sample);
     uint2* table = reinterpret_cast<uint2*>(scratch + p.off_table);
-    e = cudaMemsetAsync(sample, 0, (size_t)V * 4, s);
+    e = cudaMemsetAsync(scratch, 0, p.clear_bytes, s);
     if (e != cudaSuccess) return e;
-    static int done_pick[kMaxDevices] = {0}, done_hot[kMaxDevices] = {0};
+    static int done_pick[kMaxDevices] = {0}, done_hot[kMaxDevices] = {0}, done_packed[kMaxDevices] = {0};
     e = set_smem_once(reinterpret_cast<const void*>(k_hist_pick), kMaxTableBytes, done_pick);
     if (e != cudaSuccess) return e;
     e = set_smem_once(reinterpret_cast<const void*>(k_hist_hot), kDynSmem, done_hot);
     if (e != cudaSuccess) return e;
     // a refused launch must stop the chain: the main pass would count through an unwritten table
-    k_hist_sample<<<grid, kThreads, 0, s>>>(ids, n, V, sample);
+    const uint32_t* gate = nullptr;
+    if (packed_path) {
+        // all bins in shared memory, packed; the three kernels after it return at once unless a field wrapped
+        e = set_smem_once(reinterpret_cast<const void*>(k_hist_packed), kDynSmem, done_packed);
+        if (e != cudaSuccess) return e;
+        const uint32_t W = ((uint32_t)V + 2) / 3;
+        uint32_t* packed = reinterpret_cast<uint32_t*>(scratch + p.off_packed);
+        uint32_t* g = reinterpret_cast<uint32_t*>(scratch + p.off_gate);
+        k_hist_packed<<<grid, kThreads, (size_t)W * 4, s>>>(ids, n, V, W, packed, g);
+        count_launch();
+        if ((e = cudaGetLastError()) != cudaSuccess) return e;
+        k_hist_settle<<<grid, kThreads, 0, s>>>(ids, n, V, packed, counts, accumulate, sample, g, ctrl);
+        gate = g;
+    } else {
+        k_hist_sample<<<grid, kThreads, 0, s>>>(ids, n, V, sample);
+    }
     count_launch();
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
-    k_hist_pick<<<1, kThreads, T32 * 8, s>>>(sample, V, H, table);
+    k_hist_pick<<<1, kThreads, T32 * 8, s>>>(sample, V, H, table, gate);
     count_launch();
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
-    k_hist_hot<<<grid, kThreads, kDynSmem, s>>>(ids, n, V, counts, table, H, ctrl);
+    k_hist_hot<<<grid, kThreads, kDynSmem, s>>>(ids, n, V, counts, table, H, ctrl, gate);
     count_launch();
     return cudaGetLastError();
 }
