@@ -384,49 +384,141 @@ k_hist_hot(const int32_t* __restrict__ ids, int64_t n, int32_t V, uint32_t* __re
 }
 
 // ---- every bin in shared memory, three 10-bit fields to a word -----------------------------------------
-// Word w holds the counters of ids w, W + w and 2W + w (W = ceil(V / 3)).  Each token is one returning
-// shared-memory add of 1 << (10 * field); the thread looks at the field's old value before it touches the
-// next token.  The add that takes a field from kSpill-1 to kSpill subtracts kSpill again and credits them
-// to out[id] in global memory, so a field holds fewer than kSpill counts plus whatever other threads add
-// between those two operations: at most one add per other thread of the CTA is in flight at any time,
-// which keeps a field under 2 * kSpill as long as no single token makes up half of the stream.  An add that
-// finds kFieldMax in its field has carried into the neighbour: it raises the gate, and the launcher's
-// next kernels throw this count away and count the stream again with the hot / cold kernels.
+// Word w holds the counters of ids w, W + w and 2W + w (W >= ceil(V / 3)).  Each token is one returning
+// shared-memory add of 1 << (10 * field).  The add that takes a field from kSpill-1 to kSpill subtracts
+// kSpill again and credits them to out[id] in global memory, so a field holds fewer than kSpill counts plus
+// whatever other threads add between those two operations.  With four adds in flight per thread that keeps
+// a field from wrapping as long as no token makes up an eighth of the stream, so the most frequent token is
+// taken out of the fields: the first id of a CTA that hands counts on becomes its hot id (the most frequent
+// token gets to kSpill first), and from then on a lane that meets it adds 1 to a 32-bit word of its own
+// instead (one per lane, so those adds never collide).  Until the hot id is known (kCarefulTrips trips)
+// every add is tested before the thread's next one is issued.  An add that finds kFieldMax in its field has
+// carried into the neighbour: it raises the gate, and the launcher's next kernels throw this count away
+// and count the stream again with the hot / cold kernels.
 constexpr uint32_t kFieldBits = 10, kFieldMax = (1u << kFieldBits) - 1, kSpill = 512;
+constexpr uint32_t kNoId = 0xffffffffu;        // no token id: ids are tallied only when < V <= 2^31
+constexpr int kCarefulTrips = 2;               // trips a CTA counts one add at a time, until its hot id is known
 constexpr int kGateWords = 4;                  // {recount, unused, skipped ids (64 bits)}
 
+// Words per CTA for V bins, 0 when they do not fit: the smallest W >= ceil(V / 3) for which
+// field = (id * M) >> 32 with M = 2^32 / W + 1 is exact for every id < 3W (the quotient steps at W and 2W:
+// it is monotone, so the four ids around the steps decide).
+static uint32_t packed_words(int32_t V, uint32_t* magic) {
+    for (uint64_t W = ((uint64_t)V + 2) / 3; W >= 2 && W * 4 <= kDynSmem; ++W) {
+        const uint64_t M = (1ull << 32) / W + 1;
+        if (M >> 32) continue;
+        if ((((W - 1) * M) >> 32) == 0 && ((W * M) >> 32) == 1 && (((2 * W - 1) * M) >> 32) == 1 &&
+            (((2 * W) * M) >> 32) == 2 && (((3 * W - 1) * M) >> 32) == 2) {
+            if (magic) *magic = (uint32_t)M;
+            return (uint32_t)W;
+        }
+    }
+    return 0;
+}
+
 __global__ void __launch_bounds__(kThreads, 1)
-k_hist_packed(const int32_t* __restrict__ ids, int64_t n, int32_t V, uint32_t W, uint32_t* __restrict__ out,
-              uint32_t* __restrict__ gate) {
+k_hist_packed(const int32_t* __restrict__ ids, int64_t n, int32_t V, uint32_t W, uint32_t M,
+              uint32_t* __restrict__ out, uint32_t* __restrict__ gate) {
     extern __shared__ __align__(16) uint32_t s_fields[];
+    __shared__ uint32_t s_hot;
+    __shared__ uint32_t s_own[32];                           // the hot id's counts, one word per lane
     for (uint32_t i = threadIdx.x; i < W; i += kThreads) s_fields[i] = 0;
+    if (threadIdx.x == 0) s_hot = kNoId;
+    if (threadIdx.x < 32) s_own[threadIdx.x] = 0;
     __syncthreads();
     unsigned long long bad = 0;
-    uint32_t wrapped = 0;
-    const uint32_t W2 = 2 * W;
-    auto tally_in_range = [&](uint32_t id) {
-        const uint32_t f = (id >= W) + (id >= W2);
-        const uint32_t w = id - f * W, sh = f * kFieldBits;
-        const uint32_t fld = (atomicAdd(&s_fields[w], 1u << sh) >> sh) & kFieldMax;
-        if ((fld & (kSpill - 1)) == kSpill - 1) {           // kSpill-1 or kFieldMax: one add in kSpill gets here
-            if (fld == kFieldMax) {
-                wrapped = 1;
-            } else {
-                atomicSub(&s_fields[w], kSpill << sh);
-                atomicAdd(&out[id], kSpill);
-            }
+    uint32_t wrapped = 0, hot = kNoId;
+    const uint32_t base = (uint32_t)__cvta_generic_to_shared(s_fields);
+    const uint32_t own = (uint32_t)__cvta_generic_to_shared(&s_own[threadIdx.x & 31]);
+    const uint32_t neg_w = 0u - W;
+    // One token with id < V: the add, and what its test needs.  `low` is the field's low nine bits in place;
+    // for the hot id it is bit 31 of the lane's own word, which is never set, so the test never fires there.
+    auto add_one = [&](uint32_t id, uint32_t& a, uint32_t& inc, uint32_t& low) -> uint32_t {
+        uint32_t old;
+        asm volatile("{\n\t"
+            ".reg .pred ph;\n\t"
+            ".reg .b32 f, w, sh;\n\t"
+            "mul.hi.u32 f, %4, %5;\n\t"
+            "mad.lo.u32 w, f, %6, %4;\n\t"
+            "mul.lo.u32 sh, f, 10;\n\t"
+            "shl.b32 %2, 1, sh;\n\t"
+            "shl.b32 %3, 511, sh;\n\t"
+            "mad.lo.u32 %1, w, 4, %7;\n\t"
+            "setp.eq.u32 ph, %4, %8;\n\t"
+            "selp.u32 %1, %9, %1, ph;\n\t"
+            "selp.u32 %2, 1, %2, ph;\n\t"
+            "selp.u32 %3, 0x80000000, %3, ph;\n\t"
+            "atom.shared.add.u32 %0, [%1], %2;\n\t"
+            "}" : "=&r"(old), "=&r"(a), "=&r"(inc), "=&r"(low)
+                : "r"(id), "r"(M), "r"(neg_w), "r"(base), "r"(hot), "r"(own) : "memory");
+        return old;
+    };
+    static_assert(kFieldBits == 10 && kSpill == 512, "written into the instructions above");
+    // The add found the low nine bits of its field set: kSpill-1 (hand kSpill counts on) or kFieldMax (wrapped).
+    auto settle_field = [&](uint32_t id, uint32_t a, uint32_t inc, uint32_t old) {
+        if ((old & (inc * kFieldMax)) == inc * kFieldMax) {
+            wrapped = 1;
+        } else {
+            atomicSub(&s_fields[(a - base) >> 2], inc * kSpill);
+            atomicAdd(&out[id], kSpill);
+            if (*reinterpret_cast<volatile uint32_t*>(&s_hot) == kNoId) atomicCAS(&s_hot, kNoId, id);
         }
+    };
+    auto tally_in_range = [&](uint32_t id) {
+        uint32_t a, inc, low;
+        const uint32_t old = add_one(id, a, inc, low);
+        if ((~old & low) == 0) settle_field(id, a, inc, old);
     };
     auto tally1 = [&](uint32_t id) {
         if (id < (uint32_t)V) tally_in_range(id); else ++bad;
     };
-    stream_ids4(ids, n, [&](uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
-        if (max(max(a, b), max(c, d)) < (uint32_t)V) {       // one range test per 128-bit load
-            tally_in_range(a); tally_in_range(b); tally_in_range(c); tally_in_range(d);
+    // Four tokens of one 128-bit load: four adds in flight, their tests folded into one branch (taken once
+    // in about kSpill / 4 loads).
+    auto tally4 = [&](uint4 x) {
+        if (max(max(x.x, x.y), max(x.z, x.w)) < (uint32_t)V) {       // one range test per 128-bit load
+            uint32_t aa, ab, ac, ad, ia, ib, ic, id, la, lb, lc, ld;
+            const uint32_t oa = add_one(x.x, aa, ia, la);
+            const uint32_t ob = add_one(x.y, ab, ib, lb);
+            const uint32_t oc = add_one(x.z, ac, ic, lc);
+            const uint32_t od = add_one(x.w, ad, id, ld);
+            const uint32_t za = ~oa & la, zb = ~ob & lb, zc = ~oc & lc, zd = ~od & ld;
+            if (min(min(za, zb), min(zc, zd)) == 0) {
+                if (za == 0) settle_field(x.x, aa, ia, oa);
+                if (zb == 0) settle_field(x.y, ab, ib, ob);
+                if (zc == 0) settle_field(x.z, ac, ic, oc);
+                if (zd == 0) settle_field(x.w, ad, id, od);
+            }
         } else {
-            tally1(a); tally1(b); tally1(c); tally1(d);
+            tally1(x.x); tally1(x.y); tally1(x.z); tally1(x.w);
         }
-    }, tally1);
+    };
+    // the same, each add tested before the next is issued (one add in flight per thread)
+    auto tally4_in_turn = [&](uint4 x) { tally1(x.x); tally1(x.y); tally1(x.z); tally1(x.w); };
+    // The walk over the CTA's share of the 16-byte-aligned body: whole trips of four rows (kThreads 128-bit
+    // loads each) without a bounds test, then one guarded trip; CTA 0 takes the ragged ends.
+    const uintptr_t addr = reinterpret_cast<uintptr_t>(ids);
+    int64_t head = ((16 - (addr & 15)) & 15) >> 2;
+    if (head > n) head = n;
+    const int64_t nvec = (n - head) >> 2;
+    const int64_t tail0 = head + nvec * 4;
+    if (blockIdx.x == 0) {
+        if ((int64_t)threadIdx.x < head) tally1((uint32_t)ids[threadIdx.x]);
+        const int64_t t = tail0 + threadIdx.x;
+        if (t < n) tally1((uint32_t)ids[t]);
+    }
+    const uint4* vec = reinterpret_cast<const uint4*>(ids + head);
+    const int64_t v0 = nvec * blockIdx.x / gridDim.x;
+    const int64_t v1 = nvec * (blockIdx.x + 1) / gridDim.x;
+    const int64_t trips = (v1 - v0) / (4 * kThreads);
+    const uint4* p = vec + v0 + threadIdx.x;
+    for (int64_t t = 0; t < trips; ++t, p += 4 * kThreads) {
+        const uint4 a = ld_stream_u4(p), b = ld_stream_u4(p + kThreads), c = ld_stream_u4(p + 2 * kThreads),
+                    d = ld_stream_u4(p + 3 * kThreads);
+        if (hot == kNoId) hot = *reinterpret_cast<volatile uint32_t*>(&s_hot);   // once set it stays
+        if (t < kCarefulTrips) { tally4_in_turn(a); tally4_in_turn(b); tally4_in_turn(c); tally4_in_turn(d); }
+        else { tally4(a); tally4(b); tally4(c); tally4(d); }
+    }
+    for (int64_t v = v0 + trips * (4 * kThreads) + threadIdx.x; v < v1; v += kThreads) tally4_in_turn(ld_stream_u4(vec + v));
     __syncthreads();
     for (uint32_t i = threadIdx.x; i < W; i += kThreads) {
         const uint32_t w = (i + blockIdx.x * 61u) % W;       // de-phase the CTAs' flushes
@@ -436,6 +528,11 @@ k_hist_packed(const int32_t* __restrict__ ids, int64_t n, int32_t V, uint32_t W,
             const uint32_t c = (x >> (f * kFieldBits)) & kFieldMax, id = f * W + w;
             if (c && id < (uint32_t)V) atomicAdd(&out[id], c);
         }
+    }
+    if (threadIdx.x < 32) {                                  // (only lanes that had read s_hot added to s_own)
+        uint32_t c = s_own[threadIdx.x];
+        for (int o = 16; o; o >>= 1) c += __shfl_xor_sync(0xffffffffu, c, o);
+        if (threadIdx.x == 0 && c) atomicAdd(&out[s_hot], c);
     }
     if (wrapped) atomicOr(&gate[0], 1u);
     for (int o = 16; o; o >>= 1) bad += __shfl_xor_sync(0xffffffffu, bad, o);
@@ -528,7 +625,7 @@ bool hist_supported(int32_t V) {
     return ((size_t)V + 31) / 32 * 8 <= kMaxTableBytes;
 }
 
-static bool packed_fits(int32_t V) { return ((size_t)V + 2) / 3 * 4 <= kDynSmem; }
+static bool packed_fits(int32_t V) { return packed_words(V, nullptr) != 0; }
 
 HistPlan hist_plan(int32_t V) {
     HistPlan p{};
@@ -587,10 +684,11 @@ cudaError_t launch_histogram(const int32_t* ids, int64_t n, int32_t V, uint32_t*
         // all bins in shared memory, packed; the three kernels after it return at once unless a field wrapped
         e = set_smem_once(reinterpret_cast<const void*>(k_hist_packed), kDynSmem, done_packed);
         if (e != cudaSuccess) return e;
-        const uint32_t W = ((uint32_t)V + 2) / 3;
+        uint32_t M = 0;
+        const uint32_t W = packed_words(V, &M);
         uint32_t* packed = reinterpret_cast<uint32_t*>(scratch + p.off_packed);
         uint32_t* g = reinterpret_cast<uint32_t*>(scratch + p.off_gate);
-        k_hist_packed<<<grid, kThreads, (size_t)W * 4, s>>>(ids, n, V, W, packed, g);
+        k_hist_packed<<<grid, kThreads, (size_t)W * 4, s>>>(ids, n, V, W, M, packed, g);
         count_launch();
         if ((e = cudaGetLastError()) != cudaSuccess) return e;
         k_hist_settle<<<grid, kThreads, 0, s>>>(ids, n, V, packed, counts, accumulate, sample, g, ctrl);

@@ -88,6 +88,45 @@ def test_histogram_degenerate_streams():
     assert np.array_equal(_u32(vt.vt_histogram(ramp, V, ws=ws)), ref)
 
 
+@pytest.mark.parametrize("V", [57_345, 100_003, 128256, 151_936, 172_032, 172_033])
+def test_histogram_every_vocabulary_size_around_the_packed_layout(V):
+    """Sizes on both sides of what three bins per shared-memory word can hold, with ids on the field borders."""
+    n = 3_000_017
+    ids = vt_inputs.zipf_ids(n, V, 1.07, seed=V % 1000, noise_frac=0.05, device=DEV)
+    W = (V + 2) // 3
+    edge = torch.tensor([0, W - 1, W, W + 1, 2 * W - 1, 2 * W, 2 * W + 1, V - 1], dtype=torch.int32, device=DEV).clamp_(0, V - 1)
+    ids[:: 1013] = edge[torch.arange(ids[::1013].numel(), device=DEV) % edge.numel()]
+    ws = vt.Workspace(vt.workspace_bytes(vt.VT_OP_HISTOGRAM, n, V))
+    ref, bad = oracle.histogram(ids.cpu().numpy(), V)
+    assert bad == 0
+    assert np.array_equal(_u32(vt.vt_histogram(ids, V, ws=ws)), ref)
+    _assert_clean(ws)
+
+
+def test_histogram_hot_tokens_that_arrive_late_and_skipped_ids_are_counted_once():
+    """A stream whose first part is flat and whose second part is mostly two tokens, with ids outside
+    [0, V) sprinkled in: whichever kernels end up counting it, every id is counted once and every skipped id
+    is reported once."""
+    V = 128256
+    n = 24_000_000
+    g = torch.Generator(device=DEV).manual_seed(5)
+    ids = torch.randint(0, V, (n,), device=DEV, dtype=torch.int32, generator=g)
+    late = ids[n // 2:]
+    u = torch.rand(late.numel(), device=DEV, generator=g)
+    late[u < 0.45] = 31_337
+    late[(u >= 0.45) & (u < 0.85)] = 90_001
+    ids[5::100_003] = V
+    ids[7::200_003] = -3
+    ws = vt.Workspace(vt.workspace_bytes(vt.VT_OP_HISTOGRAM, n, V))
+    ref, bad = oracle.histogram(ids.cpu().numpy(), V)
+    assert bad > 0
+    for _ in range(2):                                          # the second call starts from a used workspace
+        got = _u32(vt.vt_histogram(ids, V, ws=ws))
+        assert np.array_equal(got, ref)
+        st, flags, n_bad = ws.read_status()
+        assert flags == vt.VT_FLAG_BAD_ID and n_bad == bad
+
+
 def test_histogram_three_ids_carry_the_whole_stream():
     """Streams that drive single bins to 1e7 and more: neighbouring ids, ids around the middle and the
     end of the vocabulary, with a sprinkle of a fourth id."""
