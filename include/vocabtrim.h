@@ -115,10 +115,10 @@ vt_status vt_histogram(const int32_t *ids, int64_t n, int32_t V, uint32_t *count
 /*
  * Measurement aid beside Algorithm 1 (no counterpart in the paper): counts[id mod bins] += 1 for every id
  * inside [0,V), with all `bins` counters (at most VT_FOLDED_MAX_BINS) directly indexed in shared
- * memory -- the same stream walk and the same one shared-memory reduction per token as vt_histogram,
- * without its lookup and without its path for cold ids.  Its rate is what shared-memory atomics can
- * take on a given stream; the benchmark reports it beside vt_histogram's.  counts [bins] uint32 is
- * cleared first; ids outside [0,V) are skipped silently.  Exact.
+ * memory as 32-bit words -- a plain walk over the stream (four 128-bit loads in flight per thread) and one
+ * shared-memory reduction per token.  An independent, simpler kernel over the same stream: the benchmark
+ * reports its rate beside vt_histogram's.  counts [bins] uint32 is cleared first; ids outside [0,V) are
+ * skipped silently.  Exact.
  */
 #define VT_FOLDED_MAX_BINS 57344
 vt_status vt_histogram_folded(const int32_t *ids, int64_t n, int32_t V, int32_t bins, uint32_t *counts,
