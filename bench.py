@@ -565,6 +565,11 @@ STAMP_NAMES = ("entry", "ring_requested", "released", "first_stage_landed", "las
                "after_fence_barrier", "after_ticket", "merge_loads_done", "merge_selection_done", "merge_outputs_written")
 
 
+DENSE_STAMP_NAMES = ("entry", "set_up", "released", "first_stage_landed", "mmas_issued_first_tile", "mmas_issued_last_tile",
+                     "accumulators_complete_first_tile", "accumulators_complete_last_tile", "epilogue_done_first_tile",
+                     "epilogue_done_last_tile", "record_written", "leaving")
+
+
 def stamps_case(vt, vt_build, dev, args):
     """Where a head step's time goes: runs the headline step with the instrumented twin of the library
     (-DVT_STAMPS, built on demand) whose streaming kernel writes a nanosecond stamp per CTA and phase into
@@ -619,6 +624,44 @@ def stamps_case(vt, vt_build, dev, args):
         print(json.dumps(rec), flush=True)
         del wl
         torch.cuda.empty_cache()
+    # the batched head (config 4): its own stamp layout, times after the first CTA's entry
+    d, K, B, topk = DENSE["d"], DENSE["K"], DENSE["B"], DENSE["topk"]
+    wl = build_head_workload(vt, dev, d, K, B, topk, 1.0, True, seed=1004, pool=4)
+    wl["T"] = vt_inputs.temperatures(B, 0.5, 1.5, seed=5001, device=dev)
+    off, slots, ctas = ctypes.c_size_t(0), ctypes.c_int32(0), ctypes.c_int32(0)
+    if L.vt_stamps_region(B, d, topk, ctypes.byref(off), ctypes.byref(slots), ctypes.byref(ctas)):
+        ws = wl["ws"]
+        view = ws.buf[(ws.ptr - ws.buf.data_ptr()) + off.value:][: ctas.value * slots.value * 8].view(torch.int64)
+        first_touch(vt, wl)
+        rec = {"case": "stamps", "workload": "config4", "unit": "us after the first CTA's entry, median over launches of "
+               "[median CTA, first CTA, last CTA]"}
+        for mode, ov in (("overlapped", True), ("plain", False)):
+            rows = []
+            for rep_ in range(max(8, args.steps)):
+                view.zero_()
+                run_head_steps(vt, wl, 4, start=rep_ * 4, overlapped=ov)
+                torch.cuda.synchronize()
+                x = view.cpu().numpy().reshape(ctas.value, slots.value).astype(np.float64)
+                live = x[:, 0] > 0
+                t0 = x[live, 0].min()
+                row = {}
+                for k, nm in enumerate(DENSE_STAMP_NAMES):
+                    col = x[live, k]
+                    col = col[col > 0]
+                    if col.size:
+                        row[nm] = [(float(np.median(col)) - t0) / 1e3, (col.min() - t0) / 1e3, (col.max() - t0) / 1e3]
+                row["merge_started"] = [(x[0, 12] - t0) / 1e3] * 3
+                row["merge_row0_written"] = [(x[0, 13] - t0) / 1e3] * 3
+                rows.append(row)
+            rec[mode] = {k: [round(float(v), 2) for v in np.median(np.array([r[k] for r in rows if k in r]), axis=0)]
+                         for k in rows[0]}
+            e0, e1 = _events()
+            e0.record()
+            run_head_steps(vt, wl, 200, overlapped=ov)
+            e1.record()
+            torch.cuda.synchronize()
+            rec[mode]["us_per_step_with_stamps"] = round(e0.elapsed_time(e1) * 5, 2)
+        print(json.dumps(rec), flush=True)
 
 
 def small_case(vt, dev, args, peak_gbs):

@@ -165,8 +165,10 @@ const char* vt_status_str(vt_status s) {
 
 #ifdef VT_STAMPS
 int32_t vt_stamps_region(int32_t B, int32_t d, int32_t topk, size_t* offset, int32_t* slots, int32_t* max_ctas) {
-    if (!head_skinny_supported(B, d) || !offset || !slots || !max_ctas) return 0;
-    *offset = VT_CTRL_BYTES + head_skinny_stamps_offset(B, topk);
+    if (!offset || !slots || !max_ctas) return 0;
+    if (head_skinny_supported(B, d)) *offset = VT_CTRL_BYTES + head_skinny_stamps_offset(B, topk);
+    else if (head_dense_supported(B, 1, d)) *offset = VT_CTRL_BYTES + head_dense_stamps_offset(B, topk);
+    else return 0;
     *slots = 16;
     *max_ctas = 160;
     return 1;

@@ -97,6 +97,7 @@ size_t head_skinny_scratch_bytes(int32_t B, int32_t K, int32_t topk);
 cudaError_t launch_head_skinny(const HeadArgs& a, Ctrl* ctrl, uint8_t* scratch, cudaStream_t s);
 #ifdef VT_STAMPS
 size_t head_skinny_stamps_offset(int32_t B, int32_t topk);   // offset of the phase stamps in the head scratch
+size_t head_dense_stamps_offset(int32_t B, int32_t topk);    // the same for the batched head
 #endif
 
 bool head_dense_supported(int32_t B, int32_t K, int32_t d);

@@ -17,8 +17,8 @@
 // descriptors and the accumulators in tensor memory: two accumulator stages of up to 256 columns, so
 // the epilogue of tile t overlaps the MMAs of tile t+1.  tcgen05.commit releases ring stages and
 // publishes accumulators (to both CTAs of a pair).  Eight epilogue warps read the accumulators back
-// with tcgen05.ld -- TMEM lane = hidden row; warps 0-3 take the first half of a tile's columns, warps
-// 4-7 the second -- 16 columns at a time: running max / sum-exp of z = logit / T_b, Gumbel-max candidate
+// with tcgen05.ld -- TMEM lane = hidden row; the two warps of a lane quadrant take one half of a tile's
+// columns each -- 16 columns at a time: running max / sum-exp of z = logit / T_b, Gumbel-max candidate
 // from the caller's uniforms, and a sorted top-k list kept in registers.  Logits never go to HBM.  The
 // two column halves of a row are merged through shared memory; per CTA (pair) and hidden row one
 // record goes to scratch; a second small kernel (one warp per hidden row) merges the records,
@@ -40,13 +40,26 @@ constexpr int kMaxBN = 256;               // vocabulary rows per tile at most (T
 constexpr int kBK = 64;                   // columns of d per ring stage: 128 bytes, one swizzle row
 constexpr int kMaxStages = 8;
 constexpr int kHTileBytes = kBM * kBK * 2; // 16 KB: the hidden-row operand of a stage
-constexpr int kEpiWarps = 8;
-constexpr int kThreads = (2 + kEpiWarps) * 32;   // TMA producer, MMA issuer, 8 epilogue warps
+constexpr int kParts8 = 2, kParts16 = 2;  // epilogue warps per TMEM lane quadrant for lists of 8 / 16 (3 and 4 were no
+                                          // faster: the epilogue is bound by the instructions it issues, not by latency)
+constexpr int epi_threads(int parts) { return (2 + 4 * parts) * 32; }   // TMA producer, MMA issuer, epilogue warps
 constexpr int kCh = 16;                   // accumulator columns per epilogue step (keeps the row state in registers)
 constexpr int kTmemCols = 512;            // 2 accumulator stages x kMaxBN columns
 constexpr int kMaxTopk = 16;              // top-k list lives in registers
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 constexpr size_t kRingBudget = 225 * 1024;   // ring bytes at most (227 KB per CTA less alignment slack and statics)
+
+// Phase stamps (-DVT_STAMPS builds only): one thread per role writes %globaltimer into a region behind the
+// records; bench.py --case stamps reads them back.  Slots per CTA: 0 entry, 1 set up (barriers, tensor
+// memory), 2 producer released by the launch dependency, 3 first stage landed (MMA issuer), 4 / 5 MMAs of the
+// CTA's first / last tile issued, 6 / 7 accumulators of the first / last tile complete (epilogue warp 0),
+// 8 / 9 first / last tile's epilogue done, 10 record written, 11 leaving; CTA 0 also carries the merge
+// kernel's 12 start (records complete) and 13 end for hidden row 0.
+#ifdef VT_STAMPS
+#define VT_DSTAMP(slot) do { stamps[(size_t)blockIdx.x * kStampSlots + (slot)] = global_ns(); } while (0)
+#else
+#define VT_DSTAMP(slot) do {} while (0)
+#endif
 
 // ---- PTX wrappers ----------------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -223,8 +236,11 @@ __device__ __forceinline__ void list_insert(float (&tv)[KT], int (&tj)[KT], floa
 }
 
 // KT: capacity of the register top-k list (8 or kMaxTopk).  PAIR: two CTAs of a cluster form one MMA.
-template <int KT, bool PAIR>
-__global__ void __launch_bounds__(kThreads, 1)
+// PARTS: epilogue warps per TMEM lane quadrant; each takes a contiguous share of a tile's 16-column chunks.
+// The epilogue is a long chain of dependent arithmetic per column: it runs at the rate the schedulers can
+// interleave warps, so more warps per scheduler shorten it almost in proportion.
+template <int KT, bool PAIR, int PARTS>
+__global__ void __launch_bounds__(epi_threads(PARTS), 1)
 k_head_dense(const HeadArgs a, Ctrl* ctrl, float* __restrict__ recs, const DenseGeo geo,
              const __grid_constant__ CUtensorMap tm_h, const __grid_constant__ CUtensorMap tm_w) {
     extern __shared__ uint8_t s_dyn[];
@@ -232,6 +248,11 @@ k_head_dense(const HeadArgs a, Ctrl* ctrl, float* __restrict__ recs, const Dense
     __shared__ uint32_t s_tmem_base;
     __shared__ int s_abort;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#ifdef VT_STAMPS
+    unsigned long long* stamps = reinterpret_cast<unsigned long long*>(
+        reinterpret_cast<uint8_t*>(recs) + align_up_dev((size_t)kMaxGrid * a.B * rec_fields(a.topk) * 4, 256));
+    if (threadIdx.x == 0) VT_DSTAMP(0);
+#endif
     // identical in both CTAs of a pair: the MMA addresses the peer's operands by the leader's offsets
     uint8_t* ring = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(s_dyn) + 1023) & ~(uintptr_t)1023);
     const uint32_t ring_u32 = smem_u32(ring);
@@ -243,7 +264,7 @@ k_head_dense(const HeadArgs a, Ctrl* ctrl, float* __restrict__ recs, const Dense
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kMaxStages; ++s) { mbar_init(&s_full[s], 1); mbar_init(&s_empty[s], 1); }
-        for (int p = 0; p < 2; ++p) { mbar_init(&s_acc_full[p], 1); mbar_init(&s_acc_empty[p], (PAIR ? 2 : 1) * kEpiWarps); }
+        for (int p = 0; p < 2; ++p) { mbar_init(&s_acc_full[p], 1); mbar_init(&s_acc_empty[p], (PAIR ? 2 : 1) * 4 * PARTS); }
         s_abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -264,6 +285,9 @@ k_head_dense(const HeadArgs a, Ctrl* ctrl, float* __restrict__ recs, const Dense
     const uint32_t tmem_base = s_tmem_base;
     volatile int* abort_flag = &s_abort;
     griddep_launch_dependents();                                  // the merge kernel may take its seats
+#ifdef VT_STAMPS
+    if (threadIdx.x == 0) VT_DSTAMP(1);
+#endif
 
     if (warp == 0) {
         // ================= TMA producer (both CTAs of a pair) ==========================================
@@ -293,6 +317,7 @@ k_head_dense(const HeadArgs a, Ctrl* ctrl, float* __restrict__ recs, const Dense
                 load_w(g);
             }
             griddep_wait();
+            VT_DSTAMP(2);
             for (int g = 0; g < pre; ++g) load_h(g);
             int done = pre;
             for (int g = pre; g < total; ++g, ++done) {
@@ -329,6 +354,9 @@ k_head_dense(const HeadArgs a, Ctrl* ctrl, float* __restrict__ recs, const Dense
                 const uint32_t d_tmem = tmem_base + (uint32_t)(as * kMaxBN);
                 for (int kc = 0; kc < geo.n_kc; ++kc) {
                     if (!mbar_wait(&s_full[s], ph, abort_flag)) { alive = false; break; }
+#ifdef VT_STAMPS
+                    if (t_local == 0 && kc == 0) VT_DSTAMP(3);
+#endif
                     tc_fence_after();
                     const uint32_t base = ring_u32 + (uint32_t)s * (uint32_t)geo.stage_bytes;
 #pragma unroll
@@ -343,6 +371,10 @@ k_head_dense(const HeadArgs a, Ctrl* ctrl, float* __restrict__ recs, const Dense
                 }
                 if (alive) {                                      // accumulators of this tile are complete
                     if (PAIR) tc_commit_pair(&s_acc_full[as]); else tc_commit(&s_acc_full[as]);
+#ifdef VT_STAMPS
+                    if (t_local == 0) VT_DSTAMP(4);
+                    VT_DSTAMP(5);
+#endif
                 }
             }
             // the last accumulators have been read (every arrival of the peer has landed) before leaving
@@ -350,11 +382,12 @@ k_head_dense(const HeadArgs a, Ctrl* ctrl, float* __restrict__ recs, const Dense
                 if (!mbar_wait(&s_acc_empty[t & 1], (uint32_t)((t >> 1) & 1), abort_flag)) break;
         }
     } else {
-        // ================= epilogue warps: one hidden row and one half of the tile's columns per thread =
+        // ================= epilogue warps: one hidden row and one share of the tile's columns per thread =
         const int ew = warp - 2;
         const int quad = warp & 3;                            // TMEM lanes this warp may read
-        const int half = ew >> 2;                             // which half of the tile's columns
-        const int cols_half = bn / 2, n_ch = cols_half / kCh;
+        const int part = ew >> 2;                             // which share of the tile's chunks
+        const int n_ch_tile = bn / kCh;
+        const int ch_lo = part * n_ch_tile / PARTS, ch_hi = (part + 1) * n_ch_tile / PARTS;
         const int b = (int)rank * kBM + quad * 32 + lane;
         const bool row_live = b < B;
         griddep_wait();                                       // temp, uniforms and the record scratch belong to earlier work until here
@@ -378,10 +411,13 @@ k_head_dense(const HeadArgs a, Ctrl* ctrl, float* __restrict__ recs, const Dense
         for (int tile = group; tile < geo.n_tiles; tile += geo.n_groups, ++t_local) {
             const int as = t_local & 1;
             if (!mbar_wait_warp(&s_acc_full[as], (uint32_t)((t_local >> 1) & 1), abort_flag)) break;
+#ifdef VT_STAMPS
+            if (warp == 2 && lane == 0) { if (t_local == 0) VT_DSTAMP(6); VT_DSTAMP(7); }
+#endif
             tc_fence_after();
-            const int jt = tile * bn + half * cols_half;      // first vocabulary row of this thread's columns
+            const int jt = tile * bn;                         // first vocabulary row of the tile
 #pragma unroll 1
-            for (int ch = 0; ch < n_ch; ++ch) {
+            for (int ch = ch_lo; ch < ch_hi; ++ch) {
                 const int j0 = jt + ch * kCh;
                 // this chunk's uniforms are requested first (they are needed last), and a later
                 // chunk's line is pulled into L2 meanwhile
@@ -398,11 +434,11 @@ k_head_dense(const HeadArgs a, Ctrl* ctrl, float* __restrict__ recs, const Dense
                         for (int i = 0; i < kCh; ++i) u[i] = (j0 + i < K) ? __ldg(up + i) : 0.5f;
                     }
                 }
-                const int jn = (ch + 2 < n_ch) ? j0 + 2 * kCh : jt + geo.n_groups * bn;
+                const int jn = (ch + 2 < ch_hi) ? j0 + 2 * kCh : jt + geo.n_groups * bn + ch_lo * kCh;
                 if (use_u && jn < K && (ch & 1) == 0)
                     asm volatile("prefetch.global.L2 [%0];" ::"l"(a.uniforms + (size_t)b * K + jn));
                 uint32_t r[kCh];
-                tc_ld16(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(as * kMaxBN + half * cols_half + ch * kCh), r);
+                tc_ld16(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(as * kMaxBN + ch * kCh), r);
                 // Warp-uniform from here on (j0 and K are): rows that do not exist simply carry nv = 0,
                 // i.e. columns of -inf, so the warp votes below always see all 32 lanes.
                 if (j0 < K) {
@@ -451,30 +487,27 @@ k_head_dense(const HeadArgs a, Ctrl* ctrl, float* __restrict__ recs, const Dense
                     // chunk's other candidates: it competes as -inf
 #pragma unroll
                     for (int i = 0; i < kCh; ++i) z[i] = (z[i] == z[i]) ? z[i] : -CUDART_INF_F;
-                    float mx = z[0];
-                    int mi = 0;
+                    // candidates: the columns that beat the list's last entry as it stands; they go in by
+                    // ascending column (equal values keep the lower column ahead), one per trip of a warp-
+                    // uniform loop that runs while any row still has one.  A candidate that has fallen under
+                    // the entry that moved up meanwhile simply finds no slot.
+                    uint32_t cand = 0;
 #pragma unroll
-                    for (int i = 1; i < kCh; ++i) {
-                        const bool gt = z[i] > mx;                    // strict: ties keep the lower column
-                        mx = gt ? z[i] : mx;
-                        mi = gt ? i : mi;
-                    }
-                    while (__any_sync(0xffffffffu, mx > thr)) {
-                        const bool take = mx > thr;
-                        list_insert<KT>(st.tv, st.tj, take ? mx : -CUDART_INF_F, j0 + mi);
+                    for (int i = 0; i < kCh; ++i) cand |= (z[i] > thr) ? (1u << i) : 0u;
+                    while (__any_sync(0xffffffffu, cand != 0)) {
+                        const bool take = cand != 0;
+                        const int i = take ? __ffs(cand) - 1 : 0;
+                        float q8[8], q4[4], q2[2];
+#pragma unroll
+                        for (int k = 0; k < 8; ++k) q8[k] = (i & 1) ? z[2 * k + 1] : z[2 * k];
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) q4[k] = (i & 2) ? q8[2 * k + 1] : q8[2 * k];
+#pragma unroll
+                        for (int k = 0; k < 2; ++k) q2[k] = (i & 4) ? q4[2 * k + 1] : q4[2 * k];
+                        const float v = (i & 8) ? q2[1] : q2[0];
+                        list_insert<KT>(st.tv, st.tj, take ? v : -CUDART_INF_F, j0 + i);
                         thr = st.tj[KT - 1] >= 0 ? st.tv[KT - 1] : -CUDART_INF_F;   // a threshold only once the list is full
-                        // drop the extracted element, find the next maximum
-                        float nmx = -CUDART_INF_F;
-                        int nmi = 0;
-#pragma unroll
-                        for (int i = 0; i < kCh; ++i) {
-                            z[i] = (take && i == mi) ? -CUDART_INF_F : z[i];
-                            const bool gt = z[i] > nmx;
-                            nmx = gt ? z[i] : nmx;
-                            nmi = gt ? i : nmi;
-                        }
-                        mx = nmx;
-                        mi = nmi;
+                        cand &= cand - 1;
                     }
                 }
             }
@@ -484,40 +517,47 @@ k_head_dense(const HeadArgs a, Ctrl* ctrl, float* __restrict__ recs, const Dense
                 if (PAIR) mbar_arrive_cluster(acc_empty_bar + (uint32_t)(as * sizeof(uint64_t)));
                 else mbar_arrive(&s_acc_empty[as]);
             }
+#ifdef VT_STAMPS
+            if (warp == 2 && lane == 0) { if (t_local == 0) VT_DSTAMP(8); VT_DSTAMP(9); }
+#endif
         }
-        // ---- the two column halves of a row meet in shared memory (the ring is idle by now: the last
+        // ---- the column shares of a row meet in shared memory (the ring is idle by now: the last
         // accumulators were complete, so every MMA has read its operands and every copy has landed) ----
         float* xch = reinterpret_cast<float*>(ring);
+        constexpr int kXchFields = 5 + 2 * KT;
         const int slot = quad * 32 + lane;                    // row within the CTA
         const bool ok = !*abort_flag;
-        if (half == 1 && ok) {
-            float* x = xch + slot;                            // field-major: conflict-free
+        if (part > 0 && ok) {
+            float* x = xch + (size_t)(part - 1) * kXchFields * kBM + slot;     // field-major: conflict-free
             x[0 * kBM] = st.m; x[1 * kBM] = st.s; x[2 * kBM] = st.gb_s; x[3 * kBM] = __int_as_float(st.gb_j); x[4 * kBM] = st.gb_z;
 #pragma unroll
             for (int p = 0; p < KT; ++p) { x[(5 + p) * kBM] = st.tv[p]; x[(5 + KT + p) * kBM] = __int_as_float(st.tj[p]); }
         }
-        asm volatile("bar.sync 1, %0;" ::"n"(kEpiWarps * 32) : "memory");
-        if (half == 0 && ok && row_live) {
-            const float* x = xch + slot;
-            lse_merge(st.m, st.s, x[0 * kBM], x[1 * kBM]);
-            const float os = x[2 * kBM];
-            const int oj = __float_as_int(x[3 * kBM]);
-            if (better(os, oj, st.gb_s, st.gb_j) && oj >= 0) { st.gb_s = os; st.gb_j = oj; st.gb_z = x[4 * kBM]; }
+        asm volatile("bar.sync 1, %0;" ::"n"(4 * PARTS * 32) : "memory");
+        if (part == 0 && ok && row_live) {
+#pragma unroll 1
+            for (int o = 0; o < PARTS - 1; ++o) {
+                const float* x = xch + (size_t)o * kXchFields * kBM + slot;
+                lse_merge(st.m, st.s, x[0 * kBM], x[1 * kBM]);
+                const float os = x[2 * kBM];
+                const int oj = __float_as_int(x[3 * kBM]);
+                if (better(os, oj, st.gb_s, st.gb_j) && oj >= 0) { st.gb_s = os; st.gb_j = oj; st.gb_z = x[4 * kBM]; }
 #pragma unroll
-            for (int p = 0; p < KT; ++p) {
-                // entries of the other half: equal values must still order by index, so compare keys
-                float cv = x[(5 + p) * kBM];
-                int cj = __float_as_int(x[(5 + KT + p) * kBM]);
-                if (p < KT - topk) continue;                  // its sentinels
+                for (int p = 0; p < KT; ++p) {
+                    // entries of the other share: equal values must still order by index, so compare keys
+                    float cv = x[(5 + p) * kBM];
+                    int cj = __float_as_int(x[(5 + KT + p) * kBM]);
+                    if (p < KT - topk) continue;              // its sentinels
 #pragma unroll
-                for (int q = 0; q < KT; ++q) {
-                    const bool sw = key64(cv, cj) > key64(st.tv[q], st.tj[q]) && q >= KT - topk;
-                    const float ov = st.tv[q];
-                    const int oj2 = st.tj[q];
-                    st.tv[q] = sw ? cv : ov;
-                    st.tj[q] = sw ? cj : oj2;
-                    cv = sw ? ov : cv;
-                    cj = sw ? oj2 : cj;
+                    for (int q = 0; q < KT; ++q) {
+                        const bool sw = key64(cv, cj) > key64(st.tv[q], st.tj[q]) && q >= KT - topk;
+                        const float ov = st.tv[q];
+                        const int oj2 = st.tj[q];
+                        st.tv[q] = sw ? cv : ov;
+                        st.tj[q] = sw ? cj : oj2;
+                        cv = sw ? ov : cv;
+                        cj = sw ? oj2 : cj;
+                    }
                 }
             }
             // ---- this CTA's record of hidden row b ---------------------------------------------------------
@@ -533,6 +573,9 @@ k_head_dense(const HeadArgs a, Ctrl* ctrl, float* __restrict__ recs, const Dense
                 if (p >= KT - topk)
                     kp[(size_t)(1 + p - (KT - topk)) * kMaxGrid + c] = st.tj[p] >= 0 ? key64(st.tv[p], st.tj[p]) : 0ull;
         }
+#ifdef VT_STAMPS
+        if (warp == 2 && lane == 0) VT_DSTAMP(10);
+#endif
     }
     tc_fence_before();
     __syncwarp();                                                 // lanes of the single-thread roles rejoin their warps
@@ -543,6 +586,9 @@ k_head_dense(const HeadArgs a, Ctrl* ctrl, float* __restrict__ recs, const Dense
         else asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)kTmemCols) : "memory");
     }
     if (threadIdx.x == 0 && s_abort) atomicOr(&ctrl->flags, (uint32_t)VT_FLAG_TIMEOUT);
+#ifdef VT_STAMPS
+    if (threadIdx.x == 0) VT_DSTAMP(11);
+#endif
 }
 
 // Two warps per hidden row (candidates / statistics): merge the CTA records, remap, write the outputs.
@@ -553,10 +599,18 @@ k_head_merge(const HeadArgs a, Ctrl* ctrl, float* __restrict__ recs, int G) {
     const int b = blockIdx.x;
     griddep_launch_dependents();                                  // the next step may start fetching its weights
     griddep_wait();                                               // the records are complete
+#ifdef VT_STAMPS
+    unsigned long long* stamps = reinterpret_cast<unsigned long long*>(
+        reinterpret_cast<uint8_t*>(recs) + align_up_dev((size_t)kMaxGrid * a.B * rec_fields(a.topk) * 4, 256));
+    if (b == 0 && threadIdx.x == 0) stamps[12] = global_ns();
+#endif
     const float T = a.temp[b];
     const bool row_ok = (T > 0.f) && (T < CUDART_INF_F);
     const MergeOut mo{a.map, a.out_ids, a.out_logprobs, a.dbg_lse, a.topk, a.uniforms != nullptr};
     merge_records(mo, ctrl, recs, b, row_ok, G, s_stage, threadIdx.x < 32 ? kRoleCand : kRoleStats, &s_xch, 1);
+#ifdef VT_STAMPS
+    if (b == 0 && threadIdx.x == 0) stamps[13] = global_ns();
+#endif
 }
 
 // ---- host side ----------------------------------------------------------------------------------------
@@ -611,7 +665,7 @@ DenseGeo make_geo(int32_t K, int32_t d, bool pair, int max_groups) {
     return g;
 }
 
-template <int KT, bool PAIR>
+template <int KT, bool PAIR, int PARTS>
 cudaError_t launch_variant(const HeadArgs& a, Ctrl* ctrl, float* recs, const DenseGeo& geo, const CUtensorMap& tm_h,
                            const CUtensorMap& tm_w, cudaStream_t s) {
     static int attr_done[64] = {0};
@@ -619,14 +673,14 @@ cudaError_t launch_variant(const HeadArgs& a, Ctrl* ctrl, float* recs, const Den
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev < 0 || dev >= 64 || !attr_done[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(k_head_dense<KT, PAIR>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaError_t e = cudaFuncSetAttribute(k_head_dense<KT, PAIR, PARTS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              (int)(kRingBudget + 1024));
         if (e != cudaSuccess) return e;
         if (dev >= 0 && dev < 64) attr_done[dev] = 1;
     }
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3((unsigned)(PAIR ? 2 * geo.n_groups : geo.n_groups));
-    cfg.blockDim = dim3(kThreads);
+    cfg.blockDim = dim3(epi_threads(PARTS));
     cfg.dynamicSmemBytes = smem;
     cfg.stream = s;
     cudaLaunchAttribute at[2];
@@ -638,7 +692,7 @@ cudaError_t launch_variant(const HeadArgs& a, Ctrl* ctrl, float* recs, const Den
     at[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = at;
     cfg.numAttrs = a.overlap ? 2 : 1;
-    return cudaLaunchKernelEx(&cfg, k_head_dense<KT, PAIR>, a, ctrl, recs, geo, tm_h, tm_w);
+    return cudaLaunchKernelEx(&cfg, k_head_dense<KT, PAIR, PARTS>, a, ctrl, recs, geo, tm_h, tm_w);
 }
 
 }  // namespace
@@ -651,8 +705,14 @@ bool head_dense_topk_ok(int32_t topk) { return topk >= 1 && topk <= kMaxTopk; }
 
 size_t head_dense_scratch_bytes(int32_t B, int32_t K, int32_t topk) {
     (void)K;
+    return align_up((size_t)kMaxGrid * B * rec_fields(topk) * 4, 256) + kStampBytes;
+}
+
+#ifdef VT_STAMPS
+size_t head_dense_stamps_offset(int32_t B, int32_t topk) {
     return align_up((size_t)kMaxGrid * B * rec_fields(topk) * 4, 256);
 }
+#endif
 
 cudaError_t launch_head_dense(const HeadArgs& a, Ctrl* ctrl, uint8_t* scratch, cudaStream_t s) {
     if (!head_dense_supported(a.B, a.K, a.d) || !head_dense_topk_ok(a.topk)) return cudaErrorInvalidValue;
@@ -666,10 +726,10 @@ cudaError_t launch_head_dense(const HeadArgs& a, Ctrl* ctrl, uint8_t* scratch, c
         return cudaErrorInvalidValue;
     float* recs = reinterpret_cast<float*>(scratch);
     cudaError_t e;
-    if (a.topk <= 8) e = pair ? launch_variant<8, true>(a, ctrl, recs, geo, tm_h, tm_w, s)
-                              : launch_variant<8, false>(a, ctrl, recs, geo, tm_h, tm_w, s);
-    else e = pair ? launch_variant<kMaxTopk, true>(a, ctrl, recs, geo, tm_h, tm_w, s)
-                  : launch_variant<kMaxTopk, false>(a, ctrl, recs, geo, tm_h, tm_w, s);
+    if (a.topk <= 8) e = pair ? launch_variant<8, true, kParts8>(a, ctrl, recs, geo, tm_h, tm_w, s)
+                              : launch_variant<8, false, kParts8>(a, ctrl, recs, geo, tm_h, tm_w, s);
+    else e = pair ? launch_variant<kMaxTopk, true, kParts16>(a, ctrl, recs, geo, tm_h, tm_w, s)
+                  : launch_variant<kMaxTopk, false, kParts16>(a, ctrl, recs, geo, tm_h, tm_w, s);
     if (e != cudaSuccess) return e;
     // the merge always follows its own producer closely: it takes its seats early and waits on the device
     cudaLaunchConfig_t cfg{};
