@@ -139,8 +139,9 @@ vt_status vt_select_topk(const uint32_t *counts, int32_t V, int32_t K, int32_t *
  *   vt_select_topp    : smallest K whose K most frequent ids hold at least ceil(p * total) of all
  *                       counted tokens, 0 < p <= 1 (evaluated in fp64);
  *   vt_select_minfreq : K = number of ids with count >= min_count.
- * K is clamped to [1, V] and written to the DEVICE int32 *k_out.  map receives the FULL ranking
- * ([V], the first K entries are the trimmed vocabulary), inv_map [V] is -1 for ranks >= K.
+ * K is clamped to [1, V] and written to the DEVICE int32 *k_out.  map [V]: the first K entries are the
+ * trimmed vocabulary in rank order, the entries behind them are not defined (K is not known to the host, so
+ * the array must hold V); inv_map [V] is -1 for ranks >= K.
  * Workspace: vt_workspace_bytes(VT_OP_SELECT_TOPK, 0, V, V, ...).  Integer work: exact and unique.
  */
 vt_status vt_select_topp(const uint32_t *counts, int32_t V, double p, int32_t *map, int32_t *inv_map,

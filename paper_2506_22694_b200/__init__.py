@@ -203,12 +203,12 @@ def _select_cut(counts: torch.Tensor, ws, call, *arg):
 
 
 def vt_select_topp(counts: torch.Tensor, p: float, ws: Workspace | None = None):
-    """Top-P selection (Method section): returns (K device int32 [1], map [V] full ranking, inv_map [V])."""
+    """Top-P selection (Method section): returns (K device int32 [1], map [V] whose first K entries are the trimmed vocabulary, inv_map [V])."""
     return _select_cut(counts, ws, "vt_select_topp", c_double(float(p)))
 
 
 def vt_select_minfreq(counts: torch.Tensor, min_count: int, ws: Workspace | None = None):
-    """Minimum-frequency selection (Method section): returns (K device int32 [1], map [V], inv_map [V])."""
+    """Minimum-frequency selection (Method section): returns (K device int32 [1], map [V] (first K entries), inv_map [V])."""
     return _select_cut(counts, ws, "vt_select_minfreq", c_uint32(int(min_count)))
 
 

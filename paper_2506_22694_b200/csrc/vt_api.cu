@@ -86,12 +86,12 @@ size_t vt_workspace_bytes(int op, int64_t n, int32_t V, int32_t K, int32_t d, in
             return VT_CTRL_BYTES + hist_plan(V).bytes;
         case VT_OP_SELECT_TOPK:
             if (V < 1 || K < 1 || K > V) return 0;
-            return VT_CTRL_BYTES + select_scratch_bytes(V);
+            return VT_CTRL_BYTES + select_cut_scratch_bytes(V);
         case VT_OP_BUILD_VOCAB:
         case VT_OP_BUILD_VOCAB_HOST: {
             if (!hist_shape_ok(V) || n < 0 || K < 1 || K > V) return 0;
             size_t inner = hist_plan(V).bytes;
-            if (select_scratch_bytes(V) > inner) inner = select_scratch_bytes(V);
+            if (select_cut_scratch_bytes(V) > inner) inner = select_cut_scratch_bytes(V);
             size_t total = VT_CTRL_BYTES + align_up((size_t)V * 4, 256) + inner;
             if (op == VT_OP_BUILD_VOCAB_HOST) {
                 const int64_t chunk = n < kHostChunkIds ? (n > 0 ? n : 1) : kHostChunkIds;
@@ -216,9 +216,8 @@ static vt_status select_cut_impl(const uint32_t* counts, int32_t V, int mode, do
     vt_status st = check_ws(ws, ws_bytes, vt_workspace_bytes(VT_OP_SELECT_TOPK, 0, V, V, 0, 0, 0));
     if (st != VT_OK) return st;
     uint8_t* base = static_cast<uint8_t*>(ws);
-    cudaError_t e = launch_select_topk(counts, V, V, map, inv_map, base + VT_CTRL_BYTES, as_stream(stream));
-    if (e != cudaSuccess) return from_cuda(e);
-    return from_cuda(launch_select_cut(counts, V, mode, p, min_count, map, inv_map, k_out, as_stream(stream)));
+    return from_cuda(launch_select_cut(counts, V, mode, p, min_count, map, inv_map, k_out, base + VT_CTRL_BYTES,
+                                       as_stream(stream)));
 }
 
 vt_status vt_select_topp(const uint32_t* counts, int32_t V, double p, int32_t* map, int32_t* inv_map,

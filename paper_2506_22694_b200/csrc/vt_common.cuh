@@ -50,8 +50,9 @@ size_t select_scratch_bytes(int32_t V);
 cudaError_t launch_select_topk(const uint32_t* counts, int32_t V, int32_t K, int32_t* map,
                                int32_t* inv_map, uint8_t* scratch, cudaStream_t s);
 
+size_t select_cut_scratch_bytes(int32_t V);
 cudaError_t launch_select_cut(const uint32_t* counts, int32_t V, int mode, double pfrac, uint32_t min_count,
-                              const int32_t* map, int32_t* inv_map, int32_t* k_out, cudaStream_t s);
+                              int32_t* map, int32_t* inv_map, int32_t* k_out, uint8_t* scratch, cudaStream_t s);
 
 cudaError_t launch_verify_greedy(const int32_t* token, const int32_t* parent, const int32_t* target, int32_t S,
                                  int32_t N, int32_t* n_accept, int32_t* path, int32_t* emitted,

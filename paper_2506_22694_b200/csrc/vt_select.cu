@@ -30,13 +30,28 @@ constexpr int kSortCap = 16384;                  // 64-bit keys one CTA ranks in
 constexpr int kCountCap = 2048;                  // largest bucket ranked by counting its greater keys
 constexpr uint32_t kWorkCap = 6u << 10;          // key comparisons one CTA spends on that at most, in units of 1024 (~6 K per thread)
 constexpr size_t kSelectSmem = sizeof(uint32_t) * 4 * kFine + sizeof(unsigned long long) * kSortCap;
+constexpr size_t kSelectCutSmem = kSelectSmem + sizeof(uint32_t) * 2 * kFine;   // + the buckets' token mass in two 16-bit halves
+constexpr int kKeysPerThread = kSortCap / kThreads;   // keys of a CTA's run per thread at most
 static_assert(sizeof(uint32_t) * 4 * kFine >= sizeof(uint32_t) * kWarps * kDigits, "the full ranking reuses the bucket arrays");
 
+// What the full ranking needs to find K itself (Top-P / minimum frequency): the cut bucket's ranks
+// [first, end) from the bucket pass and what lies before them.
+struct CutSpec {
+    int mode;                        // 1: Top-P, 2: minimum frequency
+    int valid;                       // 0: no cut bucket (no tokens counted, or nothing as frequent as asked): K = 1
+    uint32_t first, end;             // ranks of the cut bucket
+    unsigned long long mass_before;  // tokens held by the ranks before it
+    double target;                   // ceil(p * total)
+    uint32_t min_count;
+    int32_t* k_out;
+};
+
 // ---- full ranking: least-significant-digit radix sort over the whole cluster -------------------------
-// s_wcnt: [kWarps][kDigits] words of shared memory.
+// s_wcnt: [kWarps][kDigits] words of shared memory.  With `spec`, K is read off the sorted counts before the
+// ranking is emitted (every CTA works it out for itself: the same reads, the same answer).
 __device__ void lsd_rank_all(cg::cluster_group& cluster, const uint32_t* counts, int32_t V, int32_t K, int32_t* map,
                              int32_t* inv_map, uint32_t* keyA, uint32_t* valA, uint32_t* keyB, uint32_t* valB,
-                             uint32_t (*s_wcnt)[kDigits]) {
+                             uint32_t (*s_wcnt)[kDigits], const CutSpec* spec = nullptr) {
     const unsigned rank = cluster.block_rank();
     __shared__ uint32_t s_tot[kDigits];            // this CTA's digit totals (read by the peers)
     __shared__ uint32_t s_base[kDigits];           // global start of (digit, this CTA)
@@ -138,6 +153,46 @@ __device__ void lsd_rank_all(cg::cluster_group& cluster, const uint32_t* counts,
             dst_val = (dst_val == valA) ? valB : valA;
         }
     }
+    if (spec) {
+        __shared__ int s_kfound;
+        if (threadIdx.x == 0) s_kfound = 1;
+        __syncthreads();
+        if (spec->valid && warp == 0) {
+            // the sorted counts of the cut bucket's ranks, 32 at a time, until the prefix reaches the target
+            // (Top-P) or the counts fall under min_count; equal counts (every bucket under 256) by division
+            const uint32_t a = spec->first, b = spec->end;
+            const uint32_t c0 = src_key[a];
+            int found = (int)b;                                        // (the bucket pass says the cut lies in [a, b])
+            if (spec->mode == 1 && c0 < 256u) {
+                const unsigned long long rem = (unsigned long long)spec->target - spec->mass_before;
+                found = (int)(a + (uint32_t)((rem + c0 - 1) / c0));
+            } else {
+                unsigned long long cum = spec->mass_before;
+                bool done = false;
+                for (uint32_t j0 = a; j0 < b && !done; j0 += 32) {
+                    const uint32_t j = j0 + lane;
+                    const uint32_t c = j < b ? src_key[j] : 0u;
+                    if (spec->mode == 1) {
+                        unsigned long long incl = c;
+                        for (int o = 1; o < 32; o <<= 1) {
+                            const unsigned long long y = __shfl_up_sync(0xffffffffu, incl, o);
+                            if (lane >= o) incl += y;
+                        }
+                        const unsigned hit = __ballot_sync(0xffffffffu, j < b && (double)(cum + incl) >= spec->target);
+                        if (hit) { found = (int)(j0 + __ffs(hit)); done = true; }
+                        cum += __shfl_sync(0xffffffffu, incl, 31);
+                    } else {
+                        const unsigned low = __ballot_sync(0xffffffffu, j >= b || c < spec->min_count);
+                        if (low) { found = (int)(j0 + __ffs(low) - 1); done = true; }
+                    }
+                }
+            }
+            if (lane == 0) s_kfound = max(1, min(V, found));
+        }
+        __syncthreads();
+        K = s_kfound;
+        if (rank == 0 && threadIdx.x == 0) *spec->k_out = K;
+    }
     // emit: sorted position j holds id v
     for (int j = rank * kThreads + threadIdx.x; j < V; j += kCluster * kThreads) {
         const int32_t v = src_val ? (int32_t)src_val[j] : j;
@@ -164,9 +219,19 @@ __device__ __forceinline__ uint32_t fine_bucket(uint32_t c) {
 // the cut is never touched again.  When a run does not fit a CTA's shared memory (K close to V) or a
 // bucket is too large to rank by counting (counts that all fall into one bucket), the full ranking
 // above takes over.
+//
+// MODE 1 / 2 (the Method section's Top-P and minimum-frequency rules): K is not given but found on the way.
+// The bucket pass also sums the token mass of every bucket (Top-P), the cut bucket is the one in which the
+// prefix mass reaches ceil(p * total) / the one min_count falls into, everything down to the end of that
+// bucket is ranked as above, and the CTA that ranks the cut bucket reads K off the ranks (the key whose
+// prefix mass crosses the target / the number of keys with count >= min_count) before anything is
+// emitted.  map[0, K) and inv_map are written; k_out receives K.  When the run does not fit (see above) or
+// the histogram is degenerate (no tokens, nothing down to the cut), the full ranking takes over here too and
+// reads K off the sorted counts of the cut bucket's ranks.
+template <int MODE>
 __global__ void __cluster_dims__(kCluster, 1, 1) __launch_bounds__(kThreads, 1)
 k_select_sort(const uint32_t* counts, int32_t V, int32_t K, int32_t* map, int32_t* inv_map, uint32_t* keyA, uint32_t* valA, uint32_t* keyB,
-              uint32_t* valB) {
+              uint32_t* valB, double pfrac, uint32_t min_count, int32_t* k_out) {
     cg::cluster_group cluster = cg::this_cluster();
     const unsigned rank = cluster.block_rank();
     extern __shared__ __align__(16) uint8_t s_dyn[];
@@ -175,7 +240,12 @@ k_select_sort(const uint32_t* counts, int32_t V, int32_t K, int32_t* map, int32_
     uint32_t* s_gsize = s_gstart + kFine;                              // [kFine] its size over all CTAs
     uint32_t* s_next = s_gsize + kFine;                                // [kFine] scratch position of this CTA's next key
     unsigned long long* s_run = reinterpret_cast<unsigned long long*>(s_next + kFine);     // [kSortCap]
+    uint32_t* s_mlo = reinterpret_cast<uint32_t*>(s_run + kSortCap);   // [kFine] MODE 1: sum of the counts' low 16 bits (read by the peers)
+    uint32_t* s_mhi = s_mlo + kFine;                                   // [kFine]         and of their high 16 bits
     __shared__ uint32_t s_warp[kWarps + 1];
+    __shared__ unsigned long long s_wmass[kWarps + 1];
+    __shared__ unsigned long long s_mass_before;    // token mass of the buckets above the cut
+    __shared__ int s_cut_owner, s_K;
     __shared__ uint32_t s_load[kCluster];          // keys each CTA would have to rank
     __shared__ uint32_t s_work[kCluster];          // key comparisons that would take: sum of squared bucket sizes, in units of 1024
     __shared__ uint32_t s_T;
@@ -188,9 +258,12 @@ k_select_sort(const uint32_t* counts, int32_t V, int32_t K, int32_t* map, int32_
     constexpr int kInFlight = 8;
     unsigned long long* pairs = reinterpret_cast<unsigned long long*>(keyA);       // [V] 64-bit keys (keyA and valA are adjacent)
 
-    for (int i = threadIdx.x; i < kFine; i += kThreads) s_hist[i] = 0;
+    for (int i = threadIdx.x; i < kFine; i += kThreads) {
+        s_hist[i] = 0;
+        if (MODE == 1) { s_mlo[i] = 0; s_mhi[i] = 0; }
+    }
     if (threadIdx.x < kCluster) { s_load[threadIdx.x] = 0; s_work[threadIdx.x] = 0u; }
-    if (threadIdx.x == 0) { s_cut = 0; s_lo = 0x7fffffff; s_hi = 0; s_big = 0; }
+    if (threadIdx.x == 0) { s_cut = -1; s_lo = 0x7fffffff; s_hi = 0; s_big = 0; s_cut_owner = -1; s_K = 0; s_T = 0; s_mass_before = 0; }
     __syncthreads();
     // phase 1: bucket counts (descending order: inverted bucket index)
     for (int i = i0 + (int)threadIdx.x; i < i1; i += kThreads * kInFlight) {
@@ -199,7 +272,14 @@ k_select_sort(const uint32_t* counts, int32_t V, int32_t K, int32_t* map, int32_
         for (int q = 0; q < kInFlight; ++q) c[q] = i + q * kThreads < i1 ? __ldg(counts + i + q * kThreads) : 0u;
 #pragma unroll
         for (int q = 0; q < kInFlight; ++q)
-            if (i + q * kThreads < i1) atomicAdd(&s_hist[kFine - 1 - fine_bucket(c[q])], 1u);
+            if (i + q * kThreads < i1) {
+                const uint32_t b = kFine - 1 - fine_bucket(c[q]);
+                atomicAdd(&s_hist[b], 1u);
+                if (MODE == 1 && c[q] >= 256u) {   // (a bucket under 256 holds one value: its mass is a product)
+                    atomicAdd(&s_mlo[b], c[q] & 0xffffu);   // at most 2^14 ids per CTA: neither half can overflow 32 bits
+                    atomicAdd(&s_mhi[b], c[q] >> 16);
+                }
+            }
     }
     cluster.sync();
     // phase 2: start of every bucket in descending order (each thread owns kFine / kThreads neighbouring
@@ -224,6 +304,34 @@ k_select_sort(const uint32_t* counts, int32_t V, int32_t K, int32_t* map, int32_
     }
 #pragma unroll
     for (int q = 0; q < BPT; ++q) sum += tot[q];
+    unsigned long long mass[BPT], msum = 0;
+#pragma unroll
+    for (int q = 0; q < BPT; ++q) mass[q] = 0;
+    if (MODE == 1) {
+#pragma unroll
+        for (unsigned c = 0; c < kCluster; ++c) {
+            const uint4 lo4 = reinterpret_cast<const uint4*>(cluster.map_shared_rank(s_mlo, c))[threadIdx.x];
+            const uint4 hi4 = reinterpret_cast<const uint4*>(cluster.map_shared_rank(s_mhi, c))[threadIdx.x];
+            mass[0] += (unsigned long long)lo4.x + ((unsigned long long)hi4.x << 16);
+            mass[1] += (unsigned long long)lo4.y + ((unsigned long long)hi4.y << 16);
+            mass[2] += (unsigned long long)lo4.z + ((unsigned long long)hi4.z << 16);
+            mass[3] += (unsigned long long)lo4.w + ((unsigned long long)hi4.w << 16);
+        }
+#pragma unroll
+        for (int q = 0; q < BPT; ++q) {
+            const uint32_t value = (uint32_t)(kFine - 1 - (threadIdx.x * BPT + q));      // the bucket's count when under 256
+            if (value < 256u) mass[q] = (unsigned long long)value * tot[q];
+            msum += mass[q];
+        }
+    }
+    unsigned long long mincl = msum;
+    if (MODE == 1) {
+        for (int o = 1; o < 32; o <<= 1) {
+            const unsigned long long y = __shfl_up_sync(0xffffffffu, mincl, o);
+            if (lane >= o) mincl += y;
+        }
+        if (lane == 31) s_wmass[warp] = mincl;
+    }
     uint32_t incl = sum;
     for (int o = 1; o < 32; o <<= 1) {
         const uint32_t y = __shfl_up_sync(0xffffffffu, incl, o);
@@ -233,18 +341,38 @@ k_select_sort(const uint32_t* counts, int32_t V, int32_t K, int32_t* map, int32_
     __syncthreads();
     uint32_t start = incl - sum;
     for (int w = 0; w < warp; ++w) start += s_warp[w];
+    unsigned long long mstart = mincl - msum, mtotal = 0;
+    double target = 0.0;
+    if (MODE == 1) {
+        for (int w = 0; w < warp; ++w) mstart += s_wmass[w];
+        for (int w = 0; w < kWarps; ++w) mtotal += s_wmass[w];
+        target = ceil(pfrac * (double)mtotal);
+    }
+    const int min_bucket = MODE == 2 ? (int)(kFine - 1 - fine_bucket(min_count)) : 0;
 #pragma unroll
     for (int q = 0; q < BPT; ++q) {
         const int b = threadIdx.x * BPT + q;
         s_gstart[b] = start;
         s_gsize[b] = tot[q];
         s_next[b] = start + mine_before[q];
-        if (start < (uint32_t)K && start + tot[q] >= (uint32_t)K) { s_cut = b; s_T = start + tot[q]; }   // exactly one bucket
+        bool is_cut;
+        if (MODE == 0) is_cut = start < (uint32_t)K && start + tot[q] >= (uint32_t)K;                   // exactly one bucket
+        else if (MODE == 1) is_cut = (double)mstart < target && (double)(mstart + mass[q]) >= target;  // exactly one, if any token was counted
+        else is_cut = b == min_bucket;
+        if (is_cut) { s_cut = b; s_T = start + tot[q]; s_mass_before = mstart; s_K = (int)start; }
         start += tot[q];
+        mstart += mass[q];
     }
     __syncthreads();
     const int cut = s_cut;
     const uint32_t T = s_T;                             // keys to be ranked = end of the cut bucket
+    CutSpec spec{MODE, cut >= 0 && T > 0, (uint32_t)s_K, T, s_mass_before, target, min_count, k_out};
+    if (MODE != 0 && !spec.valid) {                     // no tokens at all / nothing as frequent as asked: K = 1 of the full ranking
+        cluster.sync();                                 // peers are done reading this CTA's counts
+        lsd_rank_all(cluster, counts, V, V, map, inv_map, keyA, valA, keyB, valB,
+                     reinterpret_cast<uint32_t (*)[kDigits]>(s_dyn), &spec);
+        return;
+    }
 #pragma unroll
     for (int q = 0; q < BPT; ++q) {
         const int b = threadIdx.x * BPT + q;
@@ -258,6 +386,7 @@ k_select_sort(const uint32_t* counts, int32_t V, int32_t K, int32_t* map, int32_
                 atomicMin(&s_lo, (int)st);
                 atomicMax(&s_hi, (int)(st + tot[q]));
             }
+            if (b == cut) s_cut_owner = (int)owner;
         }
     }
     __syncthreads();
@@ -265,6 +394,11 @@ k_select_sort(const uint32_t* counts, int32_t V, int32_t K, int32_t* map, int32_
     for (int c = 0; c < kCluster; ++c) fits = fits && s_load[c] <= (uint32_t)kSortCap && s_work[c] <= kWorkCap;
     if (!fits) {                                        // the same decision in every CTA (same inputs)
         cluster.sync();                                 // peers are done reading this CTA's counts
+        if (MODE != 0) {
+            lsd_rank_all(cluster, counts, V, V, map, inv_map, keyA, valA, keyB, valB,
+                         reinterpret_cast<uint32_t (*)[kDigits]>(s_dyn), &spec);
+            return;
+        }
         lsd_rank_all(cluster, counts, V, K, map, inv_map, keyA, valA, keyB, valB,
                      reinterpret_cast<uint32_t (*)[kDigits]>(s_dyn));
         return;
@@ -291,16 +425,63 @@ k_select_sort(const uint32_t* counts, int32_t V, int32_t K, int32_t* map, int32_
     const int r0 = s_lo, n = s_hi > s_lo ? s_hi - s_lo : 0;
     for (int j = threadIdx.x; j < n; j += kThreads) s_run[j] = __ldcg(pairs + r0 + j);
     __syncthreads();
-    for (int j = threadIdx.x; j < n; j += kThreads) {
+    if (MODE == 0) {
+        for (int j = threadIdx.x; j < n; j += kThreads) {
+            const unsigned long long key = s_run[j];
+            const int b = (int)(kFine - 1 - fine_bucket((uint32_t)(key >> 32)));
+            const int bs = (int)s_gstart[b] - r0, be = bs + (int)s_gsize[b];
+            int r = 0;
+            for (int i = bs; i < be; ++i) r += s_run[i] > key ? 1 : 0;
+            const int rk = r0 + bs + r;
+            const int32_t v = (int32_t)(0xffffffffu - (uint32_t)key);
+            if (rk < K) map[rk] = v;
+            inv_map[v] = rk < K ? rk : -1;
+        }
+        return;
+    }
+    // K from the ranks: first every key's place (and, inside the cut bucket, the token mass ranked before it),
+    // then -- in the CTA that ranks the cut bucket -- K, then the outputs.  The other CTAs rank buckets above
+    // the cut only: all of theirs is kept.
+    int place[kKeysPerThread];
+    const bool owns_cut = s_cut_owner == (int)rank || (s_cut_owner < 0 && rank == 0);   // (an empty cut bucket has no owner)
+    const unsigned long long mass_before = s_mass_before;
+#pragma unroll
+    for (int q = 0; q < kKeysPerThread; ++q) {
+        const int j = threadIdx.x + q * kThreads;
+        place[q] = -1;
+        if (j >= n) continue;
         const unsigned long long key = s_run[j];
-        const int b = (int)(kFine - 1 - fine_bucket((uint32_t)(key >> 32)));
+        const uint32_t cnt = (uint32_t)(key >> 32);
+        const int b = (int)(kFine - 1 - fine_bucket(cnt));
         const int bs = (int)s_gstart[b] - r0, be = bs + (int)s_gsize[b];
         int r = 0;
-        for (int i = bs; i < be; ++i) r += s_run[i] > key ? 1 : 0;
-        const int rk = r0 + bs + r;
-        const int32_t v = (int32_t)(0xffffffffu - (uint32_t)key);
-        if (rk < K) map[rk] = v;
-        inv_map[v] = rk < K ? rk : -1;
+        unsigned long long m = 0;
+        if (b == cut && MODE == 1) {
+            for (int i = bs; i < be; ++i) {
+                const unsigned long long o = s_run[i];
+                const bool gt = o > key;
+                r += gt ? 1 : 0;
+                m += gt ? (o >> 32) : 0ull;
+            }
+            const unsigned long long cum = mass_before + m;
+            if ((double)cum < target && (double)(cum + cnt) >= target) s_K = r0 + bs + r + 1;   // exactly one key
+        } else {
+            for (int i = bs; i < be; ++i) r += s_run[i] > key ? 1 : 0;
+            if (b == cut && MODE == 2 && cnt >= min_count) atomicMax(&s_K, r0 + bs + r + 1);
+        }
+        place[q] = r0 + bs + r;
+    }
+    __syncthreads();
+    const int Kf = owns_cut ? max(1, min(V, s_K)) : (int)T;
+    if (owns_cut && threadIdx.x == 0) *k_out = Kf;
+#pragma unroll
+    for (int q = 0; q < kKeysPerThread; ++q) {
+        const int j = threadIdx.x + q * kThreads;
+        if (j >= n) continue;
+        const int32_t v = (int32_t)(0xffffffffu - (uint32_t)s_run[j]);
+        const int rk = place[q];
+        if (rk < Kf) map[rk] = v;
+        inv_map[v] = rk < Kf ? rk : -1;
     }
 }
 
@@ -313,108 +494,41 @@ k_select_full(const uint32_t* counts, int32_t V, int32_t K, int32_t* map, int32_
     lsd_rank_all(cluster, counts, V, K, map, inv_map, keyA, valA, keyB, valB, reinterpret_cast<uint32_t (*)[kDigits]>(s_dyn));
 }
 
-// Cut of a full ranking at a data-dependent K (the Method section's Top-P and minimum-frequency
-// variants of the selection).  `map` holds all V ids in rank order.  mode 0: smallest K whose prefix
-// of counts reaches ceil(p * total); mode 1: K = number of ids with count >= min_count.  K is clamped
-// to [1, V]; inv_map entries of ranks >= K become -1.  Pure latency (two dependent loads per rank), so
-// the ranks are dealt to the 8 CTAs of a cluster, each thread a contiguous run; the CTAs' sums meet
-// through distributed shared memory, like the digit totals of the sort.
-__global__ void __cluster_dims__(kCluster, 1, 1) __launch_bounds__(kThreads, 1)
-k_select_cut(const uint32_t* __restrict__ counts, int32_t V, int mode, double pfrac, uint32_t min_count,
-             const int32_t* __restrict__ map, int32_t* __restrict__ inv_map, int32_t* __restrict__ k_out) {
-    cg::cluster_group cluster = cg::this_cluster();
-    const unsigned rank = cluster.block_rank();
-    __shared__ unsigned long long s_part[kThreads];
-    __shared__ unsigned long long s_cta_total;          // this CTA's sum (read by the peers)
-    __shared__ int s_k;                                 // CTA 0's copy is the cluster's answer
-    const int T = kCluster * kThreads;                  // threads of the cluster, in rank order
-    const int t = (int)rank * kThreads + (int)threadIdx.x;
-    const int per = (V + T - 1) / T;                    // consecutive ranks per thread
-    const int j0 = min(V, t * per), j1 = min(V, j0 + per);
-    unsigned long long sum = 0;
-    int ge = 0;
-    for (int j = j0; j < j1; j += 8) {                  // eight ranks (id, then its count) in flight per thread
-        int32_t id[8];
-        uint32_t c[8];
-#pragma unroll
-        for (int q = 0; q < 8; ++q) id[q] = j + q < j1 ? map[j + q] : -1;
-#pragma unroll
-        for (int q = 0; q < 8; ++q) c[q] = id[q] >= 0 ? counts[id[q]] : 0u;
-#pragma unroll
-        for (int q = 0; q < 8; ++q) {
-            sum += c[q];
-            ge += (id[q] >= 0) & (c[q] >= min_count);
-        }
-    }
-    s_part[threadIdx.x] = mode == 0 ? sum : (unsigned long long)ge;
-    if (threadIdx.x == 0) s_k = V;
-    __syncthreads();
-    if (threadIdx.x < 32) {                             // exclusive scan of this CTA's 1024 partials by one warp
-        unsigned long long x[kThreads / 32], run = 0;
-#pragma unroll
-        for (int q = 0; q < kThreads / 32; ++q) {       // lane l owns partials 32 l .. 32 l + 31
-            x[q] = s_part[threadIdx.x * (kThreads / 32) + q];
-            run += x[q];
-        }
-        unsigned long long incl = run;
-        for (int o = 1; o < 32; o <<= 1) {
-            const unsigned long long y = __shfl_up_sync(0xffffffffu, incl, o);
-            if ((int)threadIdx.x >= o) incl += y;
-        }
-        unsigned long long pre = incl - run;
-#pragma unroll
-        for (int q = 0; q < kThreads / 32; ++q) {
-            s_part[threadIdx.x * (kThreads / 32) + q] = pre;
-            pre += x[q];
-        }
-        if (threadIdx.x == 31) s_cta_total = incl;
-    }
-    cluster.sync();                                     // every CTA's total and s_k are in place
-    unsigned long long before = 0, total = 0;           // sums of the CTAs before this one / of all
-    for (unsigned c = 0; c < kCluster; ++c) {
-        const unsigned long long x = *cluster.map_shared_rank(&s_cta_total, c);
-        before += c < rank ? x : 0ull;
-        total += x;
-    }
-    int* k_shared = cluster.map_shared_rank(&s_k, 0);
-    if (mode == 0) {
-        const double target = ceil(pfrac * (double)total);
-        unsigned long long cum = before + s_part[threadIdx.x];
-        if (t == 0 && target <= 0.0) atomicMin(k_shared, 1);           // an empty histogram: the first rank already reaches it
-        // only the thread whose run of ranks crosses the target walks it again
-        if ((double)cum < target && (double)(cum + sum) >= target) {
-            for (int j = j0; j < j1; ++j) {
-                cum += counts[map[j]];
-                if ((double)cum >= target) { atomicMin(k_shared, j + 1); break; }
-            }
-        }
-    } else if (t == 0) {
-        atomicMin(k_shared, (int)total);
-    }
-    cluster.sync();                                     // the answer is final; CTA 0 stays until all have read it
-    const int K = max(1, min(V, *k_shared));
-    if (t == 0) *k_out = K;
-    for (int j = K + t; j < V; j += T * 8) {            // eight ids in flight per thread
-        int32_t id[8];
-#pragma unroll
-        for (int q = 0; q < 8; ++q) id[q] = j + q * T < V ? map[j + q * T] : -1;
-#pragma unroll
-        for (int q = 0; q < 8; ++q)
-            if (id[q] >= 0) inv_map[id[q]] = -1;
-    }
-    cluster.sync();                                     // nobody leaves while a peer may still read its shared memory
-}
-
 }  // namespace
 
+static cudaError_t select_smem_attr() {
+    static int attr_done[64] = {0};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev >= 0 && dev < 64 && attr_done[dev]) return cudaSuccess;
+    e = cudaFuncSetAttribute(k_select_sort<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSelectSmem);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(k_select_sort<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSelectCutSmem);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(k_select_sort<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSelectCutSmem);
+    if (e == cudaSuccess && dev >= 0 && dev < 64) attr_done[dev] = 1;
+    return e;
+}
+
+// Top-P (mode 0) / minimum frequency (mode 1): the selection kernel in the mode that finds K on its way.
 cudaError_t launch_select_cut(const uint32_t* counts, int32_t V, int mode, double pfrac, uint32_t min_count,
-                              const int32_t* map, int32_t* inv_map, int32_t* k_out, cudaStream_t s) {
-    k_select_cut<<<kCluster, kThreads, 0, s>>>(counts, V, mode, pfrac, min_count, map, inv_map, k_out);
+                              int32_t* map, int32_t* inv_map, int32_t* k_out, uint8_t* scratch, cudaStream_t s) {
+    const size_t seg = align_up((size_t)V * 4, 256);
+    uint32_t* keyA = reinterpret_cast<uint32_t*>(scratch);
+    uint32_t* valA = reinterpret_cast<uint32_t*>(scratch + seg);
+    uint32_t* keyB = reinterpret_cast<uint32_t*>(scratch + 2 * seg);
+    uint32_t* valB = reinterpret_cast<uint32_t*>(scratch + 3 * seg);
+    cudaError_t e = select_smem_attr();
+    if (e != cudaSuccess) return e;
+    if (mode == 0)
+        k_select_sort<1><<<kCluster, kThreads, kSelectCutSmem, s>>>(counts, V, 0, map, inv_map, keyA, valA, keyB, valB, pfrac, 0u, k_out);
+    else
+        k_select_sort<2><<<kCluster, kThreads, kSelectCutSmem, s>>>(counts, V, 0, map, inv_map, keyA, valA, keyB, valB, 1.0, min_count, k_out);
     count_launch();
     return cudaGetLastError();
 }
 
 size_t select_scratch_bytes(int32_t V) { return 4 * align_up((size_t)V * 4, 256); }
+size_t select_cut_scratch_bytes(int32_t V) { return select_scratch_bytes(V); }
 
 cudaError_t launch_select_topk(const uint32_t* counts, int32_t V, int32_t K, int32_t* map,
                                int32_t* inv_map, uint8_t* scratch, cudaStream_t s) {
@@ -423,19 +537,12 @@ cudaError_t launch_select_topk(const uint32_t* counts, int32_t V, int32_t K, int
     uint32_t* valA = reinterpret_cast<uint32_t*>(scratch + seg);
     uint32_t* keyB = reinterpret_cast<uint32_t*>(scratch + 2 * seg);
     uint32_t* valB = reinterpret_cast<uint32_t*>(scratch + 3 * seg);
-    static int attr_done[64] = {0};
-    int dev = 0;
-    cudaError_t e = cudaGetDevice(&dev);
+    cudaError_t e = select_smem_attr();
     if (e != cudaSuccess) return e;
-    if (dev < 0 || dev >= 64 || !attr_done[dev]) {
-        e = cudaFuncSetAttribute(k_select_sort, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSelectSmem);
-        if (e != cudaSuccess) return e;
-        if (dev >= 0 && dev < 64) attr_done[dev] = 1;
-    }
     if ((long long)K * 2 > V)          // more than half the ranking is wanted: rank everything, select nothing
         k_select_full<<<kCluster, kThreads, sizeof(uint32_t) * kWarps * kDigits, s>>>(counts, V, K, map, inv_map, keyA, valA, keyB, valB);
     else
-        k_select_sort<<<kCluster, kThreads, kSelectSmem, s>>>(counts, V, K, map, inv_map, keyA, valA, keyB, valB);
+        k_select_sort<0><<<kCluster, kThreads, kSelectSmem, s>>>(counts, V, K, map, inv_map, keyA, valA, keyB, valB, 1.0, 0u, nullptr);
     count_launch();
     return cudaGetLastError();
 }
