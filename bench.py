@@ -462,10 +462,10 @@ def extras(vt, dev, peak_gbs, peak_kind):
         vb["build_vocab_K%d_gtok_s" % K] = n / (ms_b * 1e-3) / 1e9
     ms_s = timed(lambda: vt.vt_select_topk(counts, 32768, ws=ws), reps=20)
     vb["select_topk_K32768_us"] = ms_s * 1e3
-    ms_p = timed(lambda: vt.vt_select_topp(counts, 0.99, ws=ws), reps=20)
-    vb["select_topp_p0.99_us"] = ms_p * 1e3
-    ms_f = timed(lambda: vt.vt_select_minfreq(counts, 100, ws=ws), reps=20)
-    vb["select_minfreq_100_us"] = ms_f * 1e3
+    for p_ in (0.9, 0.99):
+        vb["select_topp_p%g_us" % p_] = timed(lambda: vt.vt_select_topp(counts, p_, ws=ws), reps=20) * 1e3
+    for f_ in (1000, 100):
+        vb["select_minfreq_%d_us" % f_] = timed(lambda: vt.vt_select_minfreq(counts, f_, ws=ws), reps=20) * 1e3
     del ids
     torch.cuda.empty_cache()
     W_full = vt_inputs.gaussian_bf16((V, 4096), 0.02, seed=1006, device=dev)
