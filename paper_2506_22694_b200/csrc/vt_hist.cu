@@ -100,6 +100,10 @@ __device__ __forceinline__ void report_bad(unsigned long long bad, Ctrl* ctrl) {
 }
 
 // ---- all bins private to each CTA ----------------------------------------------------------------
+// Same walk as the packed kernel below: whole trips of kRows 128-bit loads per thread without a bounds test,
+// one range test per load, then the guarded rest; CTA 0 takes the ragged ends.
+constexpr int kRows = 6;                       // 128-bit loads a thread has in flight per trip (96 KB per CTA): four
+                                               // leave HBM waiting, seven leave no registers for the tally
 __global__ void __launch_bounds__(kThreads, 1)
 k_hist_small(const int32_t* __restrict__ ids, int64_t n, int32_t V, uint32_t* __restrict__ counts,
              Ctrl* ctrl) {
@@ -107,13 +111,43 @@ k_hist_small(const int32_t* __restrict__ ids, int64_t n, int32_t V, uint32_t* __
     for (int i = threadIdx.x; i < V; i += kThreads) s_bins[i] = 0;
     __syncthreads();
     unsigned long long bad = 0;
-    stream_ids(ids, n, [&](uint32_t id) {
+    auto tally1 = [&](uint32_t id) {
         if (id < (uint32_t)V) atomicAdd(&s_bins[id], 1u);
         else ++bad;
-    });
+    };
+    auto tally4 = [&](uint4 x) {
+        if (max(max(x.x, x.y), max(x.z, x.w)) < (uint32_t)V) {
+            atomicAdd(&s_bins[x.x], 1u); atomicAdd(&s_bins[x.y], 1u); atomicAdd(&s_bins[x.z], 1u); atomicAdd(&s_bins[x.w], 1u);
+        } else {
+            tally1(x.x); tally1(x.y); tally1(x.z); tally1(x.w);
+        }
+    };
+    const uintptr_t addr = reinterpret_cast<uintptr_t>(ids);
+    int64_t head = ((16 - (addr & 15)) & 15) >> 2;
+    if (head > n) head = n;
+    const int64_t nvec = (n - head) >> 2;
+    const int64_t tail0 = head + nvec * 4;
+    if (blockIdx.x == 0) {
+        if ((int64_t)threadIdx.x < head) tally1((uint32_t)ids[threadIdx.x]);
+        const int64_t t = tail0 + threadIdx.x;
+        if (t < n) tally1((uint32_t)ids[t]);
+    }
+    const uint4* vec = reinterpret_cast<const uint4*>(ids + head);
+    const int64_t v0 = nvec * blockIdx.x / gridDim.x;
+    const int64_t v1 = nvec * (blockIdx.x + 1) / gridDim.x;
+    const int64_t trips = (v1 - v0) / (kRows * kThreads);
+    const uint4* p = vec + v0 + threadIdx.x;
+    for (int64_t t = 0; t < trips; ++t, p += kRows * kThreads) {
+        uint4 x[kRows];
+#pragma unroll
+        for (int r = 0; r < kRows; ++r) x[r] = ld_stream_u4(p + r * kThreads);
+#pragma unroll
+        for (int r = 0; r < kRows; ++r) tally4(x[r]);
+    }
+    for (int64_t v = v0 + trips * (kRows * kThreads) + threadIdx.x; v < v1; v += kThreads) tally4(ld_stream_u4(vec + v));
     __syncthreads();
     for (int i = threadIdx.x; i < V; i += kThreads) {
-        const int v = (i + blockIdx.x * 61) % V;        // de-phase the CTAs' flushes
+        const int v = (i + blockIdx.x * (V / (int)gridDim.x)) % V;   // the CTAs' flushes spread over the whole array
         const uint32_t c = s_bins[v];
         if (c) atomicAdd(&counts[v], c);
     }
@@ -397,8 +431,6 @@ k_hist_hot(const int32_t* __restrict__ ids, int64_t n, int32_t V, uint32_t* __re
 // and count the stream again with the hot / cold kernels.
 constexpr uint32_t kFieldBits = 10, kFieldMax = (1u << kFieldBits) - 1, kSpill = 512;
 constexpr uint32_t kNoId = 0xffffffffu;        // no token id: ids are tallied only when < V <= 2^31
-constexpr int kRows = 6;                       // 128-bit loads a thread has in flight per trip (96 KB per CTA): four
-                                               // leave HBM waiting, seven leave no registers for the tally
 constexpr int kCarefulTrips = 2;               // trips a CTA counts one add at a time, until its hot id is known
 constexpr int kGateWords = 4;                  // {recount, unused, skipped ids (64 bits)}
 
