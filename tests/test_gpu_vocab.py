@@ -127,6 +127,26 @@ def test_histogram_hot_tokens_that_arrive_late_and_skipped_ids_are_counted_once(
         assert flags == vt.VT_FLAG_BAD_ID and n_bad == bad
 
 
+@pytest.mark.parametrize("shares", [(0.05,), (0.125, 0.125), (0.2,), (0.35, 0.1), (0.6,), (0.3, 0.3, 0.3), (1.0,)])
+def test_histogram_skewed_streams_whichever_kernels_count_them(shares):
+    """Streams in which one to three tokens hold the given shares, plus a run of 700 000 repeats of one token
+    in the middle: some stay with the packed kernel, some make a field wrap and are counted again."""
+    V, n = 128256, 8_000_000
+    g = torch.Generator(device=DEV).manual_seed(int(sum(shares) * 1000) + len(shares))
+    ids = torch.randint(0, V, (n,), device=DEV, dtype=torch.int32, generator=g)
+    u = torch.rand(n, device=DEV, generator=g)
+    lo = 0.0
+    for k, sh in enumerate(shares):
+        ids[(u >= lo) & (u < lo + sh)] = (k * 40_009 + 17) % V
+        lo += sh
+    ids[n // 3: n // 3 + 700_000] = 99_991
+    ws = vt.Workspace(vt.workspace_bytes(vt.VT_OP_HISTOGRAM, n, V))
+    ref, bad = oracle.histogram(ids.cpu().numpy(), V)
+    assert bad == 0
+    assert np.array_equal(_u32(vt.vt_histogram(ids, V, ws=ws)), ref)
+    _assert_clean(ws)
+
+
 def test_histogram_three_ids_carry_the_whole_stream():
     """Streams that drive single bins to 1e7 and more: neighbouring ids, ids around the middle and the
     end of the vocabulary, with a sprinkle of a fourth id."""
