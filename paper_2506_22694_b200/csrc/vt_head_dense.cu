@@ -38,6 +38,7 @@ namespace {
 constexpr int kBM = 128;                  // hidden rows per CTA (TMEM lanes)
 constexpr int kMaxBN = 256;               // vocabulary rows per tile at most (TMEM columns per accumulator)
 constexpr int kBK = 64;                   // columns of d per ring stage: 128 bytes, one swizzle row
+constexpr int kMaxSub = 2;                // d-steps of kBK columns one ring stage holds at most
 constexpr int kMaxStages = 8;
 constexpr int kHTileBytes = kBM * kBK * 2; // 16 KB: the hidden-row operand of a stage
 constexpr int kParts8 = 2, kParts16 = 2;  // epilogue warps per TMEM lane quadrant for lists of 8 / 16 (3 and 4 were no
@@ -208,6 +209,8 @@ struct DenseGeo {
     int n_stages;     // ring depth
     int stage_bytes;  // bytes one CTA stages per step: hidden rows + its share of the vocabulary rows
     int n_groups;     // CTAs (or CTA pairs) walking the tiles round-robin
+    int sub;          // d-steps per ring stage (1 or 2): one wait and one release per stage, so two steps per stage halve
+                      // what the two single threads that drive the ring spend per MMA; taken when three such stages fit
 };
 
 // Per-thread state of one hidden row over the columns the thread has seen.
@@ -263,6 +266,9 @@ k_head_dense(const HeadArgs a, Ctrl* ctrl, float* __restrict__ recs, const Dense
     const int w_rows = PAIR ? bn / 2 : bn;                         // vocabulary rows this CTA stages per step
 
     if (threadIdx.x == 0) {
+        // the two tensor maps are fetched now, not by the first copy that needs them
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_h)) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_w)) : "memory");
         for (int s = 0; s < kMaxStages; ++s) { mbar_init(&s_full[s], 1); mbar_init(&s_empty[s], 1); }
         for (int p = 0; p < 2; ++p) { mbar_init(&s_acc_full[p], 1); mbar_init(&s_acc_empty[p], (PAIR ? 2 : 1) * 4 * PARTS); }
         s_abort = 0;
@@ -294,38 +300,71 @@ k_head_dense(const HeadArgs a, Ctrl* ctrl, float* __restrict__ recs, const Dense
         if (lane == 0) {
             // fills are numbered g = 0 .. total-1 over (tile, step in d); fill g uses stage g % n_stages
             const int my_tiles = (geo.n_tiles - group + geo.n_groups - 1) / geo.n_groups;
-            const int total = my_tiles * geo.n_kc;
-            const uint32_t bytes = (uint32_t)(PAIR ? 2 : 1) * (uint32_t)geo.stage_bytes;
+            const int sub = geo.sub;
+            const int n_ks = (geo.n_kc + sub - 1) / sub;               // ring stages per tile
+            const int total = my_tiles * n_ks;
+            const uint32_t sub_bytes = (uint32_t)geo.stage_bytes / (uint32_t)sub;
             const uint32_t full0 = PAIR ? mapa_u32(smem_u32(&s_full[0]), 0) : 0u;      // the leader's full barriers
+            auto subs_of = [&](int g) { return min(sub, geo.n_kc - (g % n_ks) * sub); };
             auto load_w = [&](int g) {
-                const int s = g % n_stages, tile = group + (g / geo.n_kc) * geo.n_groups, kc = g % geo.n_kc;
-                const uint32_t dst = ring_u32 + (uint32_t)s * (uint32_t)geo.stage_bytes + kHTileBytes;
-                if (PAIR) tma_load_2d_pair(dst, &tm_w, kc * kBK, tile * bn + (int)rank * w_rows, full0 + (uint32_t)(s * sizeof(uint64_t)));
-                else tma_load_2d(dst, &tm_w, kc * kBK, tile * bn, &s_full[s]);
+                const int s = g % n_stages, tile = group + (g / n_ks) * geo.n_groups;
+                for (int u = 0; u < subs_of(g); ++u) {
+                    const int kc = (g % n_ks) * sub + u;
+                    const uint32_t dst = ring_u32 + (uint32_t)s * (uint32_t)geo.stage_bytes + (uint32_t)u * sub_bytes + kHTileBytes;
+                    if (PAIR) tma_load_2d_pair(dst, &tm_w, kc * kBK, tile * bn + (int)rank * w_rows, full0 + (uint32_t)(s * sizeof(uint64_t)));
+                    else tma_load_2d(dst, &tm_w, kc * kBK, tile * bn, &s_full[s]);
+                }
             };
             auto load_h = [&](int g) {
-                const int s = g % n_stages, kc = g % geo.n_kc;
-                const uint32_t dst = ring_u32 + (uint32_t)s * (uint32_t)geo.stage_bytes;
-                if (PAIR) tma_load_2d_pair(dst, &tm_h, kc * kBK, (int)rank * kBM, full0 + (uint32_t)(s * sizeof(uint64_t)));
-                else tma_load_2d(dst, &tm_h, kc * kBK, 0, &s_full[s]);
+                const int s = g % n_stages;
+                for (int u = 0; u < subs_of(g); ++u) {
+                    const int kc = (g % n_ks) * sub + u;
+                    const uint32_t dst = ring_u32 + (uint32_t)s * (uint32_t)geo.stage_bytes + (uint32_t)u * sub_bytes;
+                    if (PAIR) tma_load_2d_pair(dst, &tm_h, kc * kBK, (int)rank * kBM, full0 + (uint32_t)(s * sizeof(uint64_t)));
+                    else tma_load_2d(dst, &tm_h, kc * kBK, 0, &s_full[s]);
+                }
             };
+            auto bytes_of = [&](int g) { return (uint32_t)(PAIR ? 2 : 1) * sub_bytes * (uint32_t)subs_of(g); };
             // The weights are static: the first ring of them is requested before the work this launch
             // depends on has finished; everything that work may have produced is touched after the wait.
             const int pre = min(n_stages, total);
             for (int g = 0; g < pre; ++g) {
-                if (rank == 0) mbar_expect_tx(&s_full[g], bytes);
+                if (rank == 0) mbar_expect_tx(&s_full[g], bytes_of(g));
                 load_w(g);
             }
             griddep_wait();
             VT_DSTAMP(2);
             for (int g = 0; g < pre; ++g) load_h(g);
             int done = pre;
-            for (int g = pre; g < total; ++g, ++done) {
-                const int s = g % n_stages;
-                if (!mbar_wait(&s_empty[s], (uint32_t)((g / n_stages) & 1) ^ 1u, abort_flag)) break;
-                if (rank == 0) mbar_expect_tx(&s_full[s], bytes);
-                load_h(g);
-                load_w(g);
+            {
+                // steady state: the cursor over (stage, step in d, tile) moves by additions only -- this thread's
+                // turn-around between "stage free" and "copies asked for" is on the ring's critical path
+                int sc = pre % n_stages, ks = pre % n_ks, tl = pre / n_ks;
+                uint32_t par = (uint32_t)((pre / n_stages) & 1) ^ 1u;
+                const uint32_t pair_mul = PAIR ? 2u : 1u;
+                for (int g = pre; g < total; ++g, ++done) {
+                    if (!mbar_wait(&s_empty[sc], par, abort_flag)) break;
+                    const int subs = min(sub, geo.n_kc - ks * sub);
+                    if (rank == 0) mbar_expect_tx(&s_full[sc], pair_mul * sub_bytes * (uint32_t)subs);
+                    const uint32_t dst0 = ring_u32 + (uint32_t)sc * (uint32_t)geo.stage_bytes;
+                    const uint32_t bar = full0 + (uint32_t)(sc * sizeof(uint64_t));
+                    const int row_w = (group + tl * geo.n_groups) * bn + (PAIR ? (int)rank * w_rows : 0);
+#pragma unroll
+                    for (int u = 0; u < kMaxSub; ++u) {
+                        if (u < subs) {
+                            const int x = (ks * sub + u) * kBK;
+                            if (PAIR) {
+                                tma_load_2d_pair(dst0 + (uint32_t)u * sub_bytes, &tm_h, x, (int)rank * kBM, bar);
+                                tma_load_2d_pair(dst0 + (uint32_t)u * sub_bytes + kHTileBytes, &tm_w, x, row_w, bar);
+                            } else {
+                                tma_load_2d(dst0 + (uint32_t)u * sub_bytes, &tm_h, x, 0, &s_full[sc]);
+                                tma_load_2d(dst0 + (uint32_t)u * sub_bytes + kHTileBytes, &tm_w, x, row_w, &s_full[sc]);
+                            }
+                        }
+                    }
+                    if (++sc == n_stages) { sc = 0; par ^= 1u; }
+                    if (++ks == n_ks) { ks = 0; ++tl; }
+                }
             }
             if (done == total && !*abort_flag) {
                 // every fill consumed: all copies have landed and every commit aimed at this CTA's
@@ -343,6 +382,8 @@ k_head_dense(const HeadArgs a, Ctrl* ctrl, float* __restrict__ recs, const Dense
         // ================= MMA issuer (leader CTA only) ================================================
         if (lane == 0 && rank == 0) {
             const uint32_t idesc = make_idesc(PAIR ? 2 * kBM : kBM, bn);
+            const uint64_t desc_a0 = make_desc(ring_u32);                       // (the ring is 1024-byte aligned and under 256 KB:
+            const uint64_t sub16 = (uint64_t)(((uint32_t)geo.stage_bytes / (uint32_t)geo.sub) >> 4);   //  adding byte offsets >> 4 stays inside the address field)
             int s = 0, t_local = 0;
             uint32_t ph = 0;
             bool alive = true;
@@ -352,18 +393,27 @@ k_head_dense(const HeadArgs a, Ctrl* ctrl, float* __restrict__ recs, const Dense
                 if (t_local >= 2 && !mbar_wait(&s_acc_empty[as], (use - 1) & 1, abort_flag)) { alive = false; break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(as * kMaxBN);
-                for (int kc = 0; kc < geo.n_kc; ++kc) {
+                const int n_ks = (geo.n_kc + geo.sub - 1) / geo.sub;
+                for (int ks = 0; ks < n_ks; ++ks) {
+                    const int kc = ks * geo.sub;
                     if (!mbar_wait(&s_full[s], ph, abort_flag)) { alive = false; break; }
 #ifdef VT_STAMPS
                     if (t_local == 0 && kc == 0) VT_DSTAMP(3);
 #endif
                     tc_fence_after();
-                    const uint32_t base = ring_u32 + (uint32_t)s * (uint32_t)geo.stage_bytes;
+                    const int subs = min(geo.sub, geo.n_kc - kc);
+                    const uint64_t da0 = desc_a0 + (uint64_t)(((uint32_t)s * (uint32_t)geo.stage_bytes) >> 4);
+                    const uint64_t db0 = da0 + (uint64_t)(kHTileBytes >> 4);
 #pragma unroll
-                    for (int k = 0; k < kBK / 16; ++k) {
-                        const uint64_t da = make_desc(base + k * 32), db = make_desc(base + kHTileBytes + k * 32);
-                        if (PAIR) tc_mma_pair(d_tmem, da, db, idesc, (kc | k) != 0 ? 1u : 0u);
-                        else tc_mma(d_tmem, da, db, idesc, (kc | k) != 0 ? 1u : 0u);
+                    for (int u = 0; u < kMaxSub; ++u) {
+                        if (u < subs) {
+#pragma unroll
+                            for (int k = 0; k < kBK / 16; ++k) {
+                                const uint64_t step = (uint64_t)u * sub16 + (uint64_t)(k * 2);
+                                if (PAIR) tc_mma_pair(d_tmem, da0 + step, db0 + step, idesc, (kc | u | k) != 0 ? 1u : 0u);
+                                else tc_mma(d_tmem, da0 + step, db0 + step, idesc, (kc | u | k) != 0 ? 1u : 0u);
+                            }
+                        }
                     }
                     // the stage is free (in both CTAs) once these MMAs have read it
                     if (PAIR) tc_commit_pair(&s_empty[s]); else tc_commit(&s_empty[s]);
@@ -659,7 +709,9 @@ DenseGeo make_geo(int32_t K, int32_t d, bool pair, int max_groups) {
     g.n_tiles = (K + g.bn - 1) / g.bn;
     g.n_kc = (d + kBK - 1) / kBK;
     g.n_groups = g.n_tiles < max_groups ? g.n_tiles : max_groups;
-    g.stage_bytes = kHTileBytes + (pair ? g.bn / 2 : g.bn) * kBK * 2;
+    const int step_bytes = kHTileBytes + (pair ? g.bn / 2 : g.bn) * kBK * 2;
+    g.sub = (3 * kMaxSub * (size_t)step_bytes <= kRingBudget && g.n_kc >= kMaxSub) ? kMaxSub : 1;
+    g.stage_bytes = step_bytes * g.sub;
     g.n_stages = (int)(kRingBudget / (size_t)g.stage_bytes);
     if (g.n_stages > kMaxStages) g.n_stages = kMaxStages;
     return g;
