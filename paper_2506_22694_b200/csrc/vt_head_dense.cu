@@ -12,7 +12,9 @@
 // bytes staged and read compared with two M tiles in one CTA, which is what bounded that form.
 //
 // Warp 0 feeds a shared-memory ring with TMA tensor copies (128-byte swizzle, every CTA fetches its own tiles); in a pair
-// both CTAs' copies count their bytes on the leader's barrier.  One thread of warp 1 (of the leader)
+// both CTAs' copies count their bytes on the leader's barrier.  A ring stage holds one or two 64-column steps of d
+// (two where three such stages fit): the two threads that drive the ring wait and release once per stage, and their
+// turn-around is on its critical path, so they also move their cursors by additions only.  One thread of warp 1 (of the leader)
 // issues the MMAs (bf16 x bf16 -> fp32) with the operands described in place by shared-memory
 // descriptors and the accumulators in tensor memory: two accumulator stages of up to 256 columns, so
 // the epilogue of tile t overlaps the MMAs of tile t+1.  tcgen05.commit releases ring stages and
