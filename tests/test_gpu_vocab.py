@@ -294,6 +294,35 @@ def test_select_minfreq_matches_oracle(V, n, f):
     _assert_clean(ws)
 
 
+@pytest.mark.parametrize("shape", ["tiny_values", "few_wide_buckets", "spikes_over_noise", "around_256", "one_value"])
+def test_select_cuts_over_count_shapes_that_stress_the_buckets(shape):
+    """Count vectors chosen against the bucket scheme of the selection kernel: huge buckets of equal counts, all
+    counts in a handful of wide buckets, a few enormous counts over noise, counts on both sides of the value from
+    which a bucket holds more than one count, and a single value.  Top-P, minimum frequency and Top-K."""
+    V = 50_000
+    rng = np.random.default_rng(len(shape))
+    c = {"tiny_values": rng.integers(0, 4, V), "few_wide_buckets": rng.integers(1 << 20, 1 << 21, V),
+         "spikes_over_noise": np.where(rng.random(V) < 0.01, rng.integers(1 << 28, 1 << 31, V), rng.integers(0, 3, V)),
+         "around_256": rng.integers(250, 262, V), "one_value": np.full(V, 12345)}[shape].astype(np.uint64)
+    counts = torch.from_numpy(c.astype(np.uint32).view(np.int32)).to(DEV)
+    ws = vt.Workspace(vt.workspace_bytes(vt.VT_OP_SELECT_TOPK, 0, V, V))
+    for p in (1e-12, 0.3, 0.9, 1.0):
+        k_out, map_, inv = vt.vt_select_topp(counts, p, ws=ws)
+        K, rmap, rinv = oracle.select_topp(c, p)
+        assert int(k_out.item()) == K
+        assert np.array_equal(map_.cpu().numpy()[:K], rmap[:K]) and np.array_equal(inv.cpu().numpy(), rinv)
+    for f in (0, 1, 255, 256, 257, int(np.median(c)), int(c.max()), int(c.max()) + 1):
+        k_out, map_, inv = vt.vt_select_minfreq(counts, f, ws=ws)
+        K, rmap, rinv = oracle.select_minfreq(c, f)
+        assert int(k_out.item()) == K
+        assert np.array_equal(map_.cpu().numpy()[:K], rmap[:K]) and np.array_equal(inv.cpu().numpy(), rinv)
+    for K in (1, V // 3, V // 2 + 1, V):
+        map_, inv = vt.vt_select_topk(counts, K, ws=ws)
+        rmap, rinv = oracle.select_topk(c, K)
+        assert np.array_equal(map_.cpu().numpy(), rmap) and np.array_equal(inv.cpu().numpy(), rinv)
+    _assert_clean(ws)
+
+
 def test_select_cut_degenerate_counts_and_bad_arguments():
     V = 4096
     ws = vt.Workspace(vt.workspace_bytes(vt.VT_OP_SELECT_TOPK, 0, V, V))
