@@ -784,25 +784,30 @@ def main():
     wl = build_head_workload(vt, dev, HEAD["d"], HEAD["K"], HEAD["B"], HEAD["topk"], HEAD["temp"], False,
                              seed=1002)
     first_touch(vt, wl)                          # set-up: every weight copy and every h has been used once
-    run_head_steps(vt, wl, args.warmup)
-    torch.cuda.synchronize()
+
+    def bracketed(n, start):
+        """n steps between two events on the launching stream.  The region opens on the device behind an
+        untimed delay kernel (about 0.1 ms of torch's spin kernel): the host has queued the first steps by
+        then, so what the events bracket is n steps of device time and not the host's latency in launching
+        the first of them into an idle GPU."""
+        e0, e1 = _events()
+        torch.cuda._sleep(200_000)
+        e0.record()
+        run_head_steps(vt, wl, n, start=start)
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1)
+
+    bracketed(args.warmup, 0)                    # the W warm-up steps take the same path as the timed ones
     if dist:
         dist.barrier()
     launches0 = vt.launch_count()
     torch.cuda.synchronize()
-    e0, e1 = _events()
-    # The timed region opens on the device behind an untimed delay kernel (about 0.1 ms of torch's spin kernel):
-    # the host has queued the first steps by then, so what the events bracket is K steps of device time and not
-    # the host's latency in launching the first of them into an idle GPU.
-    torch.cuda._sleep(200_000)
-    e0.record()
-    run_head_steps(vt, wl, args.steps, start=args.warmup)
-    e1.record()
-    torch.cuda.synchronize()
+    elapsed_ms = bracketed(args.steps, args.warmup)
     launches = vt.launch_count() - launches0
     if dist:
         dist.barrier()
-    ms_step = max_over_ranks(e0.elapsed_time(e1), dist, dev) / args.steps
+    ms_step = max_over_ranks(elapsed_ms, dist, dev) / args.steps
     # clocks: sampled while the same steps repeat for a few dozen milliseconds (the timed region above can
     # be shorter than one sampling period)
     clocks = clocks_under(lambda i: run_head_steps(vt, wl, 1, start=i), local)
