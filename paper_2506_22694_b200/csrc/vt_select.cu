@@ -31,6 +31,7 @@ constexpr int kCountCap = 2048;                  // largest bucket ranked by cou
 constexpr uint32_t kWorkCap = 6u << 10;          // key comparisons one CTA spends on that at most, in units of 1024 (~6 K per thread)
 constexpr size_t kSelectSmem = sizeof(uint32_t) * 4 * kFine + sizeof(unsigned long long) * kSortCap;
 constexpr size_t kSelectCutSmem = kSelectSmem + sizeof(uint32_t) * 2 * kFine;   // + the buckets' token mass in two 16-bit halves
+constexpr int kKeyCost = 64;                     // comparisons a key is counted as, besides those with its bucket's keys
 constexpr int kKeysPerThread = kSortCap / kThreads;   // keys of a CTA's run per thread at most
 static_assert(sizeof(uint32_t) * 4 * kFine >= sizeof(uint32_t) * kWarps * kDigits, "the full ranking reuses the bucket arrays");
 
@@ -373,12 +374,36 @@ k_select_sort(const uint32_t* counts, int32_t V, int32_t K, int32_t* map, int32_
                      reinterpret_cast<uint32_t (*)[kDigits]>(s_dyn), &spec);
         return;
     }
+    // Who ranks what: contiguous runs of whole buckets with equal COST, not equal key counts -- a key's place costs
+    // one comparison per key of its bucket, so the wide buckets of small counts near the cut dominate (dealt by
+    // keys, one CTA ranked for 22 us while another was done in 5).  cost(bucket) = size * (size + kKeyCost); the
+    // linear term stands for the per-key work and keeps a run of tiny buckets from outgrowing shared memory.
+    uint32_t cost[BPT], csum = 0;
+#pragma unroll
+    for (int q = 0; q < BPT; ++q) {
+        const int b = threadIdx.x * BPT + q;
+        const uint32_t sz = (b <= cut) ? tot[q] : 0u;
+        cost[q] = sz * (min(sz, (uint32_t)kCountCap) + (uint32_t)kKeyCost);     // (<= 64 K keys in all: the sum fits 32 bits)
+        csum += cost[q];
+    }
+    uint32_t cincl = csum;
+    for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t y = __shfl_up_sync(0xffffffffu, cincl, o);
+        if (lane >= o) cincl += y;
+    }
+    if (lane == 31) s_warp[warp] = cincl;                // (the scan above was read before the last barrier)
+    __syncthreads();
+    uint32_t cstart = cincl - csum, ctotal = 0;
+    for (int w = 0; w < kWarps; ++w) {
+        if (w < warp) cstart += s_warp[w];
+        ctotal += s_warp[w];
+    }
 #pragma unroll
     for (int q = 0; q < BPT; ++q) {
         const int b = threadIdx.x * BPT + q;
         if (b <= cut && tot[q] > 0) {
             const uint32_t st = s_gstart[b];
-            const unsigned owner = min((unsigned)kCluster - 1u, (unsigned)(((unsigned long long)st * kCluster) / T));
+            const unsigned owner = min((unsigned)kCluster - 1u, (unsigned)(((unsigned long long)cstart * kCluster) / max(ctotal, 1u)));
             atomicAdd(&s_load[owner], tot[q]);
             if (tot[q] > (uint32_t)kCountCap) s_big = 1;
             else atomicAdd(&s_work[owner], (tot[q] * tot[q] + 1023u) >> 10);
@@ -388,6 +413,7 @@ k_select_sort(const uint32_t* counts, int32_t V, int32_t K, int32_t* map, int32_
             }
             if (b == cut) s_cut_owner = (int)owner;
         }
+        cstart += cost[q];
     }
     __syncthreads();
     bool fits = s_big == 0;
