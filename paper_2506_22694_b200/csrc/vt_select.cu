@@ -287,42 +287,62 @@ k_select_sort(const uint32_t* counts, int32_t V, int32_t K, int32_t* map, int32_
     // buckets), the bucket of the K-th key, who ranks what
     constexpr int BPT = kFine / kThreads;
     static_assert(BPT == 4, "one 128-bit load per peer and thread");
-    uint32_t tot[BPT], mine_before[BPT], sum = 0;
+    // The eight CTAs' counts meet in two steps, so that 48 KB instead of 128 KB cross between the SMs per CTA: CTA r
+    // adds up the buckets [r * kSlice, (r + 1) * kSlice) of all eight (and, per peer, what the peers before it hold),
+    // leaves the sums in its own shared memory (the key buffer is idle until the ranking), and after one more cluster
+    // barrier every CTA reads the totals and its own row of the prefix table from the bucket's summing CTA.
+    constexpr int kSlice = kFine / kCluster;                         // buckets summed by one CTA
+    uint32_t* s_tot = reinterpret_cast<uint32_t*>(s_run);            // [kSlice] totals of this CTA's slice
+    uint32_t* s_pre = s_tot + kSlice;                                // [kCluster][kSlice] counts held by the peers before peer c
+    unsigned long long* s_mtot = reinterpret_cast<unsigned long long*>(s_pre + kCluster * kSlice);   // [kSlice] token mass (MODE 1)
+    if (threadIdx.x < kSlice / BPT) {
+        const int i4 = (int)rank * (kSlice / BPT) + (int)threadIdx.x;   // which 128-bit group of the bucket arrays
+        uint4 pv[kCluster];
 #pragma unroll
-    for (int q = 0; q < BPT; ++q) { tot[q] = 0; mine_before[q] = 0; }
-    uint4 pv[kCluster];
-#pragma unroll
-    for (unsigned c = 0; c < kCluster; ++c)                         // all eight remote loads in flight
-        pv[c] = reinterpret_cast<const uint4*>(cluster.map_shared_rank(s_hist, c))[threadIdx.x];
-#pragma unroll
-    for (unsigned c = 0; c < kCluster; ++c) {
-        const uint32_t t4[BPT] = {pv[c].x, pv[c].y, pv[c].z, pv[c].w};
-#pragma unroll
-        for (int q = 0; q < BPT; ++q) {
-            if (c < rank) mine_before[q] += t4[q];
-            tot[q] += t4[q];
-        }
-    }
-#pragma unroll
-    for (int q = 0; q < BPT; ++q) sum += tot[q];
-    unsigned long long mass[BPT], msum = 0;
-#pragma unroll
-    for (int q = 0; q < BPT; ++q) mass[q] = 0;
-    if (MODE == 1) {
+        for (unsigned c = 0; c < kCluster; ++c)                     // all eight remote loads in flight
+            pv[c] = reinterpret_cast<const uint4*>(cluster.map_shared_rank(s_hist, c))[i4];
+        uint4 run = make_uint4(0, 0, 0, 0);
 #pragma unroll
         for (unsigned c = 0; c < kCluster; ++c) {
-            const uint4 lo4 = reinterpret_cast<const uint4*>(cluster.map_shared_rank(s_mlo, c))[threadIdx.x];
-            const uint4 hi4 = reinterpret_cast<const uint4*>(cluster.map_shared_rank(s_mhi, c))[threadIdx.x];
-            mass[0] += (unsigned long long)lo4.x + ((unsigned long long)hi4.x << 16);
-            mass[1] += (unsigned long long)lo4.y + ((unsigned long long)hi4.y << 16);
-            mass[2] += (unsigned long long)lo4.z + ((unsigned long long)hi4.z << 16);
-            mass[3] += (unsigned long long)lo4.w + ((unsigned long long)hi4.w << 16);
+            reinterpret_cast<uint4*>(s_pre + c * kSlice)[threadIdx.x] = run;
+            run.x += pv[c].x; run.y += pv[c].y; run.z += pv[c].z; run.w += pv[c].w;
         }
+        reinterpret_cast<uint4*>(s_tot)[threadIdx.x] = run;
+        if (MODE == 1) {
+            unsigned long long m4[BPT] = {0, 0, 0, 0};
 #pragma unroll
-        for (int q = 0; q < BPT; ++q) {
-            const uint32_t value = (uint32_t)(kFine - 1 - (threadIdx.x * BPT + q));      // the bucket's count when under 256
-            if (value < 256u) mass[q] = (unsigned long long)value * tot[q];
-            msum += mass[q];
+            for (unsigned c = 0; c < kCluster; ++c) {
+                const uint4 lo4 = reinterpret_cast<const uint4*>(cluster.map_shared_rank(s_mlo, c))[i4];
+                const uint4 hi4 = reinterpret_cast<const uint4*>(cluster.map_shared_rank(s_mhi, c))[i4];
+                m4[0] += (unsigned long long)lo4.x + ((unsigned long long)hi4.x << 16);
+                m4[1] += (unsigned long long)lo4.y + ((unsigned long long)hi4.y << 16);
+                m4[2] += (unsigned long long)lo4.z + ((unsigned long long)hi4.z << 16);
+                m4[3] += (unsigned long long)lo4.w + ((unsigned long long)hi4.w << 16);
+            }
+#pragma unroll
+            for (int q = 0; q < BPT; ++q) s_mtot[threadIdx.x * BPT + q] = m4[q];
+        }
+    }
+    cluster.sync();
+    uint32_t tot[BPT], mine_before[BPT], sum = 0;
+    unsigned long long mass[BPT], msum = 0;
+    {
+        const unsigned summer = threadIdx.x / (kSlice / BPT);        // the CTA that summed this thread's buckets
+        const int i4 = (int)threadIdx.x % (kSlice / BPT);
+        const uint4 t4 = reinterpret_cast<const uint4*>(cluster.map_shared_rank(s_tot, summer))[i4];
+        const uint4 p4 = reinterpret_cast<const uint4*>(cluster.map_shared_rank(s_pre, summer) + rank * kSlice)[i4];
+        tot[0] = t4.x; tot[1] = t4.y; tot[2] = t4.z; tot[3] = t4.w;
+        mine_before[0] = p4.x; mine_before[1] = p4.y; mine_before[2] = p4.z; mine_before[3] = p4.w;
+#pragma unroll
+        for (int q = 0; q < BPT; ++q) { sum += tot[q]; mass[q] = 0; }
+        if (MODE == 1) {
+            const unsigned long long* mp = cluster.map_shared_rank(s_mtot, summer) + i4 * BPT;
+#pragma unroll
+            for (int q = 0; q < BPT; ++q) {
+                const uint32_t value = (uint32_t)(kFine - 1 - (threadIdx.x * BPT + q));      // the bucket's count when under 256
+                mass[q] = value < 256u ? (unsigned long long)value * tot[q] : mp[q];
+                msum += mass[q];
+            }
         }
     }
     unsigned long long mincl = msum;
