@@ -26,10 +26,12 @@ constexpr int kThreads = 1024;
 constexpr int kWarps = kThreads / 32;
 constexpr int kDigits = 256;
 constexpr int kFine = 4096;                      // buckets of the selection pass (3328 in use)
-constexpr int kSortCap = 16384;                  // 64-bit keys one CTA ranks in shared memory
+constexpr int kSortCap = 12288;                  // 64-bit keys one CTA ranks in shared memory
+constexpr int kExact = 256;                      // counts below this have a bucket to themselves (fine_bucket: leading one + 7 bits)
+constexpr int kFirstExact = kFine - kExact;      // ... the buckets kFirstExact .. kFine-1 in descending order
 constexpr int kCountCap = 2048;                  // largest bucket ranked by counting its greater keys
 constexpr uint32_t kWorkCap = 6u << 10;          // key comparisons one CTA spends on that at most, in units of 1024 (~6 K per thread)
-constexpr size_t kSelectSmem = sizeof(uint32_t) * 4 * kFine + sizeof(unsigned long long) * kSortCap;
+constexpr size_t kSelectSmem = sizeof(uint32_t) * 4 * kFine + sizeof(unsigned long long) * kSortCap + sizeof(uint32_t) * (1024 / 32) * kExact;
 constexpr size_t kSelectCutSmem = kSelectSmem + sizeof(uint32_t) * 2 * kFine;   // + the buckets' token mass in two 16-bit halves
 constexpr int kKeyCost = 64;                     // comparisons a key is counted as, besides those with its bucket's keys
 constexpr int kKeysPerThread = kSortCap / kThreads;   // keys of a CTA's run per thread at most
@@ -221,6 +223,13 @@ __device__ __forceinline__ uint32_t fine_bucket(uint32_t c) {
 // bucket is too large to rank by counting (counts that all fall into one bucket), the full ranking
 // above takes over.
 //
+// Counts under kExact are the exception to all of that.  Their buckets hold one value each, so inside them the
+// order is the order of the ids -- and they are the large ones (thousands of ids that were seen once or twice in a
+// small calibration corpus).  Such an id gets its final rank when it is first placed: start of the bucket + ids of the
+// bucket in the CTAs before this one + ids of the bucket in the warps before this one (per-warp counts from the
+// counting pass, warps walk contiguous pieces of the CTA's slice) + its place among the warp's 32 ids (match.any).
+// It is emitted on the spot and never enters the key buffer, whatever the size of its bucket.
+//
 // MODE 1 / 2 (the Method section's Top-P and minimum-frequency rules): K is not given but found on the way.
 // The bucket pass also sums the token mass of every bucket (Top-P), the cut bucket is the one in which the
 // prefix mass reaches ceil(p * total) / the one min_count falls into, everything down to the end of that
@@ -241,46 +250,61 @@ k_select_sort(const uint32_t* counts, int32_t V, int32_t K, int32_t* map, int32_
     uint32_t* s_gsize = s_gstart + kFine;                              // [kFine] its size over all CTAs
     uint32_t* s_next = s_gsize + kFine;                                // [kFine] scratch position of this CTA's next key
     unsigned long long* s_run = reinterpret_cast<unsigned long long*>(s_next + kFine);     // [kSortCap]
-    uint32_t* s_mlo = reinterpret_cast<uint32_t*>(s_run + kSortCap);   // [kFine] MODE 1: sum of the counts' low 16 bits (read by the peers)
+    uint32_t (*s_ws)[kExact] = reinterpret_cast<uint32_t (*)[kExact]>(s_run + kSortCap);   // [kWarps][kExact] ids of a warp's piece per exact count
+    uint32_t* s_mlo = reinterpret_cast<uint32_t*>(&s_ws[kWarps][0]);   // [kFine] MODE 1: sum of the counts' low 16 bits (read by the peers)
     uint32_t* s_mhi = s_mlo + kFine;                                   // [kFine]         and of their high 16 bits
     __shared__ uint32_t s_warp[kWarps + 1];
     __shared__ unsigned long long s_wmass[kWarps + 1];
     __shared__ unsigned long long s_mass_before;    // token mass of the buckets above the cut
-    __shared__ int s_cut_owner, s_K;
+    __shared__ int s_cut_owner, s_K, s_first;
     __shared__ uint32_t s_load[kCluster];          // keys each CTA would have to rank
     __shared__ uint32_t s_work[kCluster];          // key comparisons that would take: sum of squared bucket sizes, in units of 1024
     __shared__ uint32_t s_T;
     __shared__ int s_cut, s_lo, s_hi, s_big;
 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    // ids of this CTA: a contiguous slice walked with coalesced loads, eight in flight per thread
+    // ids of this CTA: a contiguous slice; every warp walks a contiguous piece of it in id order (128 bytes per
+    // load instruction), eight loads in flight per lane
     const int slice = (V + kCluster - 1) / kCluster;
     const int i0 = min(V, (int)rank * slice), i1 = min(V, i0 + slice);
     constexpr int kInFlight = 8;
+    const int piece = (((slice + kWarps - 1) / kWarps) + 31) & ~31;
+    const int w0 = min(i1, i0 + warp * piece), w1 = min(i1, w0 + piece);
     unsigned long long* pairs = reinterpret_cast<unsigned long long*>(keyA);       // [V] 64-bit keys (keyA and valA are adjacent)
 
     for (int i = threadIdx.x; i < kFine; i += kThreads) {
         s_hist[i] = 0;
         if (MODE == 1) { s_mlo[i] = 0; s_mhi[i] = 0; }
     }
+    for (int i = threadIdx.x; i < kWarps * kExact; i += kThreads) (&s_ws[0][0])[i] = 0;
     if (threadIdx.x < kCluster) { s_load[threadIdx.x] = 0; s_work[threadIdx.x] = 0u; }
-    if (threadIdx.x == 0) { s_cut = -1; s_lo = 0x7fffffff; s_hi = 0; s_big = 0; s_cut_owner = -1; s_K = 0; s_T = 0; s_mass_before = 0; }
+    if (threadIdx.x == 0) { s_cut = -1; s_lo = 0x7fffffff; s_hi = 0; s_big = 0; s_cut_owner = -1; s_K = 0; s_first = 0; s_T = 0; s_mass_before = 0; }
     __syncthreads();
-    // phase 1: bucket counts (descending order: inverted bucket index)
-    for (int i = i0 + (int)threadIdx.x; i < i1; i += kThreads * kInFlight) {
+    // phase 1: bucket counts (descending order: inverted bucket index), and per warp the ids of every exact count
+    for (int i = w0 + lane; i < w1; i += 32 * kInFlight) {
         uint32_t c[kInFlight];
 #pragma unroll
-        for (int q = 0; q < kInFlight; ++q) c[q] = i + q * kThreads < i1 ? __ldg(counts + i + q * kThreads) : 0u;
+        for (int q = 0; q < kInFlight; ++q) c[q] = i + q * 32 < w1 ? __ldg(counts + i + q * 32) : 0u;
 #pragma unroll
         for (int q = 0; q < kInFlight; ++q)
-            if (i + q * kThreads < i1) {
+            if (i + q * 32 < w1) {
                 const uint32_t b = kFine - 1 - fine_bucket(c[q]);
                 atomicAdd(&s_hist[b], 1u);
-                if (MODE == 1 && c[q] >= 256u) {   // (a bucket under 256 holds one value: its mass is a product)
+                if (c[q] < (uint32_t)kExact) atomicAdd(&s_ws[warp][c[q]], 1u);
+                if (MODE == 1 && c[q] >= (uint32_t)kExact) {   // (an exact bucket's mass is a product)
                     atomicAdd(&s_mlo[b], c[q] & 0xffffu);   // at most 2^14 ids per CTA: neither half can overflow 32 bits
                     atomicAdd(&s_mhi[b], c[q] >> 16);
                 }
             }
+    }
+    __syncthreads();
+    if (threadIdx.x < kExact) {                         // exclusive prefix over the warps, per exact count
+        uint32_t run = 0;
+        for (int w = 0; w < kWarps; ++w) {
+            const uint32_t t = s_ws[w][threadIdx.x];
+            s_ws[w][threadIdx.x] = run;
+            run += t;
+        }
     }
     cluster.sync();
     // phase 2: start of every bucket in descending order (each thread owns kFine / kThreads neighbouring
@@ -380,14 +404,24 @@ k_select_sort(const uint32_t* counts, int32_t V, int32_t K, int32_t* map, int32_
         if (MODE == 0) is_cut = start < (uint32_t)K && start + tot[q] >= (uint32_t)K;                   // exactly one bucket
         else if (MODE == 1) is_cut = (double)mstart < target && (double)(mstart + mass[q]) >= target;  // exactly one, if any token was counted
         else is_cut = b == min_bucket;
-        if (is_cut) { s_cut = b; s_T = start + tot[q]; s_mass_before = mstart; s_K = (int)start; }
+        if (is_cut) {
+            s_cut = b; s_T = start + tot[q]; s_mass_before = mstart; s_K = (int)start; s_first = (int)start;
+            if (MODE != 0 && b >= kFirstExact) {        // an exact bucket: K follows by arithmetic, here and now
+                const uint32_t value = (uint32_t)(kFine - 1 - b);
+                uint32_t kk;
+                if (MODE == 1) kk = start + (uint32_t)(((unsigned long long)target - mstart + value - 1) / value);
+                else kk = start + tot[q];               // (the bucket min_count falls into holds exactly min_count)
+                s_K = (int)max(1u, min((uint32_t)V, kk));
+                if (rank == 0) *k_out = s_K;
+            }
+        }
         start += tot[q];
         mstart += mass[q];
     }
     __syncthreads();
     const int cut = s_cut;
     const uint32_t T = s_T;                             // keys to be ranked = end of the cut bucket
-    CutSpec spec{MODE, cut >= 0 && T > 0, (uint32_t)s_K, T, s_mass_before, target, min_count, k_out};
+    CutSpec spec{MODE, cut >= 0 && T > 0, (uint32_t)s_first, T, s_mass_before, target, min_count, k_out};
     if (MODE != 0 && !spec.valid) {                     // no tokens at all / nothing as frequent as asked: K = 1 of the full ranking
         cluster.sync();                                 // peers are done reading this CTA's counts
         lsd_rank_all(cluster, counts, V, V, map, inv_map, keyA, valA, keyB, valB,
@@ -402,7 +436,7 @@ k_select_sort(const uint32_t* counts, int32_t V, int32_t K, int32_t* map, int32_
 #pragma unroll
     for (int q = 0; q < BPT; ++q) {
         const int b = threadIdx.x * BPT + q;
-        const uint32_t sz = (b <= cut) ? tot[q] : 0u;
+        const uint32_t sz = (b <= cut && b < kFirstExact) ? tot[q] : 0u;    // (ids of exact buckets are placed directly)
         cost[q] = sz * (min(sz, (uint32_t)kCountCap) + (uint32_t)kKeyCost);     // (<= 64 K keys in all: the sum fits 32 bits)
         csum += cost[q];
     }
@@ -421,7 +455,7 @@ k_select_sort(const uint32_t* counts, int32_t V, int32_t K, int32_t* map, int32_
 #pragma unroll
     for (int q = 0; q < BPT; ++q) {
         const int b = threadIdx.x * BPT + q;
-        if (b <= cut && tot[q] > 0) {
+        if (b <= cut && b < kFirstExact && tot[q] > 0) {
             const uint32_t st = s_gstart[b];
             const unsigned owner = min((unsigned)kCluster - 1u, (unsigned)(((unsigned long long)cstart * kCluster) / max(ctotal, 1u)));
             atomicAdd(&s_load[owner], tot[q]);
@@ -449,19 +483,40 @@ k_select_sort(const uint32_t* counts, int32_t V, int32_t K, int32_t* map, int32_
                      reinterpret_cast<uint32_t (*)[kDigits]>(s_dyn));
         return;
     }
-    // phase 3: move the keys of the buckets down to the cut into bucket order; order inside a bucket is
-    // whatever the atomics make of it; ids below the cut are pruned here
-    for (int i = i0 + (int)threadIdx.x; i < i1; i += kThreads * kInFlight) {
+    // phase 3: the keys of the inexact buckets down to the cut move into bucket order (order inside a bucket is
+    // whatever the atomics make of it); ids of exact buckets down to the cut take their final rank; ids below the
+    // cut are pruned here
+    const int k_exact = MODE == 0 ? K : s_K;            // (MODE 1 / 2: exact ids are kept only when the cut bucket is exact)
+    for (int i = w0 + lane; i < w1 + lane; i += 32 * kInFlight) {      // (every lane of the warp makes every trip)
         uint32_t c[kInFlight];
 #pragma unroll
-        for (int q = 0; q < kInFlight; ++q) c[q] = i + q * kThreads < i1 ? __ldg(counts + i + q * kThreads) : 0u;
+        for (int q = 0; q < kInFlight; ++q) c[q] = i + q * 32 < w1 ? __ldg(counts + i + q * 32) : 0u;
 #pragma unroll
         for (int q = 0; q < kInFlight; ++q) {
-            const int id = i + q * kThreads;
-            if (id >= i1) continue;
+            const int id = i + q * 32;
+            const bool on = id < w1;
             const int b = (int)(kFine - 1 - fine_bucket(c[q]));
-            if (b <= cut) pairs[atomicAdd(&s_next[b], 1u)] = ((unsigned long long)c[q] << 32) | (0xffffffffu - (uint32_t)id);
-            else inv_map[id] = -1;
+            const bool kept = on && b <= cut;
+            const bool exact = kept && b >= kFirstExact;
+            const unsigned group = __ballot_sync(0xffffffffu, exact);
+            if (exact) {
+                const unsigned peers = __match_any_sync(group, c[q]);
+                const int leader = __ffs(peers) - 1;
+                uint32_t before = 0;
+                if (lane == leader) {
+                    before = s_ws[warp][c[q]];
+                    s_ws[warp][c[q]] = before + __popc(peers);
+                }
+                before = __shfl_sync(peers, before, leader);
+                const int rk = (int)(s_next[b] + before + __popc(peers & lanemask_lt()));
+                if (rk < k_exact) map[rk] = id;
+                inv_map[id] = rk < k_exact ? rk : -1;
+            } else if (kept) {
+                pairs[atomicAdd(&s_next[b], 1u)] = ((unsigned long long)c[q] << 32) | (0xffffffffu - (uint32_t)id);
+            } else if (on) {
+                inv_map[id] = -1;
+            }
+            __syncwarp();
         }
     }
     __threadfence();
