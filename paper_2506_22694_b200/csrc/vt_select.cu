@@ -33,8 +33,8 @@ constexpr int kCountCap = 2048;                  // largest bucket ranked by cou
 constexpr uint32_t kWorkCap = 6u << 10;          // key comparisons one CTA spends on that at most, in units of 1024 (~6 K per thread)
 constexpr size_t kSelectSmem = sizeof(uint32_t) * 4 * kFine + sizeof(unsigned long long) * kSortCap + sizeof(uint32_t) * (1024 / 32) * kExact;
 constexpr size_t kSelectCutSmem = kSelectSmem + sizeof(uint32_t) * 2 * kFine;   // + the buckets' token mass in two 16-bit halves
-constexpr int kKeyCost = 64;                     // comparisons a key is counted as, besides those with its bucket's keys
-constexpr int kKeysPerThread = kSortCap / kThreads;   // keys of a CTA's run per thread at most
+constexpr int kDeals = 2;                        // ways of dealing the buckets to the CTAs that are tried
+constexpr uint32_t kKeyCost0 = 64, kKeyCost1 = 1024;   // comparisons a key is counted as, besides those with its bucket's keys, in each
 static_assert(sizeof(uint32_t) * 4 * kFine >= sizeof(uint32_t) * kWarps * kDigits, "the full ranking reuses the bucket arrays");
 
 // What the full ranking needs to find K itself (Top-P / minimum frequency): the cut bucket's ranks
@@ -204,6 +204,61 @@ __device__ void lsd_rank_all(cg::cluster_group& cluster, const uint32_t* counts,
     }
 }
 
+// The keys of one bucket of counts >= 256 agree in the count's leading one and the seven bits behind it; what
+// orders them is the rest of the count and then ~id.  Where that fits 32 bits (lb low bits of the count + the
+// bits of an id) it is the short key compared in shared memory; a bucket where it does not fit (counts from 2^23
+// with a 17-bit id) is called wide and compares its 64-bit keys where they lie in global memory -- the deal
+// hands such a bucket to the ranking only while it is tiny.
+__device__ __forceinline__ int id_bits(int32_t V) { return 32 - __clz(max(V - 1, 1)); }          // 1 .. 31
+__device__ __forceinline__ int low_bits(uint32_t cnt) { return 24 - __clz(cnt); }                // cnt >= 256: 1 .. 24
+__device__ __forceinline__ uint32_t short_key(unsigned long long key, int idbits) {
+    const uint32_t cnt = (uint32_t)(key >> 32);
+    const int lb = low_bits(cnt);
+    if (lb + idbits > 32) return 0u;
+    return ((cnt & ((1u << lb) - 1u)) << idbits) | ((uint32_t)key & ((1u << idbits) - 1u));       // (~id in idbits bits)
+}
+constexpr uint32_t kWideCap = 32;                // ids a wide bucket may hold and still be ranked by counting
+
+// Number of keys of the bucket [bs, be) of the CTA's run that are greater than key (and, MASS, the sum of their counts).
+template <bool MASS>
+__device__ __forceinline__ int rank_in_bucket(const uint32_t* s_c, const unsigned long long* run, unsigned long long key, int bs, int be,
+                                              int idbits, unsigned long long* mass) {
+    const uint32_t cnt = (uint32_t)(key >> 32);
+    const int lb = low_bits(cnt);
+    int r = 0;
+    if (lb + idbits > 32) {                          // wide bucket
+        unsigned long long m = 0;
+        for (int i = bs; i < be; ++i) {
+            const unsigned long long o = __ldcg(run + i);
+            const bool gt = o > key;
+            r += gt ? 1 : 0;
+            if (MASS) m += gt ? (o >> 32) : 0ull;
+        }
+        if (MASS) *mass = m;
+        return r;
+    }
+    const uint32_t ck = short_key(key, idbits);
+    if (MASS) {
+        unsigned long long m = 0;                    // of the counts' low bits
+        for (int i = bs; i < be; ++i) {
+            const uint32_t o = s_c[i];
+            const bool gt = o > ck;
+            r += gt ? 1 : 0;
+            m += gt ? (unsigned long long)(o >> idbits) : 0ull;
+        }
+        *mass = (unsigned long long)r * (cnt & ~((1u << lb) - 1u)) + m;
+        return r;
+    }
+    int i = bs;
+    for (; i < be && (i & 3); ++i) r += s_c[i] > ck ? 1 : 0;
+    for (; i + 4 <= be; i += 4) {
+        const uint4 o = *reinterpret_cast<const uint4*>(s_c + i);
+        r += (o.x > ck ? 1 : 0) + (o.y > ck ? 1 : 0) + (o.z > ck ? 1 : 0) + (o.w > ck ? 1 : 0);
+    }
+    for (; i < be; ++i) r += s_c[i] > ck ? 1 : 0;
+    return r;
+}
+
 // Order-preserving bucket of a count: its leading one and the seven bits behind it (counts below 128 map to
 // themselves).  3328 buckets whose widths grow with the count, so a heavy-tailed histogram spreads over
 // many of them and a bucket near the cut holds a few hundred ids at most.
@@ -216,12 +271,12 @@ __device__ __forceinline__ uint32_t fine_bucket(uint32_t c) {
 // Radix select (Eq. 1, Top-K(c,k)): one pass of bucket counts finds the bucket that holds the K-th key;
 // only the keys of that bucket and of the buckets above it -- K of them plus part of one bucket -- are
 // moved, bucket by bucket, into a scratch array, which is thereby already in bucket order.  Each CTA of
-// the cluster then takes a contiguous run of whole buckets into shared memory and gives every key its
-// place inside its bucket by counting the bucket's greater keys (64-bit keys (count, ~id): unique, so
-// the result is the one right answer; buckets are small, so the counting is cheap).  Everything below
-// the cut is never touched again.  When a run does not fit a CTA's shared memory (K close to V) or a
-// bucket is too large to rank by counting (counts that all fall into one bucket), the full ranking
-// above takes over.
+// the cluster then takes a contiguous run of whole buckets and gives every key its place inside its
+// bucket by counting the bucket's greater keys (keys (count, ~id) are unique, so the result is the one
+// right answer; buckets are small, so the counting is cheap; what is compared is the 32-bit short key
+// above, held in shared memory).  Everything below the cut is never touched again.  When no deal of the
+// buckets fits the CTAs' shared memory (K close to V on counts that are mostly above 255) or a bucket is
+// too large to rank by counting (counts that all fall into one bucket), the full ranking above takes over.
 //
 // Counts under kExact are the exception to all of that.  Their buckets hold one value each, so inside them the
 // order is the order of the ids -- and they are the large ones (thousands of ids that were seen once or twice in a
@@ -249,18 +304,18 @@ k_select_sort(const uint32_t* counts, int32_t V, int32_t K, int32_t* map, int32_
     uint32_t* s_gstart = s_hist + kFine;                               // [kFine] start of the bucket in the ranking
     uint32_t* s_gsize = s_gstart + kFine;                              // [kFine] its size over all CTAs
     uint32_t* s_next = s_gsize + kFine;                                // [kFine] scratch position of this CTA's next key
-    unsigned long long* s_run = reinterpret_cast<unsigned long long*>(s_next + kFine);     // [kSortCap]
+    unsigned long long* s_run = reinterpret_cast<unsigned long long*>(s_next + kFine);     // [kSortCap] phase 2: the exchange; phase 4: short keys, ranks
     uint32_t (*s_ws)[kExact] = reinterpret_cast<uint32_t (*)[kExact]>(s_run + kSortCap);   // [kWarps][kExact] ids of a warp's piece per exact count
     uint32_t* s_mlo = reinterpret_cast<uint32_t*>(&s_ws[kWarps][0]);   // [kFine] MODE 1: sum of the counts' low 16 bits (read by the peers)
     uint32_t* s_mhi = s_mlo + kFine;                                   // [kFine]         and of their high 16 bits
     __shared__ uint32_t s_warp[kWarps + 1];
     __shared__ unsigned long long s_wmass[kWarps + 1];
     __shared__ unsigned long long s_mass_before;    // token mass of the buckets above the cut
-    __shared__ int s_cut_owner, s_K, s_first;
-    __shared__ uint32_t s_load[kCluster];          // keys each CTA would have to rank
-    __shared__ uint32_t s_work[kCluster];          // key comparisons that would take: sum of squared bucket sizes, in units of 1024
+    __shared__ int s_cut_owner[kDeals], s_K, s_first;
+    __shared__ uint32_t s_load[kDeals][kCluster];  // keys each CTA would have to rank, per way of dealing the buckets
+    __shared__ uint32_t s_work[kDeals][kCluster];  // key comparisons that would take: sum of squared bucket sizes, in units of 1024
     __shared__ uint32_t s_T;
-    __shared__ int s_cut, s_lo, s_hi, s_big;
+    __shared__ int s_cut, s_lo[kDeals], s_hi[kDeals], s_big;
 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     // ids of this CTA: a contiguous slice; every warp walks a contiguous piece of it in id order (128 bytes per
@@ -277,8 +332,9 @@ k_select_sort(const uint32_t* counts, int32_t V, int32_t K, int32_t* map, int32_
         if (MODE == 1) { s_mlo[i] = 0; s_mhi[i] = 0; }
     }
     for (int i = threadIdx.x; i < kWarps * kExact; i += kThreads) (&s_ws[0][0])[i] = 0;
-    if (threadIdx.x < kCluster) { s_load[threadIdx.x] = 0; s_work[threadIdx.x] = 0u; }
-    if (threadIdx.x == 0) { s_cut = -1; s_lo = 0x7fffffff; s_hi = 0; s_big = 0; s_cut_owner = -1; s_K = 0; s_first = 0; s_T = 0; s_mass_before = 0; }
+    if (threadIdx.x < kDeals * kCluster) { (&s_load[0][0])[threadIdx.x] = 0; (&s_work[0][0])[threadIdx.x] = 0u; }
+    if (threadIdx.x < kDeals) { s_lo[threadIdx.x] = 0x7fffffff; s_hi[threadIdx.x] = 0; s_cut_owner[threadIdx.x] = -1; }
+    if (threadIdx.x == 0) { s_cut = -1; s_big = 0; s_K = 0; s_first = 0; s_T = 0; s_mass_before = 0; }
     __syncthreads();
     // phase 1: bucket counts (descending order: inverted bucket index), and per warp the ids of every exact count
     for (int i = w0 + lane; i < w1; i += 32 * kInFlight) {
@@ -430,48 +486,58 @@ k_select_sort(const uint32_t* counts, int32_t V, int32_t K, int32_t* map, int32_
     }
     // Who ranks what: contiguous runs of whole buckets with equal COST, not equal key counts -- a key's place costs
     // one comparison per key of its bucket, so the wide buckets of small counts near the cut dominate (dealt by
-    // keys, one CTA ranked for 22 us while another was done in 5).  cost(bucket) = size * (size + kKeyCost); the
+    // keys, one CTA ranked for 22 us while another was done in 5).  cost(bucket) = size * (size + key cost); the
     // linear term stands for the per-key work and keeps a run of tiny buckets from outgrowing shared memory.
-    uint32_t cost[BPT], csum = 0;
+    // Two deals are tried and the first that fits is taken: the second, with a higher key cost and so closer to
+    // equal key counts, is for rankings of 50 K keys and more, where the first one's leading CTA would get more
+    // tiny buckets than its shared memory holds.
+    int deal = -1;
+    for (int d = 0; d < kDeals && deal < 0; ++d) {      // (the same trips in every thread of every CTA: same inputs)
+        const uint32_t kc = d == 0 ? kKeyCost0 : kKeyCost1;
+        uint32_t cost[BPT], csum = 0;
 #pragma unroll
-    for (int q = 0; q < BPT; ++q) {
-        const int b = threadIdx.x * BPT + q;
-        const uint32_t sz = (b <= cut && b < kFirstExact) ? tot[q] : 0u;    // (ids of exact buckets are placed directly)
-        cost[q] = sz * (min(sz, (uint32_t)kCountCap) + (uint32_t)kKeyCost);     // (<= 64 K keys in all: the sum fits 32 bits)
-        csum += cost[q];
-    }
-    uint32_t cincl = csum;
-    for (int o = 1; o < 32; o <<= 1) {
-        const uint32_t y = __shfl_up_sync(0xffffffffu, cincl, o);
-        if (lane >= o) cincl += y;
-    }
-    if (lane == 31) s_warp[warp] = cincl;                // (the scan above was read before the last barrier)
-    __syncthreads();
-    uint32_t cstart = cincl - csum, ctotal = 0;
-    for (int w = 0; w < kWarps; ++w) {
-        if (w < warp) cstart += s_warp[w];
-        ctotal += s_warp[w];
-    }
-#pragma unroll
-    for (int q = 0; q < BPT; ++q) {
-        const int b = threadIdx.x * BPT + q;
-        if (b <= cut && b < kFirstExact && tot[q] > 0) {
-            const uint32_t st = s_gstart[b];
-            const unsigned owner = min((unsigned)kCluster - 1u, (unsigned)(((unsigned long long)cstart * kCluster) / max(ctotal, 1u)));
-            atomicAdd(&s_load[owner], tot[q]);
-            if (tot[q] > (uint32_t)kCountCap) s_big = 1;
-            else atomicAdd(&s_work[owner], (tot[q] * tot[q] + 1023u) >> 10);
-            if (owner == rank) {
-                atomicMin(&s_lo, (int)st);
-                atomicMax(&s_hi, (int)(st + tot[q]));
-            }
-            if (b == cut) s_cut_owner = (int)owner;
+        for (int q = 0; q < BPT; ++q) {
+            const int b = threadIdx.x * BPT + q;
+            const uint32_t sz = (b <= cut && b < kFirstExact) ? tot[q] : 0u;    // (ids of exact buckets are placed directly)
+            cost[q] = sz * (min(sz, (uint32_t)kCountCap) + kc);                 // (<= 128 K keys in all: the sum fits 32 bits)
+            csum += cost[q];
         }
-        cstart += cost[q];
+        uint32_t cincl = csum;
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t y = __shfl_up_sync(0xffffffffu, cincl, o);
+            if (lane >= o) cincl += y;
+        }
+        if (lane == 31) s_warp[warp] = cincl;            // (a barrier lies between this and the last reads of the array)
+        __syncthreads();
+        uint32_t cstart = cincl - csum, ctotal = 0;
+        for (int w = 0; w < kWarps; ++w) {
+            if (w < warp) cstart += s_warp[w];
+            ctotal += s_warp[w];
+        }
+#pragma unroll
+        for (int q = 0; q < BPT; ++q) {
+            const int b = threadIdx.x * BPT + q;
+            if (b <= cut && b < kFirstExact && tot[q] > 0) {
+                const uint32_t st = s_gstart[b];
+                const int lb = (kFine - 1 - b - 128) / 128;                    // low bits of the bucket's counts
+                if (tot[q] > (uint32_t)kCountCap || (lb + id_bits(V) > 32 && tot[q] > kWideCap)) s_big = 1;
+                const unsigned owner = min((unsigned)kCluster - 1u, (unsigned)(((unsigned long long)cstart * kCluster) / max(ctotal, 1u)));
+                atomicAdd(&s_load[d][owner], tot[q]);
+                if (tot[q] <= (uint32_t)kCountCap) atomicAdd(&s_work[d][owner], (tot[q] * tot[q] + 1023u) >> 10);
+                if (owner == rank) {
+                    atomicMin(&s_lo[d], (int)st);
+                    atomicMax(&s_hi[d], (int)(st + tot[q]));
+                }
+                if (b == cut) s_cut_owner[d] = (int)owner;
+            }
+            cstart += cost[q];
+        }
+        __syncthreads();
+        bool ok = s_big == 0;
+        for (int c = 0; c < kCluster; ++c) ok = ok && s_load[d][c] <= (uint32_t)kSortCap && s_work[d][c] <= kWorkCap;
+        if (ok) deal = d;
     }
-    __syncthreads();
-    bool fits = s_big == 0;
-    for (int c = 0; c < kCluster; ++c) fits = fits && s_load[c] <= (uint32_t)kSortCap && s_work[c] <= kWorkCap;
+    const bool fits = deal >= 0;
     if (!fits) {                                        // the same decision in every CTA (same inputs)
         cluster.sync();                                 // peers are done reading this CTA's counts
         if (MODE != 0) {
@@ -521,19 +587,23 @@ k_select_sort(const uint32_t* counts, int32_t V, int32_t K, int32_t* map, int32_
     }
     __threadfence();
     cluster.sync();
-    // phase 4: this CTA's run of buckets into shared memory; place of a key = start of its bucket + number
-    // of greater keys in the bucket (neighbouring lanes mostly share a bucket: the reads are broadcasts)
-    const int r0 = s_lo, n = s_hi > s_lo ? s_hi - s_lo : 0;
-    for (int j = threadIdx.x; j < n; j += kThreads) s_run[j] = __ldcg(pairs + r0 + j);
+    // phase 4: place of a key = start of its bucket + number of greater keys in the bucket.  Inside a bucket the
+    // counts differ in their low bits only, so what is compared is a 32-bit word (those low bits, then ~id) held in
+    // shared memory for the CTA's whole run of buckets, four to a load (neighbouring lanes mostly share a bucket:
+    // the reads are broadcasts).  The 64-bit keys stay where phase 3 put them and are read from there.
+    const int r0 = s_lo[deal], n = s_hi[deal] > s_lo[deal] ? s_hi[deal] - s_lo[deal] : 0;
+    const unsigned long long* run = pairs + r0;
+    uint32_t* s_c = reinterpret_cast<uint32_t*>(s_run);                 // [kSortCap]
+    uint32_t* s_place = s_c + kSortCap;                                 // [kSortCap] MODE 1 / 2: the keys' ranks
+    const int idbits = id_bits(V);
+    for (int j = threadIdx.x; j < n; j += kThreads) s_c[j] = short_key(__ldcg(run + j), idbits);
     __syncthreads();
     if (MODE == 0) {
         for (int j = threadIdx.x; j < n; j += kThreads) {
-            const unsigned long long key = s_run[j];
+            const unsigned long long key = __ldcg(run + j);
             const int b = (int)(kFine - 1 - fine_bucket((uint32_t)(key >> 32)));
             const int bs = (int)s_gstart[b] - r0, be = bs + (int)s_gsize[b];
-            int r = 0;
-            for (int i = bs; i < be; ++i) r += s_run[i] > key ? 1 : 0;
-            const int rk = r0 + bs + r;
+            const int rk = r0 + bs + rank_in_bucket<false>(s_c, run, key, bs, be, idbits, nullptr);
             const int32_t v = (int32_t)(0xffffffffu - (uint32_t)key);
             if (rk < K) map[rk] = v;
             inv_map[v] = rk < K ? rk : -1;
@@ -543,44 +613,31 @@ k_select_sort(const uint32_t* counts, int32_t V, int32_t K, int32_t* map, int32_
     // K from the ranks: first every key's place (and, inside the cut bucket, the token mass ranked before it),
     // then -- in the CTA that ranks the cut bucket -- K, then the outputs.  The other CTAs rank buckets above
     // the cut only: all of theirs is kept.
-    int place[kKeysPerThread];
-    const bool owns_cut = s_cut_owner == (int)rank || (s_cut_owner < 0 && rank == 0);   // (an empty cut bucket has no owner)
+    const bool owns_cut = s_cut_owner[deal] == (int)rank || (s_cut_owner[deal] < 0 && rank == 0);   // (an empty cut bucket has no owner)
     const unsigned long long mass_before = s_mass_before;
-#pragma unroll
-    for (int q = 0; q < kKeysPerThread; ++q) {
-        const int j = threadIdx.x + q * kThreads;
-        place[q] = -1;
-        if (j >= n) continue;
-        const unsigned long long key = s_run[j];
+    for (int j = threadIdx.x; j < n; j += kThreads) {
+        const unsigned long long key = __ldcg(run + j);
         const uint32_t cnt = (uint32_t)(key >> 32);
         const int b = (int)(kFine - 1 - fine_bucket(cnt));
         const int bs = (int)s_gstart[b] - r0, be = bs + (int)s_gsize[b];
-        int r = 0;
-        unsigned long long m = 0;
+        int r;
         if (b == cut && MODE == 1) {
-            for (int i = bs; i < be; ++i) {
-                const unsigned long long o = s_run[i];
-                const bool gt = o > key;
-                r += gt ? 1 : 0;
-                m += gt ? (o >> 32) : 0ull;
-            }
+            unsigned long long m = 0;
+            r = rank_in_bucket<true>(s_c, run, key, bs, be, idbits, &m);
             const unsigned long long cum = mass_before + m;
             if ((double)cum < target && (double)(cum + cnt) >= target) s_K = r0 + bs + r + 1;   // exactly one key
         } else {
-            for (int i = bs; i < be; ++i) r += s_run[i] > key ? 1 : 0;
+            r = rank_in_bucket<false>(s_c, run, key, bs, be, idbits, nullptr);
             if (b == cut && MODE == 2 && cnt >= min_count) atomicMax(&s_K, r0 + bs + r + 1);
         }
-        place[q] = r0 + bs + r;
+        s_place[j] = (uint32_t)(r0 + bs + r);
     }
     __syncthreads();
     const int Kf = owns_cut ? max(1, min(V, s_K)) : (int)T;
     if (owns_cut && threadIdx.x == 0) *k_out = Kf;
-#pragma unroll
-    for (int q = 0; q < kKeysPerThread; ++q) {
-        const int j = threadIdx.x + q * kThreads;
-        if (j >= n) continue;
-        const int32_t v = (int32_t)(0xffffffffu - (uint32_t)s_run[j]);
-        const int rk = place[q];
+    for (int j = threadIdx.x; j < n; j += kThreads) {
+        const int32_t v = (int32_t)(0xffffffffu - (uint32_t)__ldcg(run + j));
+        const int rk = (int)s_place[j];
         if (rk < Kf) map[rk] = v;
         inv_map[v] = rk < Kf ? rk : -1;
     }

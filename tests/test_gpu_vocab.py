@@ -294,16 +294,22 @@ def test_select_minfreq_matches_oracle(V, n, f):
     _assert_clean(ws)
 
 
-@pytest.mark.parametrize("shape", ["tiny_values", "few_wide_buckets", "spikes_over_noise", "around_256", "one_value"])
+@pytest.mark.parametrize("shape", ["tiny_values", "few_wide_buckets", "spikes_over_noise", "around_256", "one_value",
+                                   "huge_counts_few_per_bucket", "huge_counts_full_buckets"])
 def test_select_cuts_over_count_shapes_that_stress_the_buckets(shape):
     """Count vectors chosen against the bucket scheme of the selection kernel: huge buckets of equal counts, all
     counts in a handful of wide buckets, a few enormous counts over noise, counts on both sides of the value from
-    which a bucket holds more than one count, and a single value.  Top-P, minimum frequency and Top-K."""
+    which a bucket holds more than one count, a single value, and counts from 2^30.  Top-P, minimum frequency
+    and Top-K."""
     V = 50_000
     rng = np.random.default_rng(len(shape))
     c = {"tiny_values": rng.integers(0, 4, V), "few_wide_buckets": rng.integers(1 << 20, 1 << 21, V),
          "spikes_over_noise": np.where(rng.random(V) < 0.01, rng.integers(1 << 28, 1 << 31, V), rng.integers(0, 3, V)),
-         "around_256": rng.integers(250, 262, V), "one_value": np.full(V, 12345)}[shape].astype(np.uint64)
+         "around_256": rng.integers(250, 262, V), "one_value": np.full(V, 12345),
+         # counts so large that what orders a bucket's keys (the count's low bits, then the id) passes 32 bits:
+         # a dozen ids per such bucket, and hundreds
+         "huge_counts_few_per_bucket": np.where(rng.random(V) < 0.02, (1 << 30) + rng.integers(0, 1 << 30, V), rng.integers(0, 3, V)),
+         "huge_counts_full_buckets": (1 << 30) + rng.integers(0, 1 << 24, V)}[shape].astype(np.uint64)
     counts = torch.from_numpy(c.astype(np.uint32).view(np.int32)).to(DEV)
     ws = vt.Workspace(vt.workspace_bytes(vt.VT_OP_SELECT_TOPK, 0, V, V))
     for p in (1e-12, 0.3, 0.9, 1.0):
