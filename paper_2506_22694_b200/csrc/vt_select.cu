@@ -25,14 +25,18 @@ constexpr int kCluster = 8;
 constexpr int kThreads = 1024;
 constexpr int kWarps = kThreads / 32;
 constexpr int kDigits = 256;
-constexpr int kFine = 4096;                      // buckets of the selection pass (3328 in use)
+constexpr int kFine = 4096;                      // buckets of the selection pass (3968 in use)
 constexpr int kSortCap = 12288;                  // 64-bit keys one CTA ranks in shared memory
-constexpr int kExact = 256;                      // counts below this have a bucket to themselves (fine_bucket: leading one + 7 bits)
+constexpr int kExact = 1024;                     // counts below this have a bucket to themselves (fine_bucket)
+constexpr int kExactLog = 10;
 constexpr int kFirstExact = kFine - kExact;      // ... the buckets kFirstExact .. kFine-1 in descending order
+constexpr int kExactIds = 65535;                 // ids per CTA up to which such counts are ranked where they are placed (16-bit counters)
 constexpr int kCountCap = 2048;                  // largest bucket ranked by counting its greater keys
 constexpr uint32_t kWorkCap = 6u << 10;          // key comparisons one CTA spends on that at most, in units of 1024 (~6 K per thread)
-constexpr size_t kSelectSmem = sizeof(uint32_t) * 4 * kFine + sizeof(unsigned long long) * kSortCap + sizeof(uint32_t) * (1024 / 32) * kExact;
-constexpr size_t kSelectCutSmem = kSelectSmem + sizeof(uint32_t) * 2 * kFine;   // + the buckets' token mass in two 16-bit halves
+constexpr size_t kSelectSmem = sizeof(uint32_t) * 4 * kFine + sizeof(uint32_t) * 2 * kSortCap + sizeof(uint16_t) * (1024 / 32) * kExact;
+constexpr int kMassAt = 32 << 10;                // where in the key buffer the buckets' token mass lives while that buffer is idle
+static_assert(kMassAt + sizeof(unsigned long long) * kFine <= sizeof(uint32_t) * 2 * kSortCap, "the token mass fits the idle key buffer");
+static_assert(sizeof(uint32_t) * (kFine / 8) * (1 + 8) + sizeof(unsigned long long) * (kFine / 8) <= kMassAt, "... behind the exchange's sums");
 constexpr int kDeals = 2;                        // ways of dealing the buckets to the CTAs that are tried
 constexpr uint32_t kKeyCost0 = 64, kKeyCost1 = 1024;   // comparisons a key is counted as, besides those with its bucket's keys, in each
 static_assert(sizeof(uint32_t) * 4 * kFine >= sizeof(uint32_t) * kWarps * kDigits, "the full ranking reuses the bucket arrays");
@@ -162,11 +166,11 @@ __device__ void lsd_rank_all(cg::cluster_group& cluster, const uint32_t* counts,
         __syncthreads();
         if (spec->valid && warp == 0) {
             // the sorted counts of the cut bucket's ranks, 32 at a time, until the prefix reaches the target
-            // (Top-P) or the counts fall under min_count; equal counts (every bucket under 256) by division
+            // (Top-P) or the counts fall under min_count; equal counts (every bucket under kExact) by division
             const uint32_t a = spec->first, b = spec->end;
             const uint32_t c0 = src_key[a];
             int found = (int)b;                                        // (the bucket pass says the cut lies in [a, b])
-            if (spec->mode == 1 && c0 < 256u) {
+            if (spec->mode == 1 && c0 < (uint32_t)kExact) {
                 const unsigned long long rem = (unsigned long long)spec->target - spec->mass_before;
                 found = (int)(a + (uint32_t)((rem + c0 - 1) / c0));
             } else {
@@ -204,13 +208,13 @@ __device__ void lsd_rank_all(cg::cluster_group& cluster, const uint32_t* counts,
     }
 }
 
-// The keys of one bucket of counts >= 256 agree in the count's leading one and the seven bits behind it; what
+// The keys of one bucket of counts >= 1024 agree in the count's leading one and the seven bits behind it; what
 // orders them is the rest of the count and then ~id.  Where that fits 32 bits (lb low bits of the count + the
 // bits of an id) it is the short key compared in shared memory; a bucket where it does not fit (counts from 2^23
 // with a 17-bit id) is called wide and compares its 64-bit keys where they lie in global memory -- the deal
 // hands such a bucket to the ranking only while it is tiny.
 __device__ __forceinline__ int id_bits(int32_t V) { return 32 - __clz(max(V - 1, 1)); }          // 1 .. 31
-__device__ __forceinline__ int low_bits(uint32_t cnt) { return 24 - __clz(cnt); }                // cnt >= 256: 1 .. 24
+__device__ __forceinline__ int low_bits(uint32_t cnt) { return cnt < (uint32_t)kExact ? 0 : 24 - __clz(cnt); }   // 0, 3 .. 24
 __device__ __forceinline__ uint32_t short_key(unsigned long long key, int idbits) {
     const uint32_t cnt = (uint32_t)(key >> 32);
     const int lb = low_bits(cnt);
@@ -259,13 +263,13 @@ __device__ __forceinline__ int rank_in_bucket(const uint32_t* s_c, const unsigne
     return r;
 }
 
-// Order-preserving bucket of a count: its leading one and the seven bits behind it (counts below 128 map to
-// themselves).  3328 buckets whose widths grow with the count, so a heavy-tailed histogram spreads over
-// many of them and a bucket near the cut holds a few hundred ids at most.
+// Order-preserving bucket of a count: counts below 1024 map to themselves, above that the leading one and
+// the seven bits behind it pick the bucket.  3968 buckets whose widths grow with the count, so a heavy-tailed
+// histogram spreads over many of them and a bucket near the cut holds a few hundred ids at most.
 __device__ __forceinline__ uint32_t fine_bucket(uint32_t c) {
-    if (c < 128u) return c;
-    const int e = 31 - __clz(c);                                       // 7 .. 31
-    return 128u + (uint32_t)(e - 7) * 128u + ((c >> (e - 7)) & 127u);  // 128 .. 3327
+    if (c < (uint32_t)kExact) return c;
+    const int e = 31 - __clz(c);                                                           // 10 .. 31
+    return (uint32_t)kExact + (uint32_t)(e - kExactLog) * 128u + ((c >> (e - 7)) & 127u);  // 1024 .. 3967
 }
 
 // Radix select (Eq. 1, Top-K(c,k)): one pass of bucket counts finds the bucket that holds the K-th key;
@@ -305,9 +309,9 @@ k_select_sort(const uint32_t* counts, int32_t V, int32_t K, int32_t* map, int32_
     uint32_t* s_gsize = s_gstart + kFine;                              // [kFine] its size over all CTAs
     uint32_t* s_next = s_gsize + kFine;                                // [kFine] scratch position of this CTA's next key
     unsigned long long* s_run = reinterpret_cast<unsigned long long*>(s_next + kFine);     // [kSortCap] phase 2: the exchange; phase 4: short keys, ranks
-    uint32_t (*s_ws)[kExact] = reinterpret_cast<uint32_t (*)[kExact]>(s_run + kSortCap);   // [kWarps][kExact] ids of a warp's piece per exact count
-    uint32_t* s_mlo = reinterpret_cast<uint32_t*>(&s_ws[kWarps][0]);   // [kFine] MODE 1: sum of the counts' low 16 bits (read by the peers)
-    uint32_t* s_mhi = s_mlo + kFine;                                   // [kFine]         and of their high 16 bits
+    uint16_t (*s_ws)[kExact] = reinterpret_cast<uint16_t (*)[kExact]>(s_run + kSortCap);   // [kWarps][kExact] ids of a warp's piece per exact count
+    uint32_t* s_ws2 = reinterpret_cast<uint32_t*>(&s_ws[0][0]);        // ... two counters to a word for the atomics
+    unsigned long long* s_mass = reinterpret_cast<unsigned long long*>(reinterpret_cast<uint8_t*>(s_run) + kMassAt);   // [kFine] MODE 1: token mass of the buckets (read by the peers)
     __shared__ uint32_t s_warp[kWarps + 1];
     __shared__ unsigned long long s_wmass[kWarps + 1];
     __shared__ unsigned long long s_mass_before;    // token mass of the buckets above the cut
@@ -322,6 +326,8 @@ k_select_sort(const uint32_t* counts, int32_t V, int32_t K, int32_t* map, int32_
     // load instruction), eight loads in flight per lane
     const int slice = (V + kCluster - 1) / kCluster;
     const int i0 = min(V, (int)rank * slice), i1 = min(V, i0 + slice);
+    const bool exact_on = slice <= kExactIds;           // (beyond that every count is ranked through the key buffer)
+    const int first_exact = exact_on ? kFirstExact : kFine;
     constexpr int kInFlight = 8;
     const int piece = (((slice + kWarps - 1) / kWarps) + 31) & ~31;
     const int w0 = min(i1, i0 + warp * piece), w1 = min(i1, w0 + piece);
@@ -329,9 +335,9 @@ k_select_sort(const uint32_t* counts, int32_t V, int32_t K, int32_t* map, int32_
 
     for (int i = threadIdx.x; i < kFine; i += kThreads) {
         s_hist[i] = 0;
-        if (MODE == 1) { s_mlo[i] = 0; s_mhi[i] = 0; }
+        if (MODE == 1) s_mass[i] = 0ull;
     }
-    for (int i = threadIdx.x; i < kWarps * kExact; i += kThreads) (&s_ws[0][0])[i] = 0;
+    for (int i = threadIdx.x; i < kWarps * kExact / 8; i += kThreads) reinterpret_cast<uint4*>(s_ws2)[i] = make_uint4(0, 0, 0, 0);
     if (threadIdx.x < kDeals * kCluster) { (&s_load[0][0])[threadIdx.x] = 0; (&s_work[0][0])[threadIdx.x] = 0u; }
     if (threadIdx.x < kDeals) { s_lo[threadIdx.x] = 0x7fffffff; s_hi[threadIdx.x] = 0; s_cut_owner[threadIdx.x] = -1; }
     if (threadIdx.x == 0) { s_cut = -1; s_big = 0; s_K = 0; s_first = 0; s_T = 0; s_mass_before = 0; }
@@ -346,20 +352,21 @@ k_select_sort(const uint32_t* counts, int32_t V, int32_t K, int32_t* map, int32_
             if (i + q * 32 < w1) {
                 const uint32_t b = kFine - 1 - fine_bucket(c[q]);
                 atomicAdd(&s_hist[b], 1u);
-                if (c[q] < (uint32_t)kExact) atomicAdd(&s_ws[warp][c[q]], 1u);
-                if (MODE == 1 && c[q] >= (uint32_t)kExact) {   // (an exact bucket's mass is a product)
-                    atomicAdd(&s_mlo[b], c[q] & 0xffffu);   // at most 2^14 ids per CTA: neither half can overflow 32 bits
-                    atomicAdd(&s_mhi[b], c[q] >> 16);
-                }
+                if (exact_on && c[q] < (uint32_t)kExact)            // (a warp's piece is 2048 ids at most: no carry between the halves)
+                    atomicAdd(&s_ws2[(warp * kExact + (int)c[q]) >> 1], 1u << ((c[q] & 1u) * 16u));
+                if (MODE == 1 && c[q] >= (uint32_t)kExact)          // (a bucket under kExact holds one value: its mass is a product)
+                    atomicAdd(&s_mass[b], (unsigned long long)c[q]);
             }
     }
     __syncthreads();
-    if (threadIdx.x < kExact) {                         // exclusive prefix over the warps, per exact count
-        uint32_t run = 0;
+    if (exact_on && threadIdx.x < kExact / 2) {         // exclusive prefix over the warps, per exact count, two counts to a word
+        uint32_t t[kWarps], run = 0;                    // (at most kExactIds ids in the CTA's slice: no carry between the halves)
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w) t[w] = s_ws2[w * (kExact / 2) + threadIdx.x];
+#pragma unroll
         for (int w = 0; w < kWarps; ++w) {
-            const uint32_t t = s_ws[w][threadIdx.x];
-            s_ws[w][threadIdx.x] = run;
-            run += t;
+            s_ws2[w * (kExact / 2) + threadIdx.x] = run;
+            run += t[w];
         }
     }
     cluster.sync();
@@ -392,12 +399,9 @@ k_select_sort(const uint32_t* counts, int32_t V, int32_t K, int32_t* map, int32_
             unsigned long long m4[BPT] = {0, 0, 0, 0};
 #pragma unroll
             for (unsigned c = 0; c < kCluster; ++c) {
-                const uint4 lo4 = reinterpret_cast<const uint4*>(cluster.map_shared_rank(s_mlo, c))[i4];
-                const uint4 hi4 = reinterpret_cast<const uint4*>(cluster.map_shared_rank(s_mhi, c))[i4];
-                m4[0] += (unsigned long long)lo4.x + ((unsigned long long)hi4.x << 16);
-                m4[1] += (unsigned long long)lo4.y + ((unsigned long long)hi4.y << 16);
-                m4[2] += (unsigned long long)lo4.z + ((unsigned long long)hi4.z << 16);
-                m4[3] += (unsigned long long)lo4.w + ((unsigned long long)hi4.w << 16);
+                const ulonglong2* mp = reinterpret_cast<const ulonglong2*>(cluster.map_shared_rank(s_mass, c)) + i4 * 2;
+                const ulonglong2 ma = mp[0], mb = mp[1];
+                m4[0] += ma.x; m4[1] += ma.y; m4[2] += mb.x; m4[3] += mb.y;
             }
 #pragma unroll
             for (int q = 0; q < BPT; ++q) s_mtot[threadIdx.x * BPT + q] = m4[q];
@@ -419,8 +423,8 @@ k_select_sort(const uint32_t* counts, int32_t V, int32_t K, int32_t* map, int32_
             const unsigned long long* mp = cluster.map_shared_rank(s_mtot, summer) + i4 * BPT;
 #pragma unroll
             for (int q = 0; q < BPT; ++q) {
-                const uint32_t value = (uint32_t)(kFine - 1 - (threadIdx.x * BPT + q));      // the bucket's count when under 256
-                mass[q] = value < 256u ? (unsigned long long)value * tot[q] : mp[q];
+                const uint32_t value = (uint32_t)(kFine - 1 - (threadIdx.x * BPT + q));      // the bucket's count when under kExact
+                mass[q] = value < (uint32_t)kExact ? (unsigned long long)value * tot[q] : mp[q];
                 msum += mass[q];
             }
         }
@@ -462,7 +466,7 @@ k_select_sort(const uint32_t* counts, int32_t V, int32_t K, int32_t* map, int32_
         else is_cut = b == min_bucket;
         if (is_cut) {
             s_cut = b; s_T = start + tot[q]; s_mass_before = mstart; s_K = (int)start; s_first = (int)start;
-            if (MODE != 0 && b >= kFirstExact) {        // an exact bucket: K follows by arithmetic, here and now
+            if (MODE != 0 && b >= first_exact) {        // an exact bucket: K follows by arithmetic, here and now
                 const uint32_t value = (uint32_t)(kFine - 1 - b);
                 uint32_t kk;
                 if (MODE == 1) kk = start + (uint32_t)(((unsigned long long)target - mstart + value - 1) / value);
@@ -498,7 +502,7 @@ k_select_sort(const uint32_t* counts, int32_t V, int32_t K, int32_t* map, int32_
 #pragma unroll
         for (int q = 0; q < BPT; ++q) {
             const int b = threadIdx.x * BPT + q;
-            const uint32_t sz = (b <= cut && b < kFirstExact) ? tot[q] : 0u;    // (ids of exact buckets are placed directly)
+            const uint32_t sz = (b <= cut && b < first_exact) ? tot[q] : 0u;    // (ids of exact buckets are placed directly)
             cost[q] = sz * (min(sz, (uint32_t)kCountCap) + kc);                 // (<= 128 K keys in all: the sum fits 32 bits)
             csum += cost[q];
         }
@@ -517,9 +521,10 @@ k_select_sort(const uint32_t* counts, int32_t V, int32_t K, int32_t* map, int32_
 #pragma unroll
         for (int q = 0; q < BPT; ++q) {
             const int b = threadIdx.x * BPT + q;
-            if (b <= cut && b < kFirstExact && tot[q] > 0) {
+            if (b <= cut && b < first_exact && tot[q] > 0) {
                 const uint32_t st = s_gstart[b];
-                const int lb = (kFine - 1 - b - 128) / 128;                    // low bits of the bucket's counts
+                const int asc = kFine - 1 - b;                                  // low bits of the bucket's counts
+                const int lb = asc < kExact ? 0 : (asc - kExact) / 128 + kExactLog - 7;
                 if (tot[q] > (uint32_t)kCountCap || (lb + id_bits(V) > 32 && tot[q] > kWideCap)) s_big = 1;
                 const unsigned owner = min((unsigned)kCluster - 1u, (unsigned)(((unsigned long long)cstart * kCluster) / max(ctotal, 1u)));
                 atomicAdd(&s_load[d][owner], tot[q]);
@@ -563,7 +568,7 @@ k_select_sort(const uint32_t* counts, int32_t V, int32_t K, int32_t* map, int32_
             const bool on = id < w1;
             const int b = (int)(kFine - 1 - fine_bucket(c[q]));
             const bool kept = on && b <= cut;
-            const bool exact = kept && b >= kFirstExact;
+            const bool exact = kept && b >= first_exact;
             const unsigned group = __ballot_sync(0xffffffffu, exact);
             if (exact) {
                 const unsigned peers = __match_any_sync(group, c[q]);
@@ -571,7 +576,7 @@ k_select_sort(const uint32_t* counts, int32_t V, int32_t K, int32_t* map, int32_
                 uint32_t before = 0;
                 if (lane == leader) {
                     before = s_ws[warp][c[q]];
-                    s_ws[warp][c[q]] = before + __popc(peers);
+                    s_ws[warp][c[q]] = (uint16_t)(before + __popc(peers));
                 }
                 before = __shfl_sync(peers, before, leader);
                 const int rk = (int)(s_next[b] + before + __popc(peers & lanemask_lt()));
@@ -652,8 +657,8 @@ static cudaError_t select_smem_attr() {
     if (e != cudaSuccess) return e;
     if (dev >= 0 && dev < 64 && attr_done[dev]) return cudaSuccess;
     e = cudaFuncSetAttribute(k_select_sort<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSelectSmem);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(k_select_sort<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSelectCutSmem);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(k_select_sort<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSelectCutSmem);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(k_select_sort<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSelectSmem);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(k_select_sort<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSelectSmem);
     if (e == cudaSuccess && dev >= 0 && dev < 64) attr_done[dev] = 1;
     return e;
 }
@@ -669,9 +674,9 @@ cudaError_t launch_select_cut(const uint32_t* counts, int32_t V, int mode, doubl
     cudaError_t e = select_smem_attr();
     if (e != cudaSuccess) return e;
     if (mode == 0)
-        k_select_sort<1><<<kCluster, kThreads, kSelectCutSmem, s>>>(counts, V, 0, map, inv_map, keyA, valA, keyB, valB, pfrac, 0u, k_out);
+        k_select_sort<1><<<kCluster, kThreads, kSelectSmem, s>>>(counts, V, 0, map, inv_map, keyA, valA, keyB, valB, pfrac, 0u, k_out);
     else
-        k_select_sort<2><<<kCluster, kThreads, kSelectCutSmem, s>>>(counts, V, 0, map, inv_map, keyA, valA, keyB, valB, 1.0, min_count, k_out);
+        k_select_sort<2><<<kCluster, kThreads, kSelectSmem, s>>>(counts, V, 0, map, inv_map, keyA, valA, keyB, valB, 1.0, min_count, k_out);
     count_launch();
     return cudaGetLastError();
 }
@@ -688,7 +693,7 @@ cudaError_t launch_select_topk(const uint32_t* counts, int32_t V, int32_t K, int
     uint32_t* valB = reinterpret_cast<uint32_t*>(scratch + 3 * seg);
     cudaError_t e = select_smem_attr();
     if (e != cudaSuccess) return e;
-    // (whatever K: even K = V is the selection's work when most ids were seen fewer than 256 times -- 31 against
+    // (whatever K: even K = V is the selection's work when most ids were seen fewer than 1024 times -- 31 against
     // 56 us on the counts of 3 M tokens -- and costs it one bucket pass, 13 us, before the full ranking when not)
     k_select_sort<0><<<kCluster, kThreads, kSelectSmem, s>>>(counts, V, K, map, inv_map, keyA, valA, keyB, valB, 1.0, 0u, nullptr);
     count_launch();

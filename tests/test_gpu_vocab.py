@@ -295,7 +295,7 @@ def test_select_minfreq_matches_oracle(V, n, f):
 
 
 @pytest.mark.parametrize("shape", ["tiny_values", "few_wide_buckets", "spikes_over_noise", "around_256", "one_value",
-                                   "huge_counts_few_per_bucket", "huge_counts_full_buckets"])
+                                   "huge_counts_few_per_bucket", "huge_counts_full_buckets", "around_1024"])
 def test_select_cuts_over_count_shapes_that_stress_the_buckets(shape):
     """Count vectors chosen against the bucket scheme of the selection kernel: huge buckets of equal counts, all
     counts in a handful of wide buckets, a few enormous counts over noise, counts on both sides of the value from
@@ -309,7 +309,8 @@ def test_select_cuts_over_count_shapes_that_stress_the_buckets(shape):
          # counts so large that what orders a bucket's keys (the count's low bits, then the id) passes 32 bits:
          # a dozen ids per such bucket, and hundreds
          "huge_counts_few_per_bucket": np.where(rng.random(V) < 0.02, (1 << 30) + rng.integers(0, 1 << 30, V), rng.integers(0, 3, V)),
-         "huge_counts_full_buckets": (1 << 30) + rng.integers(0, 1 << 24, V)}[shape].astype(np.uint64)
+         "huge_counts_full_buckets": (1 << 30) + rng.integers(0, 1 << 24, V),
+         "around_1024": rng.integers(1000, 1050, V)}[shape].astype(np.uint64)
     counts = torch.from_numpy(c.astype(np.uint32).view(np.int32)).to(DEV)
     ws = vt.Workspace(vt.workspace_bytes(vt.VT_OP_SELECT_TOPK, 0, V, V))
     for p in (1e-12, 0.3, 0.9, 1.0):
@@ -317,7 +318,7 @@ def test_select_cuts_over_count_shapes_that_stress_the_buckets(shape):
         K, rmap, rinv = oracle.select_topp(c, p)
         assert int(k_out.item()) == K
         assert np.array_equal(map_.cpu().numpy()[:K], rmap[:K]) and np.array_equal(inv.cpu().numpy(), rinv)
-    for f in (0, 1, 255, 256, 257, int(np.median(c)), int(c.max()), int(c.max()) + 1):
+    for f in (0, 1, 255, 256, 257, 1023, 1024, 1025, int(np.median(c)), int(c.max()), int(c.max()) + 1):
         k_out, map_, inv = vt.vt_select_minfreq(counts, f, ws=ws)
         K, rmap, rinv = oracle.select_minfreq(c, f)
         assert int(k_out.item()) == K
@@ -326,6 +327,32 @@ def test_select_cuts_over_count_shapes_that_stress_the_buckets(shape):
         map_, inv = vt.vt_select_topk(counts, K, ws=ws)
         rmap, rinv = oracle.select_topk(c, K)
         assert np.array_equal(map_.cpu().numpy(), rmap) and np.array_equal(inv.cpu().numpy(), rinv)
+    _assert_clean(ws)
+
+
+def test_select_vocabulary_whose_slices_pass_the_sixteen_bit_counters():
+    """A CTA ranks rare ids where it places them only while its slice of the vocabulary has at most 65535 ids;
+    with 600 K ids every count goes through the key buffer.  Small counts in large numbers, Top-K, Top-P and
+    minimum frequency."""
+    V = 600_001
+    rng = np.random.default_rng(11)
+    c = np.where(rng.random(V) < 0.9, rng.integers(0, 6, V), (rng.pareto(1.1, V) * 800).astype(np.int64)).astype(np.uint64)
+    counts = torch.from_numpy(c.astype(np.uint32).view(np.int32)).to(DEV)
+    ws = vt.Workspace(vt.workspace_bytes(vt.VT_OP_SELECT_TOPK, 0, V, V))
+    for K in (1, 5000, 70_000, V):
+        map_, inv = vt.vt_select_topk(counts, K, ws=ws)
+        rmap, rinv = oracle.select_topk(c, K)
+        assert np.array_equal(map_.cpu().numpy(), rmap) and np.array_equal(inv.cpu().numpy(), rinv)
+    for p in (0.5, 0.97):
+        k_out, map_, inv = vt.vt_select_topp(counts, p, ws=ws)
+        K, rmap, rinv = oracle.select_topp(c, p)
+        assert int(k_out.item()) == K
+        assert np.array_equal(map_.cpu().numpy()[:K], rmap[:K]) and np.array_equal(inv.cpu().numpy(), rinv)
+    for f in (3, 1024):
+        k_out, map_, inv = vt.vt_select_minfreq(counts, f, ws=ws)
+        K, rmap, rinv = oracle.select_minfreq(c, f)
+        assert int(k_out.item()) == K
+        assert np.array_equal(map_.cpu().numpy()[:K], rmap[:K]) and np.array_equal(inv.cpu().numpy(), rinv)
     _assert_clean(ws)
 
 
