@@ -28,7 +28,6 @@ constexpr int kDigits = 256;
 constexpr int kFine = 4096;                      // buckets of the selection pass (3968 in use)
 constexpr int kSortCap = 12288;                  // 64-bit keys one CTA ranks in shared memory
 constexpr int kExact = 1024;                     // counts below this have a bucket to themselves (fine_bucket)
-constexpr int kExactLog = 10;
 constexpr int kFirstExact = kFine - kExact;      // ... the buckets kFirstExact .. kFine-1 in descending order
 constexpr int kExactIds = 65535;                 // ids per CTA up to which such counts are ranked where they are placed (16-bit counters)
 constexpr int kCountCap = 2048;                  // largest bucket ranked by counting its greater keys
@@ -208,13 +207,24 @@ __device__ void lsd_rank_all(cg::cluster_group& cluster, const uint32_t* counts,
     }
 }
 
-// The keys of one bucket of counts >= 1024 agree in the count's leading one and the seven bits behind it; what
+// The keys of one bucket of counts >= 1024 agree in the count's leading one and the six to eight bits behind it; what
 // orders them is the rest of the count and then ~id.  Where that fits 32 bits (lb low bits of the count + the
 // bits of an id) it is the short key compared in shared memory; a bucket where it does not fit (counts from 2^23
 // with a 17-bit id) is called wide and compares its 64-bit keys where they lie in global memory -- the deal
 // hands such a bucket to the ranking only while it is tiny.
 __device__ __forceinline__ int id_bits(int32_t V) { return 32 - __clz(max(V - 1, 1)); }          // 1 .. 31
-__device__ __forceinline__ int low_bits(uint32_t cnt) { return cnt < (uint32_t)kExact ? 0 : 24 - __clz(cnt); }   // 0, 3 .. 24
+// Bits of a count that its bucket leaves open, from the count and from the bucket (ascending index).
+__device__ __forceinline__ int low_bits(uint32_t cnt) {
+    if (cnt < (uint32_t)kExact) return 0;
+    const int e = 31 - __clz(cnt);
+    return e < 14 ? e - 8 : e < 26 ? e - 7 : e - 6;                                        // 2 .. 25
+}
+__device__ __forceinline__ int low_bits_of_bucket(int asc) {
+    if (asc < kExact) return 0;
+    if (asc < 2048) return 10 + (asc - 1024) / 256 - 8;
+    if (asc < 3584) return 14 + (asc - 2048) / 128 - 7;
+    return 26 + (asc - 3584) / 64 - 6;
+}
 __device__ __forceinline__ uint32_t short_key(unsigned long long key, int idbits) {
     const uint32_t cnt = (uint32_t)(key >> 32);
     const int lb = low_bits(cnt);
@@ -263,13 +273,18 @@ __device__ __forceinline__ int rank_in_bucket(const uint32_t* s_c, const unsigne
     return r;
 }
 
-// Order-preserving bucket of a count: counts below 1024 map to themselves, above that the leading one and
-// the seven bits behind it pick the bucket.  3968 buckets whose widths grow with the count, so a heavy-tailed
-// histogram spreads over many of them and a bucket near the cut holds a few hundred ids at most.
+// Order-preserving bucket of a count: counts below 1024 map to themselves; above that the leading one and the
+// bits behind it pick the bucket -- eight bits for counts below 2^14 (where the cut of a large corpus falls and a
+// bucket would otherwise hold hundreds of ids), seven below 2^26, six above.  3968 buckets whose widths grow with
+// the count, so a heavy-tailed histogram spreads over many of them.
 __device__ __forceinline__ uint32_t fine_bucket(uint32_t c) {
-    if (c < (uint32_t)kExact) return c;
-    const int e = 31 - __clz(c);                                                           // 10 .. 31
-    return (uint32_t)kExact + (uint32_t)(e - kExactLog) * 128u + ((c >> (e - 7)) & 127u);  // 1024 .. 3967
+    // (no branches: with m bits behind the leading one, c >> (e - m) is 2^m + those bits, and the octave's first
+    // bucket is linear in e, so bucket = (e << m) + (c >> (e - m)) + a constant per range of e)
+    const int e = 31 - __clz(c | 1u);                                  // 10 .. 31 where it is used
+    const int m = e < 14 ? 8 : e < 26 ? 7 : 6;
+    const int k = e < 14 ? -1792 : e < 26 ? 128 : 1856;                // 1024..2047 | 2048..3583 | 3584..3967
+    const uint32_t wide = (uint32_t)((e << m) + k) + (c >> ((e - m) & 31));
+    return c < (uint32_t)kExact ? c : wide;
 }
 
 // Radix select (Eq. 1, Top-K(c,k)): one pass of bucket counts finds the bucket that holds the K-th key;
@@ -311,7 +326,11 @@ k_select_sort(const uint32_t* counts, int32_t V, int32_t K, int32_t* map, int32_
     unsigned long long* s_run = reinterpret_cast<unsigned long long*>(s_next + kFine);     // [kSortCap] phase 2: the exchange; phase 4: short keys, ranks
     uint16_t (*s_ws)[kExact] = reinterpret_cast<uint16_t (*)[kExact]>(s_run + kSortCap);   // [kWarps][kExact] ids of a warp's piece per exact count
     uint32_t* s_ws2 = reinterpret_cast<uint32_t*>(&s_ws[0][0]);        // ... two counters to a word for the atomics
-    unsigned long long* s_mass = reinterpret_cast<unsigned long long*>(reinterpret_cast<uint8_t*>(s_run) + kMassAt);   // [kFine] MODE 1: token mass of the buckets (read by the peers)
+    // MODE 1: token mass of the buckets (read by the peers), in the key buffer while that is idle: the sums of the counts'
+    // low and high 16 bits, which cannot pass 32 bits for a slice of kExactIds ids; beyond that one 64-bit sum (a slow add)
+    uint32_t* s_mlo = reinterpret_cast<uint32_t*>(reinterpret_cast<uint8_t*>(s_run) + kMassAt);   // [kFine]
+    uint32_t* s_mhi = s_mlo + kFine;                                                              // [kFine]
+    unsigned long long* s_mass = reinterpret_cast<unsigned long long*>(s_mlo);                    // [kFine] instead of the two
     __shared__ uint32_t s_warp[kWarps + 1];
     __shared__ unsigned long long s_wmass[kWarps + 1];
     __shared__ unsigned long long s_mass_before;    // token mass of the buckets above the cut
@@ -354,8 +373,14 @@ k_select_sort(const uint32_t* counts, int32_t V, int32_t K, int32_t* map, int32_
                 atomicAdd(&s_hist[b], 1u);
                 if (exact_on && c[q] < (uint32_t)kExact)            // (a warp's piece is 2048 ids at most: no carry between the halves)
                     atomicAdd(&s_ws2[(warp * kExact + (int)c[q]) >> 1], 1u << ((c[q] & 1u) * 16u));
-                if (MODE == 1 && c[q] >= (uint32_t)kExact)          // (a bucket under kExact holds one value: its mass is a product)
-                    atomicAdd(&s_mass[b], (unsigned long long)c[q]);
+                if (MODE == 1 && c[q] >= (uint32_t)kExact) {        // (a bucket under kExact holds one value: its mass is a product)
+                    if (exact_on) {
+                        atomicAdd(&s_mlo[b], c[q] & 0xffffu);
+                        atomicAdd(&s_mhi[b], c[q] >> 16);
+                    } else {
+                        atomicAdd(&s_mass[b], (unsigned long long)c[q]);
+                    }
+                }
             }
     }
     __syncthreads();
@@ -399,9 +424,18 @@ k_select_sort(const uint32_t* counts, int32_t V, int32_t K, int32_t* map, int32_
             unsigned long long m4[BPT] = {0, 0, 0, 0};
 #pragma unroll
             for (unsigned c = 0; c < kCluster; ++c) {
-                const ulonglong2* mp = reinterpret_cast<const ulonglong2*>(cluster.map_shared_rank(s_mass, c)) + i4 * 2;
-                const ulonglong2 ma = mp[0], mb = mp[1];
-                m4[0] += ma.x; m4[1] += ma.y; m4[2] += mb.x; m4[3] += mb.y;
+                if (exact_on) {
+                    const uint4 lo4 = reinterpret_cast<const uint4*>(cluster.map_shared_rank(s_mlo, c))[i4];
+                    const uint4 hi4 = reinterpret_cast<const uint4*>(cluster.map_shared_rank(s_mhi, c))[i4];
+                    m4[0] += (unsigned long long)lo4.x + ((unsigned long long)hi4.x << 16);
+                    m4[1] += (unsigned long long)lo4.y + ((unsigned long long)hi4.y << 16);
+                    m4[2] += (unsigned long long)lo4.z + ((unsigned long long)hi4.z << 16);
+                    m4[3] += (unsigned long long)lo4.w + ((unsigned long long)hi4.w << 16);
+                } else {
+                    const ulonglong2* mp = reinterpret_cast<const ulonglong2*>(cluster.map_shared_rank(s_mass, c)) + i4 * 2;
+                    const ulonglong2 ma = mp[0], mb = mp[1];
+                    m4[0] += ma.x; m4[1] += ma.y; m4[2] += mb.x; m4[3] += mb.y;
+                }
             }
 #pragma unroll
             for (int q = 0; q < BPT; ++q) s_mtot[threadIdx.x * BPT + q] = m4[q];
@@ -420,7 +454,9 @@ k_select_sort(const uint32_t* counts, int32_t V, int32_t K, int32_t* map, int32_
 #pragma unroll
         for (int q = 0; q < BPT; ++q) { sum += tot[q]; mass[q] = 0; }
         if (MODE == 1) {
-            const unsigned long long* mp = cluster.map_shared_rank(s_mtot, summer) + i4 * BPT;
+            const ulonglong2* mp2 = reinterpret_cast<const ulonglong2*>(cluster.map_shared_rank(s_mtot, summer) + i4 * BPT);
+            const ulonglong2 ma = mp2[0], mb = mp2[1];
+            const unsigned long long mp[BPT] = {ma.x, ma.y, mb.x, mb.y};
 #pragma unroll
             for (int q = 0; q < BPT; ++q) {
                 const uint32_t value = (uint32_t)(kFine - 1 - (threadIdx.x * BPT + q));      // the bucket's count when under kExact
@@ -447,12 +483,22 @@ k_select_sort(const uint32_t* counts, int32_t V, int32_t K, int32_t* map, int32_
     uint32_t start = incl - sum;
     for (int w = 0; w < warp; ++w) start += s_warp[w];
     unsigned long long mstart = mincl - msum, mtotal = 0;
+    // Top-P: target = ceil(p * total) is the one fp64 product; what is compared with it are integers, and while the
+    // total is under 2^53 (every prefix then converts exactly) they are compared as integers -- fp64 conversions of
+    // every bucket's prefix in every thread were 5 us of this kernel
     double target = 0.0;
+    unsigned long long itarget = 0;
+    bool as_int = true;
     if (MODE == 1) {
         for (int w = 0; w < warp; ++w) mstart += s_wmass[w];
         for (int w = 0; w < kWarps; ++w) mtotal += s_wmass[w];
-        target = ceil(pfrac * (double)mtotal);
+        if (lane == 0) target = ceil(pfrac * (double)mtotal);
+        target = __shfl_sync(0xffffffffu, target, 0);
+        as_int = mtotal < (1ull << 53);
+        itarget = as_int ? (unsigned long long)target : 0ull;
     }
+    auto below = [&](unsigned long long x) { return as_int ? x < itarget : (double)x < target; };
+    auto reaches = [&](unsigned long long x) { return as_int ? x >= itarget : (double)x >= target; };
     const int min_bucket = MODE == 2 ? (int)(kFine - 1 - fine_bucket(min_count)) : 0;
 #pragma unroll
     for (int q = 0; q < BPT; ++q) {
@@ -462,7 +508,7 @@ k_select_sort(const uint32_t* counts, int32_t V, int32_t K, int32_t* map, int32_
         s_next[b] = start + mine_before[q];
         bool is_cut;
         if (MODE == 0) is_cut = start < (uint32_t)K && start + tot[q] >= (uint32_t)K;                   // exactly one bucket
-        else if (MODE == 1) is_cut = (double)mstart < target && (double)(mstart + mass[q]) >= target;  // exactly one, if any token was counted
+        else if (MODE == 1) is_cut = below(mstart) && reaches(mstart + mass[q]);                       // exactly one, if any token was counted
         else is_cut = b == min_bucket;
         if (is_cut) {
             s_cut = b; s_T = start + tot[q]; s_mass_before = mstart; s_K = (int)start; s_first = (int)start;
@@ -523,8 +569,7 @@ k_select_sort(const uint32_t* counts, int32_t V, int32_t K, int32_t* map, int32_
             const int b = threadIdx.x * BPT + q;
             if (b <= cut && b < first_exact && tot[q] > 0) {
                 const uint32_t st = s_gstart[b];
-                const int asc = kFine - 1 - b;                                  // low bits of the bucket's counts
-                const int lb = asc < kExact ? 0 : (asc - kExact) / 128 + kExactLog - 7;
+                const int lb = low_bits_of_bucket(kFine - 1 - b);
                 if (tot[q] > (uint32_t)kCountCap || (lb + id_bits(V) > 32 && tot[q] > kWideCap)) s_big = 1;
                 const unsigned owner = min((unsigned)kCluster - 1u, (unsigned)(((unsigned long long)cstart * kCluster) / max(ctotal, 1u)));
                 atomicAdd(&s_load[d][owner], tot[q]);
@@ -615,9 +660,9 @@ k_select_sort(const uint32_t* counts, int32_t V, int32_t K, int32_t* map, int32_
         }
         return;
     }
-    // K from the ranks: first every key's place (and, inside the cut bucket, the token mass ranked before it),
-    // then -- in the CTA that ranks the cut bucket -- K, then the outputs.  The other CTAs rank buckets above
-    // the cut only: all of theirs is kept.
+    // K from the ranks.  A key of a bucket above the cut is kept whatever K turns out to be (K is at least the cut
+    // bucket's first rank) and is emitted with its place; the keys of the cut bucket -- all in one CTA -- get their
+    // places (and, Top-P, the token mass ranked before them), that CTA reads K off them, and then they are emitted.
     const bool owns_cut = s_cut_owner[deal] == (int)rank || (s_cut_owner[deal] < 0 && rank == 0);   // (an empty cut bucket has no owner)
     const unsigned long long mass_before = s_mass_before;
     for (int j = threadIdx.x; j < n; j += kThreads) {
@@ -630,21 +675,31 @@ k_select_sort(const uint32_t* counts, int32_t V, int32_t K, int32_t* map, int32_
             unsigned long long m = 0;
             r = rank_in_bucket<true>(s_c, run, key, bs, be, idbits, &m);
             const unsigned long long cum = mass_before + m;
-            if ((double)cum < target && (double)(cum + cnt) >= target) s_K = r0 + bs + r + 1;   // exactly one key
+            if (below(cum) && reaches(cum + cnt)) s_K = r0 + bs + r + 1;                          // exactly one key
         } else {
             r = rank_in_bucket<false>(s_c, run, key, bs, be, idbits, nullptr);
             if (b == cut && MODE == 2 && cnt >= min_count) atomicMax(&s_K, r0 + bs + r + 1);
         }
-        s_place[j] = (uint32_t)(r0 + bs + r);
+        const int rk = r0 + bs + r;
+        if (b == cut) {
+            s_place[j] = (uint32_t)rk;
+        } else {
+            const int32_t v = (int32_t)(0xffffffffu - (uint32_t)key);
+            s_place[j] = 0xffffffffu;                   // emitted
+            map[rk] = v;
+            inv_map[v] = rk;
+        }
     }
     __syncthreads();
-    const int Kf = owns_cut ? max(1, min(V, s_K)) : (int)T;
-    if (owns_cut && threadIdx.x == 0) *k_out = Kf;
+    if (!owns_cut) return;
+    const int Kf = max(1, min(V, s_K));
+    if (threadIdx.x == 0) *k_out = Kf;
     for (int j = threadIdx.x; j < n; j += kThreads) {
+        const uint32_t rk = s_place[j];
+        if (rk == 0xffffffffu) continue;
         const int32_t v = (int32_t)(0xffffffffu - (uint32_t)__ldcg(run + j));
-        const int rk = (int)s_place[j];
-        if (rk < Kf) map[rk] = v;
-        inv_map[v] = rk < Kf ? rk : -1;
+        if ((int)rk < Kf) map[rk] = v;
+        inv_map[v] = (int)rk < Kf ? (int)rk : -1;
     }
 }
 
