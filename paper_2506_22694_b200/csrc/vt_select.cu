@@ -342,12 +342,12 @@ k_select_sort(const uint32_t* counts, int32_t V, int32_t K, int32_t* map, int32_
 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     // ids of this CTA: a contiguous slice; every warp walks a contiguous piece of it in id order (128 bytes per
-    // load instruction), eight loads in flight per lane
+    // load instruction), sixteen loads in flight per lane (all of a lane's ids at V = 128256)
     const int slice = (V + kCluster - 1) / kCluster;
     const int i0 = min(V, (int)rank * slice), i1 = min(V, i0 + slice);
     const bool exact_on = slice <= kExactIds;           // (beyond that every count is ranked through the key buffer)
     const int first_exact = exact_on ? kFirstExact : kFine;
-    constexpr int kInFlight = 8;
+    constexpr int kInFlight = 16;
     const int piece = (((slice + kWarps - 1) / kWarps) + 31) & ~31;
     const int w0 = min(i1, i0 + warp * piece), w1 = min(i1, w0 + piece);
     unsigned long long* pairs = reinterpret_cast<unsigned long long*>(keyA);       // [V] 64-bit keys (keyA and valA are adjacent)
@@ -370,9 +370,10 @@ k_select_sort(const uint32_t* counts, int32_t V, int32_t K, int32_t* map, int32_
         for (int q = 0; q < kInFlight; ++q)
             if (i + q * 32 < w1) {
                 const uint32_t b = kFine - 1 - fine_bucket(c[q]);
-                atomicAdd(&s_hist[b], 1u);
-                if (exact_on && c[q] < (uint32_t)kExact)            // (a warp's piece is 2048 ids at most: no carry between the halves)
-                    atomicAdd(&s_ws2[(warp * kExact + (int)c[q]) >> 1], 1u << ((c[q] & 1u) * 16u));
+                if (exact_on && c[q] < (uint32_t)kExact)            // (a warp's piece is 2048 ids at most: no carry between the halves;
+                    atomicAdd(&s_ws2[(warp * kExact + (int)c[q]) >> 1], 1u << ((c[q] & 1u) * 16u));   // the bucket's count is their sum, below)
+                else
+                    atomicAdd(&s_hist[b], 1u);
                 if (MODE == 1 && c[q] >= (uint32_t)kExact) {        // (a bucket under kExact holds one value: its mass is a product)
                     if (exact_on) {
                         atomicAdd(&s_mlo[b], c[q] & 0xffffu);
@@ -393,6 +394,8 @@ k_select_sort(const uint32_t* counts, int32_t V, int32_t K, int32_t* map, int32_
             s_ws2[w * (kExact / 2) + threadIdx.x] = run;
             run += t[w];
         }
+        s_hist[kFine - 1 - 2 * (int)threadIdx.x] = run & 0xffffu;       // the CTA's ids with count 2t and 2t + 1
+        s_hist[kFine - 2 - 2 * (int)threadIdx.x] = run >> 16;
     }
     cluster.sync();
     // phase 2: start of every bucket in descending order (each thread owns kFine / kThreads neighbouring
