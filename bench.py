@@ -711,6 +711,29 @@ def small_case(vt, dev, args, peak_gbs):
             rec[name] = {"ms": ms, "gtok_s": n / ms / 1e6, "gbs": 4.0 * n / ms / 1e6, "frac_of_measured": 4.0 * n / ms / 1e6 / peak_gbs}
         rec["histogram_over_ceiling"] = rec["folded"]["ms"] / rec["histogram"]["ms"]
         print(json.dumps(rec), flush=True)
+    elif args.case == "select":
+        # the three selection rules on the counts of --hist-n ids of the vocabulary-build stream: Top-K first
+        # (a capture of the first launches of the selection kernel sees the K = 32768 instance)
+        n = args.hist_n
+        ids = vt_inputs.zipf_ids(n, V, 1.07, seed=1005, noise_frac=0.05, device=dev)
+        counts = vt.vt_histogram(ids, V)
+        del ids
+        ws = vt.Workspace(vt.workspace_bytes(vt.VT_OP_SELECT_TOPK, 0, V, V), dev)
+        rec = {"case": "select", "n": n, "V": V}
+        for name, fn in (("topk_K32768_us", lambda: vt.vt_select_topk(counts, 32768, ws=ws)),
+                         ("topp_p0.9_us", lambda: vt.vt_select_topp(counts, 0.9, ws=ws)),
+                         ("minfreq_1000_us", lambda: vt.vt_select_minfreq(counts, 1000, ws=ws))):
+            for _ in range(args.warmup):
+                fn()
+            torch.cuda.synchronize()
+            e0, e1 = _events()
+            e0.record()
+            for _ in range(args.steps):
+                fn()
+            e1.record()
+            torch.cuda.synchronize()
+            rec[name] = e0.elapsed_time(e1) / args.steps * 1e3
+        print(json.dumps(rec), flush=True)
     elif args.case == "dense":
         print(json.dumps(dict(case="dense", **dense_case(vt, dev, args.steps, args.warmup))), flush=True)
     else:
@@ -747,9 +770,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-extras", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--case", default="head", choices=["head", "hist", "hist-ceiling", "tree", "dense", "stamps"],
-                    help="head: the full bench line (default); hist / tree / dense: a short run of the vocabulary "
-                         "histogram (--hist-n ids), of the tree-drafting head or of the batched head, for profiler "
+    ap.add_argument("--case", default="head", choices=["head", "hist", "hist-ceiling", "select", "tree", "dense", "stamps"],
+                    help="head: the full bench line (default); hist / select / tree / dense: a short run of the vocabulary "
+                         "histogram (--hist-n ids), of the selections on its counts, of the tree-drafting head or of the batched head, for profiler "
                          "captures; stamps: per-phase timeline of a head step from the instrumented build")
     ap.add_argument("--hist-n", type=int, default=200_000_000)
     args = ap.parse_args()
