@@ -1,16 +1,21 @@
-// Top-K vocabulary selection (Eq. 1, first line: V_trim = V[Top-K(c,k)]) in rank order.
+// Top-K vocabulary selection (Eq. 1, first line: V_trim = V[Top-K(c,k)]) in rank order, and the Method
+// section's two other rules (Top-P, minimum frequency) over the same ranking.
 //
-// The wanted order -- count descending, equal counts by ascending id -- is exactly what a STABLE
-// sort of the ids by descending count produces when it starts from ascending id order.  So the
-// whole selection is one least-significant-digit radix sort of V 32-bit counts (8-bit digits,
-// passes whose digit is constant are skipped), after which map = first K sorted ids and
-// inv_map = rank (or -1) scattered by id.
+// V is about 1e5: the job is latency-bound, not bandwidth-bound.  It runs as ONE thread-block cluster of
+// 8 CTAs (one launch, no grid-wide spin) that talk through distributed shared memory between hardware
+// cluster barriers.  Two algorithms live here:
 //
-// V is about 1e5: the job is latency-bound, not bandwidth-bound.  It runs as ONE thread-block
-// cluster of 8 CTAs (one launch, no grid-wide spin): per pass each CTA counts the digits of its
-// contiguous slice, the CTAs exchange their 256 digit totals through distributed shared memory
-// between two hardware cluster barriers, and each warp then scatters its sub-slice stably using
-// warp match ranks.  Keys and ids ping-pong between two scratch arrays that stay in L2.
+//  * the selection (k_select_sort, further down): one pass of bucket counts finds where the K-th key lies;
+//    only the keys down to there are ranked, and ids that were seen fewer than 1024 times take their
+//    rank where they are first placed.  Every call starts here.
+//  * the full ranking (lsd_rank_all, first): the wanted order -- count descending, equal counts by
+//    ascending id -- is exactly what a STABLE sort of the ids by descending count produces when it
+//    starts from ascending id order, so it is one least-significant-digit radix sort of V 32-bit counts
+//    (8-bit digits, passes whose digit is constant are skipped): per pass each CTA counts the digits of
+//    its contiguous slice, the CTAs exchange their 256 digit totals, and each warp scatters its
+//    sub-slice stably using warp match ranks; keys and ids ping-pong between two scratch arrays that stay
+//    in L2.  The selection falls through to it when what it would have to rank does not fit its shared
+//    memory or would cost more than this.
 #include <cooperative_groups.h>
 
 #include "vt_common.cuh"
@@ -26,7 +31,7 @@ constexpr int kThreads = 1024;
 constexpr int kWarps = kThreads / 32;
 constexpr int kDigits = 256;
 constexpr int kFine = 4096;                      // buckets of the selection pass (3968 in use)
-constexpr int kSortCap = 12288;                  // 64-bit keys one CTA ranks in shared memory
+constexpr int kSortCap = 12288;                  // keys one CTA ranks in shared memory (a 32-bit short key and a 32-bit rank each)
 constexpr int kExact = 1024;                     // counts below this have a bucket to themselves (fine_bucket)
 constexpr int kFirstExact = kFine - kExact;      // ... the buckets kFirstExact .. kFine-1 in descending order
 constexpr int kExactIds = 65535;                 // ids per CTA up to which such counts are ranked where they are placed (16-bit counters)
