@@ -330,11 +330,11 @@ def test_select_cuts_over_count_shapes_that_stress_the_buckets(shape):
     _assert_clean(ws)
 
 
-def test_select_vocabulary_whose_slices_pass_the_sixteen_bit_counters():
-    """A CTA ranks rare ids where it places them only while its slice of the vocabulary has at most 65535 ids;
-    with 600 K ids every count goes through the key buffer.  Small counts in large numbers, Top-K, Top-P and
-    minimum frequency."""
-    V = 600_001
+@pytest.mark.parametrize("V", [8 * 65535, 8 * 65535 + 1, 600_001])
+def test_select_vocabulary_whose_slices_pass_the_sixteen_bit_counters(V):
+    """A CTA ranks rare ids where it places them only while its slice of the vocabulary has at most 65535 ids
+    (the first V is the last to which that applies); beyond that every count goes through the key buffer.
+    Small counts in large numbers, Top-K, Top-P and minimum frequency."""
     rng = np.random.default_rng(11)
     c = np.where(rng.random(V) < 0.9, rng.integers(0, 6, V), (rng.pareto(1.1, V) * 800).astype(np.int64)).astype(np.uint64)
     counts = torch.from_numpy(c.astype(np.uint32).view(np.int32)).to(DEV)
