@@ -283,13 +283,13 @@ __device__ __forceinline__ int rank_in_bucket(const uint32_t* s_c, const unsigne
 // bucket would otherwise hold hundreds of ids), seven below 2^26, six above.  3968 buckets whose widths grow with
 // the count, so a heavy-tailed histogram spreads over many of them.
 __device__ __forceinline__ uint32_t fine_bucket(uint32_t c) {
-    // (no branches: with m bits behind the leading one, c >> (e - m) is 2^m + those bits, and the octave's first
-    // bucket is linear in e, so bucket = (e << m) + (c >> (e - m)) + a constant per range of e)
-    const int e = 31 - __clz(c | 1u);                                  // 10 .. 31 where it is used
-    const int m = e < 14 ? 8 : e < 26 ? 7 : 6;
-    const int k = e < 14 ? -1792 : e < 26 ? 128 : 1856;                // 1024..2047 | 2048..3583 | 3584..3967
-    const uint32_t wide = (uint32_t)((e << m) + k) + (c >> ((e - m) & 31));
-    return c < (uint32_t)kExact ? c : wide;
+    // (no branches: the bits of c converted to fp32 toward zero are its exponent followed by the bits behind the
+    // leading one, so a shift leaves exponent and m bits, and the octave's first bucket is a constant away)
+    const uint32_t bits = __float_as_uint(__uint2float_rz(c));
+    const bool lo = c < (1u << 14), mid = c < (1u << 26);
+    const uint32_t sh = lo ? 15u : mid ? 16u : 17u;                    // 23 - m
+    const uint32_t off = lo ? 34048u : mid ? 16000u : 6208u;           // ((127 + first e) << m) - first bucket of the range
+    return c < (uint32_t)kExact ? c : (bits >> sh) - off;
 }
 
 // Radix select (Eq. 1, Top-K(c,k)): one pass of bucket counts finds the bucket that holds the K-th key;
