@@ -463,7 +463,9 @@ def extras(vt, dev, peak_gbs, peak_kind):
         vb["build_vocab_K%d_ms" % K] = ms_b
         vb["build_vocab_K%d_gtok_s" % K] = n / (ms_b * 1e-3) / 1e9
     # the selections alone, back to back on the counts of all n ids (100 calls each: the first call's start-up is
-    # a tenth of a microsecond of the mean)
+    # a tenth of a microsecond of the mean), behind a clock-sampled run of the same call: these are latency-bound
+    # kernels on 8 SMs, and the histogram before them leaves the chip at the power cap's clock
+    vb["select_clocks"] = clocks_under(lambda i: vt.vt_select_topk(counts, 32768, ws=ws), dev.index)
     for K in (8192, 32768):
         vb["select_topk_K%d_us" % K] = timed(lambda: vt.vt_select_topk(counts, K, ws=ws), reps=100, warm=5) * 1e3
     for p_ in (0.9, 0.99):
