@@ -30,7 +30,7 @@ constexpr int kCluster = 8;
 constexpr int kThreads = 1024;
 constexpr int kWarps = kThreads / 32;
 constexpr int kDigits = 256;
-constexpr int kFine = 4096;                      // buckets of the selection pass (3968 in use)
+constexpr int kFine = 4096;                      // buckets of the selection pass (4032 in use)
 constexpr int kSortCap = 12288;                  // keys one CTA ranks in shared memory (a 32-bit short key and a 32-bit rank each)
 constexpr int kExact = 1024;                     // counts below this have a bucket to themselves (fine_bucket)
 constexpr int kFirstExact = kFine - kExact;      // ... the buckets kFirstExact .. kFine-1 in descending order
@@ -212,9 +212,9 @@ __device__ void lsd_rank_all(cg::cluster_group& cluster, const uint32_t* counts,
     }
 }
 
-// The keys of one bucket of counts >= 1024 agree in the count's leading one and the six to eight bits behind it; what
+// The keys of one bucket of counts >= 1024 agree in the count's leading one and the five to nine bits behind it; what
 // orders them is the rest of the count and then ~id.  Where that fits 32 bits (lb low bits of the count + the
-// bits of an id) it is the short key compared in shared memory; a bucket where it does not fit (counts from 2^23
+// bits of an id) it is the short key compared in shared memory; a bucket where it does not fit (counts from 2^21
 // with a 17-bit id) is called wide and compares its 64-bit keys where they lie in global memory -- the deal
 // hands such a bucket to the ranking only while it is tiny.
 __device__ __forceinline__ int id_bits(int32_t V) { return 32 - __clz(max(V - 1, 1)); }          // 1 .. 31
@@ -222,13 +222,13 @@ __device__ __forceinline__ int id_bits(int32_t V) { return 32 - __clz(max(V - 1,
 __device__ __forceinline__ int low_bits(uint32_t cnt) {
     if (cnt < (uint32_t)kExact) return 0;
     const int e = 31 - __clz(cnt);
-    return e < 14 ? e - 8 : e < 26 ? e - 7 : e - 6;                                        // 2 .. 25
+    return e < 14 ? e - 9 : e < 18 ? e - 7 : e - 5;                                        // 1 .. 26
 }
 __device__ __forceinline__ int low_bits_of_bucket(int asc) {
     if (asc < kExact) return 0;
-    if (asc < 2048) return 10 + (asc - 1024) / 256 - 8;
-    if (asc < 3584) return 14 + (asc - 2048) / 128 - 7;
-    return 26 + (asc - 3584) / 64 - 6;
+    if (asc < 3072) return 10 + (asc - 1024) / 512 - 9;
+    if (asc < 3584) return 14 + (asc - 3072) / 128 - 7;
+    return 18 + (asc - 3584) / 32 - 5;
 }
 __device__ __forceinline__ uint32_t short_key(unsigned long long key, int idbits) {
     const uint32_t cnt = (uint32_t)(key >> 32);
@@ -279,17 +279,17 @@ __device__ __forceinline__ int rank_in_bucket(const uint32_t* s_c, const unsigne
 }
 
 // Order-preserving bucket of a count: counts below 1024 map to themselves; above that the leading one and the
-// bits behind it pick the bucket -- eight bits for counts below 2^14 (where the cut of a large corpus falls and a
-// bucket would otherwise hold hundreds of ids), seven below 2^26, six above.  3968 buckets whose widths grow with
-// the count, so a heavy-tailed histogram spreads over many of them.
+// bits behind it pick the bucket -- nine bits for counts below 2^14 (where the cut of a large corpus falls and a
+// bucket would otherwise hold hundreds of ids), seven below 2^18, five above (a few hundred ids in all at such
+// counts).  4032 buckets whose widths grow with the count, so a heavy-tailed histogram spreads over many of them.
 __device__ __forceinline__ uint32_t fine_bucket(uint32_t c) {
     // (no branches: the bits of c converted to fp32 toward zero are its exponent followed by the bits behind the
     // leading one, so a shift leaves exponent and m bits, and the octave's first bucket is a constant away)
     const uint32_t bits = __float_as_uint(__uint2float_rz(c));
-    const bool lo = c < (1u << 14), mid = c < (1u << 26);
-    const uint32_t sh = lo ? 15u : mid ? 16u : 17u;                    // 23 - m
-    const uint32_t off = lo ? 34048u : mid ? 16000u : 6208u;           // ((127 + first e) << m) - first bucket of the range
-    return c < (uint32_t)kExact ? c : (bits >> sh) - off;
+    const bool lo = c < (1u << 14), mid = c < (1u << 18);
+    const uint32_t sh = lo ? 14u : mid ? 16u : 18u;                    // 23 - m
+    const uint32_t off = lo ? 69120u : mid ? 14976u : 1056u;           // ((127 + first e) << m) - first bucket of the range
+    return c < (uint32_t)kExact ? c : (bits >> sh) - off;              // 1024..3071 | 3072..3583 | 3584..4031
 }
 
 // Radix select (Eq. 1, Top-K(c,k)): one pass of bucket counts finds the bucket that holds the K-th key;
