@@ -5,7 +5,7 @@
  *   offline  : token-frequency counting (Algorithm 1), selection of the K most frequent target
  *              vocabulary ids and reconstruction of the drafter LM head (Eq. 1);
  *   online   : the drafter's trimmed LM head with its token sampling and the index mapper back
- *              to the target vocabulary (Algorithm 2, lines 5-6).
+ *              to the target vocabulary (Algorithm 2, the drafter-forward and index-mapping steps).
  *
  * Conventions (all entry points unless stated otherwise)
  *   - Every data pointer is a DEVICE pointer owned by the caller.  Entry points whose name ends
@@ -255,7 +255,7 @@ vt_status vt_trim_head(const uint16_t *W_full, const int32_t *map, uint16_t *W_t
                        int32_t K, int32_t d, void *ws, void *stream);
 
 /*
- * Algorithm 2, lines 5-6, head part: logits = h W_trim^T (bf16 inputs, fp32 accumulation),
+ * Algorithm 2 (drafter forward over the trimmed head, then the index mapping), head part: logits = h W_trim^T (bf16 inputs, fp32 accumulation),
  * z = logits / T_b, log-softmax statistics, the `topk` best candidates per row, a Gumbel-max
  * draw argmax_j (z_j - log(-log u_bj)) and the index mapper T_{d->t} (trimmed index -> target id).
  * Logits never leave the chip.
@@ -293,7 +293,7 @@ vt_status vt_draft_head_overlapped(const uint16_t *h, const uint16_t *W_trim, co
 /*
  * One tree depth in one call: vt_draft_head_overlapped followed by vt_tree_expand on its candidates
  * (out_ids / out_logprobs columns 1..topk), with the same arguments, results and limits as those two
- * (Algorithm 2 lines 5-6 with the draft tree of Section 4.1).  For the streaming kernel's shapes
+ * (Algorithm 2, the drafter-forward and index-mapping steps with the draft tree of Section 4.1).  For the streaming kernel's shapes
  * (B <= 16) the expansion runs inside the head kernel, in the CTA that merges the rows, so a tree
  * depth costs one launch; other shapes chain the expansion kernel behind the merge.  The caller's
  * promise about W_trim is that of vt_draft_head_overlapped.

@@ -90,7 +90,7 @@ def histogram(ids, V: int, counts=None):
 
 
 def select_topk(counts, K: int):
-    """Eq. 1, line 1.  Returns (map int32 [K] in rank order, inv_map int32 [V])."""
+    """Eq. 1 (token selection).  Returns (map int32 [K] in rank order, inv_map int32 [V])."""
     counts = _c(counts, np.uint64)
     V = counts.size
     m = np.empty(K, dtype=np.int32)
@@ -136,7 +136,7 @@ def build_vocab(ids, V: int, K: int):
 
 
 def trim_head(W_full, map_):
-    """Eq. 1, line 2.  W_full: bf16 bit patterns [V,d]; returns bit patterns [K,d]."""
+    """Eq. 1 (head restriction).  W_full: bf16 bit patterns [V,d]; returns bit patterns [K,d]."""
     W_full = _bits(W_full)
     map_ = _c(map_, np.int32)
     K, d = map_.size, W_full.shape[1]
@@ -189,7 +189,7 @@ class DraftHeadResult:
 
 
 def draft_head(h, W_trim, map_, temp, topk: int, uniforms=None, want_full: bool = True):
-    """Algorithm 2 lines 5-6, head part.  h [B,d], W_trim [K,d] as bf16 bit patterns; map_ int32
+    """Algorithm 2 (drafter forward over the trimmed head, then the index mapping), head part.  h [B,d], W_trim [K,d] as bf16 bit patterns; map_ int32
     [K] or None (identity); temp fp32 [B]; uniforms fp32 [B,K] or None.  Returns ids/logprobs of
     shape [B,1+topk] plus (when want_full) logits, z, lse and Gumbel scores for margin checks."""
     h, W_trim = _bits(h), _bits(W_trim)

@@ -188,7 +188,7 @@ void orc_trim_head(const uint16_t *W_full, const int32_t *map, int32_t K, int32_
 }
 
 /*
- * Algorithm 2, line 5 (drafter forward with the trimmed head), head part only: the LM head is
+ * Algorithm 2, the drafter forward with the trimmed head, head part only: the LM head is
  * a linear projection without bias, logit[b][j] = sum_i h[b][i] * W[j][i], summed in index
  * order in fp64 on exactly-decoded bf16 operands.  logits is [B,K] row-major.
  */
@@ -276,7 +276,7 @@ int32_t orc_gumbel_row(const double *z, const float *u, int32_t K, double *score
 }
 
 /*
- * Algorithm 2 lines 5-6, head part: projection, temperature softmax, top-k candidates, Gumbel
+ * Algorithm 2 (drafter forward over the trimmed head, then the index mapping), head part: projection, temperature softmax, top-k candidates, Gumbel
  * draw, then the index mapper T_{d->t}: every reported trimmed index j becomes map[j]
  * (map == NULL means the identity, i.e. the untrimmed head).
  *

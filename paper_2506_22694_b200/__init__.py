@@ -179,7 +179,7 @@ def vt_histogram_folded(ids: torch.Tensor, V: int, bins: int, counts: torch.Tens
 
 
 def vt_select_topk(counts: torch.Tensor, K: int, ws: Workspace | None = None):
-    """Eq. 1, line 1.  counts [V] -> (map int32 [K], inv_map int32 [V])."""
+    """Eq. 1 (token selection).  counts [V] -> (map int32 [K], inv_map int32 [V])."""
     _dev(counts, torch.int32, "counts")
     V = counts.numel()
     map_ = torch.empty(K, dtype=torch.int32, device=counts.device)
@@ -330,7 +330,7 @@ def vt_select_topk_static(counts: torch.Tensor, K: int, out=None):
 
 
 def vt_build_vocab(ids: torch.Tensor, V: int, K: int, ws: Workspace | None = None):
-    """Algorithm 1 + Eq. 1, line 1.  Device ids -> (map [K], inv_map [V]).  A CPU (ideally pinned)
+    """Algorithm 1 + Eq. 1 (token selection).  Device ids -> (map [K], inv_map [V]).  A CPU (ideally pinned)
     ids tensor goes through vt_build_vocab_host, which streams it to the device in chunks."""
     if not ids.is_cuda:
         return vt_build_vocab_host(ids, V, K, ws)
@@ -359,7 +359,7 @@ def vt_build_vocab_host(ids_host: torch.Tensor, V: int, K: int, ws: Workspace | 
 
 def vt_trim_head(W_full: torch.Tensor, map_: torch.Tensor, W_trim: torch.Tensor | None = None,
                  ws: Workspace | None = None) -> torch.Tensor:
-    """Eq. 1, line 2.  W_full bf16 [V,d], map int32 [K] -> W_trim bf16 [K,d]."""
+    """Eq. 1 (head restriction).  W_full bf16 [V,d], map int32 [K] -> W_trim bf16 [K,d]."""
     _dev(W_full, torch.bfloat16, "W_full")
     _dev(map_, torch.int32, "map")
     V, d = W_full.shape
@@ -375,7 +375,7 @@ def vt_trim_head(W_full: torch.Tensor, map_: torch.Tensor, W_trim: torch.Tensor 
 def vt_draft_head(h: torch.Tensor, W_trim: torch.Tensor, map_: torch.Tensor | None, temp: torch.Tensor,
                   topk: int, uniforms: torch.Tensor | None = None, ws: Workspace | None = None,
                   out=None, debug: bool = False, overlapped: bool = False):
-    """Algorithm 2, lines 5-6 (head part).  Returns (out_ids int32 [B,1+topk], out_logprobs fp32
+    """Algorithm 2 (the drafter's head over the trimmed vocabulary and the index mapping; head part).  Returns (out_ids int32 [B,1+topk], out_logprobs fp32
     [B,1+topk]); with debug=True also (logits fp32 [B,K], lse fp32 [B]).  overlapped=True uses
     vt_draft_head_overlapped (drafting loops with static weights; see the header)."""
     _dev(h, torch.bfloat16, "h")

@@ -1,5 +1,5 @@
 // Batched-serving head (17 <= B <= 256 hidden rows): the projection is a real dense contraction
-// and runs on the 5th-generation tensor cores (Algorithm 2, lines 5-6, with many sequences and
+// and runs on the 5th-generation tensor cores (Algorithm 2, the drafter-forward and index-mapping steps, with many sequences and
 // tree nodes drafted at once).
 //
 //   D[b, j] = sum_i h[b, i] * W_trim[j, i]      M = hidden rows (the TMEM lanes), N = vocabulary rows

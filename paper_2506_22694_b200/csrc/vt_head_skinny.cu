@@ -1,5 +1,5 @@
 // Trimmed LM head for a few hidden rows (B <= 16), fused with its sampling epilogue
-// (Algorithm 2, lines 5-6: drafter head over the trimmed vocabulary, then the index mapper).
+// (Algorithm 2, the drafter-forward and index-mapping steps: drafter head over the trimmed vocabulary, then the index mapper).
 //
 // HBM-bound: the only large operand is W_trim [K,d] bf16, read exactly once.  One persistent CTA
 // per SM owns a contiguous slab of vocabulary rows and streams it through a shared-memory ring

@@ -1,4 +1,4 @@
-"""GPU parity of the trimmed drafter head (Algorithm 2, lines 5-6) against the fp64 CPU oracle on
+"""GPU parity of the trimmed drafter head (Algorithm 2, the drafter-forward and index-mapping steps) against the fp64 CPU oracle on
 seeded synthetic inputs: logits, log-probabilities, greedy / top-k / Gumbel ids and the remap."""
 import numpy as np
 import pytest

@@ -57,7 +57,7 @@ def test_histogram_accumulates_over_chunks():
     assert np.array_equal(whole, part)
 
 
-# ----------------------------------------------------------------------------- top-K (Eq. 1, line 1)
+# ----------------------------------------------------------------------------- top-K (Eq. 1 (token selection))
 def _rank_by_definition(counts):
     """rank(v) = #{u : c_u > c_v or (c_u == c_v and u < v)} -- no sort involved."""
     V = len(counts)
@@ -131,7 +131,7 @@ def test_topk_K_equals_V_is_a_permutation():
     assert m.tolist() == [0, 1, 2, 3] and inv.tolist() == [0, 1, 2, 3]
 
 
-# ----------------------------------------------------------------------------- gather (Eq. 1, line 2)
+# ----------------------------------------------------------------------------- gather (Eq. 1 (head restriction))
 def test_trim_head_is_a_bit_copy_of_the_mapped_rows():
     W = _bits(vt_inputs.gaussian_bf16((50, 24), 0.02, seed=2))
     m = np.array([7, 0, 49, 7, 13], dtype=np.int32)
@@ -143,7 +143,7 @@ def test_trim_head_is_a_bit_copy_of_the_mapped_rows():
     assert np.array_equal(oracle.trim_head(W, ident), W)
 
 
-# ----------------------------------------------------------------------------- logits (Algorithm 2, line 5)
+# ----------------------------------------------------------------------------- logits (Algorithm 2, drafter forward)
 def test_logits_match_numpy_fp64_matmul_nonsquare():
     h = _bits(vt_inputs.gaussian_bf16((3, 40), 1.0, seed=4))
     W = _bits(vt_inputs.gaussian_bf16((17, 40), 0.02, seed=5))
